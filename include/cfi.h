@@ -1,0 +1,190 @@
+/*
+ * cfi — condensed constant-fan-in sparse linear layer, forward pass, for NVIDIA B200 (sm_100a).
+ *
+ * The layer is the one of "Dynamic Sparse Training with Structured Sparsity" (SRigL), Sec. 4.4 and
+ * appendix "Condensed matrix multiplication": every non-ablated output neuron keeps exactly k incoming
+ * weights, stored as two n_active x k arrays (values, column indices), and
+ *
+ *     y[b, o] = act( bias[o] + sum_{j<k} values[r, j] * x[b, indices[r, j]] )   if o = active_rows[r]
+ *     y[b, o] = act( bias[o] )                                                  if o is ablated
+ *
+ * (Algorithm 1 is the bias = 0, act = identity case; an ablated neuron has all incoming weights pruned,
+ * Sec. 3.1 step 4, so only its bias is left.)
+ *
+ * Conventions
+ *   - Plain C ABI.  No call throws; every call returns a cfi_status_t (cfi_status_string() names it).
+ *   - "host" / "device" in a parameter comment says where the pointer must live.
+ *   - The caller owns every array it passes, before and after the call.  The library owns a layer's
+ *     device memory from cfi_create until cfi_destroy.
+ *   - All matrices are row-major and dense in memory (no padding between rows).
+ *   - A layer is read-only after creation: cfi_forward may run concurrently on several streams.
+ *   - The library has no CPU implementation of the forward: without a CUDA device every device call
+ *     returns CFI_ERR_CUDA.
+ */
+#ifndef CFI_H_
+#define CFI_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cfi_layer cfi_layer_t;  /* opaque */
+typedef struct cfi_stack cfi_stack_t;  /* opaque */
+typedef struct CUstream_st* cfi_stream_t; /* same type as cudaStream_t; NULL = the default stream */
+
+typedef enum {
+    CFI_OK = 0,
+    CFI_ERR_NULL = 1,                /* a required pointer was NULL                                  */
+    CFI_ERR_SHAPE = 2,               /* a size is negative or inconsistent (k > in, n_active > out..) */
+    CFI_ERR_NOT_CONSTANT_FAN_IN = 3, /* cfi_pack: two non-empty rows keep different numbers of weights */
+    CFI_ERR_INDEX_RANGE = 4,         /* a column index or row number is out of range or repeated      */
+    CFI_ERR_BUFFER_TOO_SMALL = 5,    /* batch larger than what a stack or staging buffer was sized for */
+    CFI_ERR_DTYPE = 6,               /* unknown dtype / activation / variant, or layers do not chain   */
+    CFI_ERR_ALLOC = 7,               /* host or device allocation failed                               */
+    CFI_ERR_CUDA = 8,                /* a CUDA runtime call or kernel launch failed                    */
+    CFI_ERR_DEVICE_FLAG = 9,         /* a kernel recorded an error in the layer's device status word   */
+    CFI_ERR_ALIGNMENT = 10           /* x or y is not aligned to 16 bytes                              */
+} cfi_status_t;
+
+/* Storage type of values, x and y.  Products are exact in fp32 and accumulation is always fp32. */
+typedef enum { CFI_F32 = 0, CFI_BF16 = 1 } cfi_dtype_t;
+
+/* CFI_ACT_GELU_ERF is the exact GELU v * Phi(v) = 0.5 v (1 + erf(v / sqrt 2)), applied to every output,
+ * ablated ones included.  The paper does not write the activation; its ViT MLP blocks use GELU. */
+typedef enum { CFI_ACT_NONE = 0, CFI_ACT_GELU_ERF = 1 } cfi_act_t;
+
+/* Kernel choice for cfi_forward_variant (tests and benchmarks; cfi_forward uses CFI_VARIANT_AUTO). */
+typedef enum {
+    CFI_VARIANT_AUTO = 0,
+    CFI_VARIANT_SIMPLE = 1,   /* one thread per output element, no staging: a cross-check, not fast      */
+    CFI_VARIANT_SPLITK = 2,   /* small batch: lanes split a row's k terms, x staged in shared memory     */
+    CFI_VARIANT_BATCH = 3     /* large batch: lanes own batch columns, x tile transposed in shared memory */
+} cfi_variant_t;
+
+const char* cfi_status_string(cfi_status_t s);
+
+/*
+ * cfi_pack — dense masked weight -> condensed arrays.  Host only, no CUDA involved.
+ * (Appendix "Condensed matrix multiplication": values and column indices as two n x k arrays, Eq. 2:
+ *  k distinct columns per row; Sec. 4.4: ablated neurons and zero weights are removed.)
+ *
+ *   w_dense      host, float  [out_features, in_features]
+ *   mask         host, uint8  [out_features, in_features], non-zero = kept; or NULL, in which case an
+ *                entry is kept iff w_dense != 0 (so -0.0 counts as pruned).  With a mask, a kept entry
+ *                whose value is 0.0 still counts as one of the row's k.
+ *   k, n_active  host, written on every successful call
+ *   values       host, float  [n_active, k]   } all three NULL: size query only
+ *   indices      host, int32  [n_active, k]   } all three non-NULL: filled; the caller sized them from
+ *   active_rows  host, int32  [n_active]      } an earlier size query
+ *
+ * A row that keeps nothing is ablated.  Every other row must keep the same number k >= 1 of entries,
+ * otherwise CFI_ERR_NOT_CONSTANT_FAN_IN.  Output order is fixed: columns ascend within a row, rows
+ * ascend in active_rows, so the result is unique.  If every row is ablated, k = 0 and n_active = 0.
+ */
+cfi_status_t cfi_pack(const float* w_dense, const uint8_t* mask, int32_t out_features, int32_t in_features,
+                      int32_t* k, int32_t* n_active, float* values, int32_t* indices, int32_t* active_rows);
+
+/*
+ * cfi_create — build a device-resident layer from condensed arrays (the inputs w and indx of
+ * Algorithm 1, plus the bias that Sec. 4.4 extracts with the weights).
+ *
+ *   values       host, float [n_active, k]; stored on the device as `dtype` (bf16: round to nearest even)
+ *   indices      host, int32 [n_active, k], each in [0, in_features); any order; a repeated column in a
+ *                row is allowed and simply adds, as Algorithm 1 would
+ *   active_rows  host, int32 [n_active], distinct, each in [0, out_features); any order
+ *   bias         host, float [out_features] or NULL (zero bias = Algorithm 1 as printed); kept in fp32
+ *   dtype, act   see the enums
+ *   layer        receives the new layer; destroy it with cfi_destroy
+ *
+ * Requires 0 <= n_active <= out_features, 0 <= k <= in_features (k >= 1 if n_active > 0),
+ * in_features <= 2^20.  The arrays are copied; the caller may free them after the call.
+ * The layer lives on the CUDA device that is current when cfi_create is called.
+ */
+cfi_status_t cfi_create(const float* values, const int32_t* indices, const int32_t* active_rows, const float* bias,
+                        int32_t n_active, int32_t k, int32_t in_features, int32_t out_features,
+                        cfi_dtype_t dtype, cfi_act_t act, cfi_layer_t** layer);
+
+/*
+ * cfi_forward — y = layer(x) for `batch` rows (Algorithm 1 with bias, ablated rows and activation).
+ *
+ *   x       device, [batch, in_features]  of the layer's dtype, 16-byte aligned
+ *   y       device, [batch, out_features] of the layer's dtype, 16-byte aligned; must not overlap x
+ *   stream  the work is enqueued on this stream; the call does not synchronise
+ *
+ * Every element of y is written (ablated columns too).  batch == 0 succeeds and launches nothing.
+ * The return value reports argument and launch errors only.
+ */
+cfi_status_t cfi_forward(const cfi_layer_t* layer, const void* x, void* y, int32_t batch, cfi_stream_t stream);
+
+/* As cfi_forward with the kernel chosen by the caller.  A variant that cannot run the given shape
+ * (e.g. not enough shared memory) returns CFI_ERR_SHAPE rather than falling back. */
+cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void* x, void* y, int32_t batch,
+                                 cfi_stream_t stream, cfi_variant_t variant);
+
+/*
+ * cfi_forward_host — the same operation for a caller whose activations live in host memory.
+ *
+ *   x_host  host (pinned memory makes the copies asynchronous), [batch, in_features]  of the layer's dtype
+ *   y_host  host, [batch, out_features] of the layer's dtype
+ *
+ * Copies x to a device staging buffer owned by the layer, runs cfi_forward, copies y back, all on
+ * `stream`, then waits for the stream.  The staging buffers grow on demand (a cudaMalloc on the first
+ * call and whenever batch exceeds every earlier batch), so this entry point is NOT safe to call
+ * concurrently on the same layer.
+ */
+cfi_status_t cfi_forward_host(cfi_layer_t* layer, const void* x_host, void* y_host, int32_t batch,
+                              cfi_stream_t stream);
+
+/* Layer facts for reports: what the forward streams from memory. */
+typedef struct {
+    int32_t in_features, out_features, n_active, k;
+    int32_t dtype, act;
+    int32_t k_padded;            /* row length of the small-batch device layout (multiple of 4 or 8)    */
+    int32_t batch_slab_columns;  /* columns of x per shared-memory slab in the large-batch kernel        */
+    int32_t batch_row_stride;    /* padded row length of the large-batch device layout                   */
+    int32_t reserved;
+    int64_t weight_bytes_splitk; /* bytes of values+indices the small-batch kernel reads per pass        */
+    int64_t weight_bytes_batch;  /* bytes of values+columns the large-batch kernel reads per batch tile  */
+    int64_t device_bytes;        /* device memory held by the layer                                      */
+} cfi_layer_info_t;
+
+cfi_status_t cfi_layer_info(const cfi_layer_t* layer, cfi_layer_info_t* info);
+
+/* Which variant cfi_forward would run for this batch size (written to *variant). */
+cfi_status_t cfi_choose_variant(const cfi_layer_t* layer, int32_t batch, int32_t* variant);
+
+/*
+ * cfi_device_status — waits for `stream`, then reads the layer's device status word into *flag.
+ * 0 means no kernel of this layer has recorded an error since creation; non-zero returns
+ * CFI_ERR_DEVICE_FLAG as well.  Kernels never trap: a failed internal check records a code and returns.
+ */
+cfi_status_t cfi_device_status(const cfi_layer_t* layer, cfi_stream_t stream, int32_t* flag);
+
+/* Frees the layer's device and host memory.  No work using the layer may still be in flight. NULL is OK. */
+cfi_status_t cfi_destroy(cfi_layer_t* layer);
+
+/*
+ * cfi_stack_* — a chain of layers y = L_{n-1}( ... L_1(L_0(x)) ), e.g. the MLP blocks of a transformer
+ * (768 -> 3072 with GELU, 3072 -> 768) whose linears are the layers the paper condenses (Sec. 4.4,
+ * appendix "Condensed linear CPU benchmark details").  Layer i+1 consumes layer i's output directly:
+ * no residual, normalisation or attention in between.
+ *
+ *   layers     host array of n_layers layer handles; out_features of layer i must equal in_features of
+ *              layer i+1 and all dtypes must match, else CFI_ERR_DTYPE / CFI_ERR_SHAPE.  The stack
+ *              borrows the layers: they must outlive it and are not destroyed with it.
+ *   max_batch  the two intermediate activation buffers (device, owned by the stack) are sized for it
+ *
+ * cfi_stack_forward enqueues the n_layers forwards on `stream` without synchronising; batch above
+ * max_batch returns CFI_ERR_BUFFER_TOO_SMALL.  One stack must not run on two streams at once (the
+ * intermediates are shared).
+ */
+cfi_status_t cfi_stack_create(cfi_layer_t* const* layers, int32_t n_layers, int32_t max_batch, cfi_stack_t** stack);
+cfi_status_t cfi_stack_forward(const cfi_stack_t* stack, const void* x, void* y, int32_t batch, cfi_stream_t stream);
+cfi_status_t cfi_stack_destroy(cfi_stack_t* stack);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CFI_H_ */
