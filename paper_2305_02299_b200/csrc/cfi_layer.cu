@@ -1,0 +1,836 @@
+// Device side of the library: layer construction, the forward kernels and their launch logic.
+//
+// Two device layouts are built from the caller's condensed arrays (values / column indices, both
+// n_active x k, as in the paper's appendix "Condensed matrix multiplication"):
+//
+//   small-batch ("split-k") layout: rows padded to a multiple of 4 (fp32) or 8 (bf16) entries so that
+//     every lane reads whole 16-byte vectors; a pad entry has weight 0 and points at one extra zero
+//     element behind the staged x, so it contributes exactly 0 even when x holds inf or NaN.
+//
+//   large-batch layout: columns are cut into slabs that fit shared memory; each row's entries are
+//     grouped by slab (sorting a row by column makes the groups contiguous), every group is padded
+//     to a multiple of 4, and columns are stored relative to the slab start.  seg[r][s] is the
+//     first 4-entry "quad" of row r in slab s.
+#include "cfi.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <numeric>
+#include <vector>
+
+namespace {
+
+constexpr int kBatchTile = 64;  // batch columns per CTA in the large-batch kernel
+constexpr int kSlabBytesBudget = 80 * 1024;
+
+struct DevLayer {
+    const void* values;      // [n_active][kp]  fp32 or bf16
+    const int32_t* indices;  // [n_active][kp]
+    const float* values_b;   // [n_active][stride_b]
+    const int32_t* cols_b;   // [n_active][stride_b] slab-relative column (cs = zero row)
+    const int32_t* seg;      // [n_active][n_slabs + 1] quad offsets
+    const float* bias;       // [out]
+    const int32_t* slot;     // [out] -> row of the condensed arrays, or -1 if ablated
+    int32_t* status;
+    int in, out, n_active, k, kp, act;
+    int cs, n_slabs, stride_b;
+};
+
+}  // namespace
+
+struct cfi_layer {
+    DevLayer d{};
+    int dtype = 0, device = 0, sm_count = 0, smem_optin = 0;
+    int64_t device_bytes = 0;
+    std::vector<void*> allocs;
+    void* stage_x = nullptr;
+    void* stage_y = nullptr;
+    int staged_batch = 0;
+};
+
+struct cfi_stack {
+    std::vector<cfi_layer*> layers;
+    void* buf[2] = {nullptr, nullptr};
+    int max_batch = 0, dtype = 0;
+};
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// device helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ void from_f32(float* p, float v) { *p = v; }
+__device__ __forceinline__ void from_f32(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+// Exact GELU v * Phi(v), the erf form.
+__device__ __forceinline__ float activate(float v, int act) {
+    return act == CFI_ACT_GELU_ERF ? 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)) : v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// CFI_VARIANT_SIMPLE: Algorithm 1's loop nest with one thread per (b, o).  Reads the split-k layout.
+// ------------------------------------------------------------------------------------------------
+template <typename VT>
+__global__ void cfi_simple_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (int64_t)batch * L.out) return;
+    const int b = (int)(t / L.out), o = (int)(t % L.out);
+    const int r = L.slot[o];
+    float s = 0.0f;
+    if (r >= 0) {
+        const VT* w = reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp;
+        const int32_t* ix = L.indices + (size_t)r * L.kp;
+        const VT* xr = x + (size_t)b * L.in;
+        for (int j = 0; j < L.k; ++j) s = fmaf(to_f32(w[j]), to_f32(xr[ix[j]]), s);
+    }
+    from_f32(&y[t], activate(s + L.bias[o], L.act));
+}
+
+// ------------------------------------------------------------------------------------------------
+// CFI_VARIANT_SPLITK: small batch.  G lanes share one output row and split its k terms; the CTA's
+// x rows sit in shared memory as xs[column][BT] (+ one zero column for pad entries).
+// ------------------------------------------------------------------------------------------------
+template <typename VT> struct Chunk;
+
+template <> struct Chunk<float> {  // 4 weights + 4 columns
+    static constexpr int VEC = 4;
+    float4 w;
+    int4 c;
+    __device__ __forceinline__ void load(const void* values, const int32_t* indices, size_t row_off, int v, bool pred,
+                                         int pad_col) {
+        if (pred) {
+            w = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(values) + row_off) + v);
+            c = __ldg(reinterpret_cast<const int4*>(indices + row_off) + v);
+        } else {
+            w = make_float4(0.f, 0.f, 0.f, 0.f);
+            c = make_int4(pad_col, pad_col, pad_col, pad_col);
+        }
+    }
+    __device__ __forceinline__ float weight(int e) const { return e == 0 ? w.x : e == 1 ? w.y : e == 2 ? w.z : w.w; }
+    __device__ __forceinline__ int col(int e) const { return e == 0 ? c.x : e == 1 ? c.y : e == 2 ? c.z : c.w; }
+};
+
+template <> struct Chunk<__nv_bfloat16> {  // 8 weights + 8 columns
+    static constexpr int VEC = 8;
+    uint4 w;
+    int4 c0, c1;
+    __device__ __forceinline__ void load(const void* values, const int32_t* indices, size_t row_off, int v, bool pred,
+                                         int pad_col) {
+        if (pred) {
+            w = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(values) + row_off) + v);
+            c0 = __ldg(reinterpret_cast<const int4*>(indices + row_off) + 2 * v);
+            c1 = __ldg(reinterpret_cast<const int4*>(indices + row_off) + 2 * v + 1);
+        } else {
+            w = make_uint4(0u, 0u, 0u, 0u);
+            c0 = c1 = make_int4(pad_col, pad_col, pad_col, pad_col);
+        }
+    }
+    __device__ __forceinline__ float weight(int e) const {
+        const uint32_t u = (e >> 1) == 0 ? w.x : (e >> 1) == 1 ? w.y : (e >> 1) == 2 ? w.z : w.w;
+        return (e & 1) ? bf16_hi(u) : bf16_lo(u);
+    }
+    __device__ __forceinline__ int col(int e) const {
+        const int4& q = e < 4 ? c0 : c1;
+        const int f = e & 3;
+        return f == 0 ? q.x : f == 1 ? q.y : f == 2 ? q.z : q.w;
+    }
+};
+
+template <int BT>
+__device__ __forceinline__ void gather_fma(float (&acc)[BT], const float* xs, int col, float w) {
+    const float* p = xs + (size_t)col * BT;
+    if constexpr (BT == 1) {
+        acc[0] = fmaf(w, p[0], acc[0]);
+    } else if constexpr (BT == 2) {
+        const float2 v = *reinterpret_cast<const float2*>(p);
+        acc[0] = fmaf(w, v.x, acc[0]);
+        acc[1] = fmaf(w, v.y, acc[1]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < BT / 4; ++q) {
+            const float4 v = *reinterpret_cast<const float4*>(p + 4 * q);
+            acc[4 * q + 0] = fmaf(w, v.x, acc[4 * q + 0]);
+            acc[4 * q + 1] = fmaf(w, v.y, acc[4 * q + 1]);
+            acc[4 * q + 2] = fmaf(w, v.z, acc[4 * q + 2]);
+            acc[4 * q + 3] = fmaf(w, v.w, acc[4 * q + 3]);
+        }
+    }
+}
+
+constexpr int kSplitkUnroll = 4;  // 16-byte vector pairs in flight per lane
+
+template <typename VT, int BT, int G>
+__global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch,
+                                  int rows_per_group) {
+    extern __shared__ __align__(16) float xs_f32[];  // [(in + 1)][BT]
+    float* xs = xs_f32;
+    using CK = Chunk<VT>;
+    constexpr int U = kSplitkUnroll;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int b0 = blockIdx.y * BT;
+    const int nb = min(BT, batch - b0);
+
+    // Stage the CTA's x rows, widened to fp32, transposed to [column][b].
+    if (BT == 1 && sizeof(VT) == 4 && (L.in & 3) == 0) {
+        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(x) + (size_t)b0 * L.in);
+        for (int c = tid; c < (L.in >> 2); c += nthr) reinterpret_cast<float4*>(xs)[c] = __ldg(src + c);
+    } else {
+#pragma unroll
+        for (int b = 0; b < BT; ++b) {
+            if (b < nb) {
+                const VT* xr = x + (size_t)(b0 + b) * L.in;
+                for (int c = tid; c < L.in; c += nthr) xs[(size_t)c * BT + b] = to_f32(xr[c]);
+            } else {
+                for (int c = tid; c < L.in; c += nthr) xs[(size_t)c * BT + b] = 0.0f;
+            }
+        }
+    }
+    if (tid < BT) xs[(size_t)L.in * BT + tid] = 0.0f;
+
+    const int groups = nthr / G, g = tid / G, lg = tid % G;
+    const int nvec = L.kp / CK::VEC;
+    int o = blockIdx.x * (groups * rows_per_group) + g;
+    int r = o < L.out ? L.slot[o] : -1;
+
+    // The first vectors of the first row do not depend on x: issue them before the barrier so the
+    // weight stream and the x staging are in flight together.
+    CK ck[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int v = lg + u * G;
+        ck[u].load(L.values, L.indices, (size_t)max(r, 0) * L.kp, v, r >= 0 && v < nvec, L.in);
+    }
+    __syncthreads();
+
+    for (int i = 0;;) {
+        float acc[BT];
+#pragma unroll
+        for (int b = 0; b < BT; ++b) acc[b] = 0.0f;
+        if (r >= 0) {
+            const size_t row_off = (size_t)r * L.kp;
+            for (int v0 = lg;;) {
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int e = 0; e < CK::VEC; ++e) gather_fma<BT>(acc, xs, ck[u].col(e), ck[u].weight(e));
+                v0 += G * U;
+                if (v0 >= nvec) break;
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int v = v0 + u * G;
+                    ck[u].load(L.values, L.indices, row_off, v, v < nvec, L.in);
+                }
+            }
+        }
+        // Finish the k-sum across the G lanes of the group.
+#pragma unroll
+        for (int b = 0; b < BT; ++b) {
+            float v = acc[b];
+#pragma unroll
+            for (int m = G >> 1; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+            acc[b] = v;
+        }
+        if (lg == 0 && o < L.out) {
+            const float bias = L.bias[o];
+#pragma unroll
+            for (int b = 0; b < BT; ++b)
+                if (b < nb) from_f32(&y[(size_t)(b0 + b) * L.out + o], activate(acc[b] + bias, L.act));
+        }
+        if (++i >= rows_per_group) break;
+        o += groups;
+        r = o < L.out ? L.slot[o] : -1;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int v = lg + u * G;
+            ck[u].load(L.values, L.indices, (size_t)max(r, 0) * L.kp, v, r >= 0 && v < nvec, L.in);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// CFI_VARIANT_BATCH: large batch.  A CTA owns `rt` consecutive output rows x 64 batch columns.  Per
+// column slab it stages x transposed as xs[column][64] (so one column index yields 64 contiguous
+// batch values), then every 16-lane half-warp walks one row's entries of that slab: (weight, column)
+// are the same for the 16 lanes, each lane gathers its 4 batch values with one 16-byte (fp32) or
+// 8-byte (bf16) shared-memory load and does 4 FMAs.  Partial sums sit in ys[b][row] between slabs and
+// are written out row-contiguously at the end.
+//
+// Within a staged row the sixteen 4-value units are permuted by unit ^ (column & 15).  The staging
+// warp covers 8 consecutive columns x 4 batch rows (whole 32-byte sectors of x) and its stores then
+// fall into 32 different banks; the reading half-warp still sees each quarter in distinct banks.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int swz(int col, int unit) { return (col * (kBatchTile / 4) + (unit ^ (col & 15))) << 2; }
+
+template <typename XT> struct SmemRow;
+template <> struct SmemRow<float> {
+    static __device__ __forceinline__ void fma4(float (&a)[4], const float* xs, int col, int ll, float w) {
+        const float4 v = *reinterpret_cast<const float4*>(xs + swz(col, ll));
+        a[0] = fmaf(w, v.x, a[0]);
+        a[1] = fmaf(w, v.y, a[1]);
+        a[2] = fmaf(w, v.z, a[2]);
+        a[3] = fmaf(w, v.w, a[3]);
+    }
+};
+template <> struct SmemRow<__nv_bfloat16> {
+    static __device__ __forceinline__ void fma4(float (&a)[4], const __nv_bfloat16* xs, int col, int ll, float w) {
+        const uint2 v = *reinterpret_cast<const uint2*>(xs + swz(col, ll));
+        a[0] = fmaf(w, bf16_lo(v.x), a[0]);
+        a[1] = fmaf(w, bf16_hi(v.x), a[1]);
+        a[2] = fmaf(w, bf16_lo(v.y), a[2]);
+        a[3] = fmaf(w, bf16_hi(v.y), a[3]);
+    }
+};
+
+template <typename VT>
+__global__ void cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch, int rt) {
+    constexpr int BT = kBatchTile, LPR = BT / 4, RPW = 32 / LPR;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    VT* xs = reinterpret_cast<VT*>(smem_raw);  // [(cs + 1)][BT], units swizzled
+    const int pitch = rt | 1;                  // odd: spreads banks
+    float* ys = reinterpret_cast<float*>(smem_raw + (((size_t)(L.cs + 1) * BT * sizeof(VT) + 15) & ~(size_t)15));
+
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int b0 = blockIdx.y * BT, nb = min(BT, batch - b0);
+    const int o0 = blockIdx.x * rt, nrows = min(rt, L.out - o0);
+    const int lane = tid & 31, sub = lane / LPR, ll = lane % LPR;
+    const int row_step = (nthr >> 5) * RPW;
+
+    if (tid < BT) xs[(size_t)L.cs * BT + tid] = VT(0.0f);  // the zero row that pad entries point at
+
+    for (int s = 0; s < L.n_slabs; ++s) {
+        const int c0 = s * L.cs, ncol = min(L.cs, L.in - c0);
+        if (s) __syncthreads();  // everyone is done reading the previous slab
+        // Stage: element e <-> (column block of 8, batch block of 4, batch row in block, column in block).
+        const int total = ((ncol + 7) >> 3) * (BT / 4) * 32;
+        for (int e = tid; e < total; e += nthr) {
+            const int cl = e & 7, bl = (e >> 3) & 3, t = e >> 5;
+            const int bblk = t % (BT / 4), c = (t / (BT / 4)) * 8 + cl, b = bblk * 4 + bl;
+            if (c < ncol) xs[swz(c, bblk) + bl] = b < nb ? x[(size_t)(b0 + b) * L.in + c0 + c] : VT(0.0f);
+        }
+        __syncthreads();
+
+        for (int i = (tid >> 5) * RPW + sub; i < nrows; i += row_step) {
+            const int r = L.slot[o0 + i];
+            float acc[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[e] = s ? ys[(size_t)(4 * ll + e) * pitch + i] : 0.0f;
+            if (r >= 0) {
+                const int q0 = L.seg[(size_t)r * (L.n_slabs + 1) + s], q1 = L.seg[(size_t)r * (L.n_slabs + 1) + s + 1];
+                const float4* wq = reinterpret_cast<const float4*>(L.values_b + (size_t)r * L.stride_b);
+                const int4* cq = reinterpret_cast<const int4*>(L.cols_b + (size_t)r * L.stride_b);
+#pragma unroll 2
+                for (int q = q0; q < q1; ++q) {
+                    const float4 w = __ldg(wq + q);
+                    const int4 c = __ldg(cq + q);
+                    SmemRow<VT>::fma4(acc, xs, c.x, ll, w.x);
+                    SmemRow<VT>::fma4(acc, xs, c.y, ll, w.y);
+                    SmemRow<VT>::fma4(acc, xs, c.z, ll, w.z);
+                    SmemRow<VT>::fma4(acc, xs, c.w, ll, w.w);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) ys[(size_t)(4 * ll + e) * pitch + i] = acc[e];
+        }
+    }
+    __syncthreads();
+    // Epilogue: consecutive threads write consecutive output rows of one batch row.
+    for (int e = tid; e < nb * nrows; e += nthr) {
+        const int b = e / nrows, i = e - b * nrows;
+        const float v = ys[(size_t)b * pitch + i] + L.bias[o0 + i];
+        from_f32(&y[(size_t)(b0 + b) * L.out + o0 + i], activate(v, L.act));
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host: launch shapes
+// ------------------------------------------------------------------------------------------------
+struct SplitkShape { int bt, g, threads, rows_per_group, grid_x, grid_y; size_t smem; };
+struct BatchShape { int threads, rt, grid_x, grid_y; size_t smem; };
+
+int vec_of(int dtype) { return dtype == CFI_BF16 ? 8 : 4; }
+
+SplitkShape splitk_shape(const cfi_layer* l, int batch) {
+    SplitkShape s{};
+    s.bt = batch >= 8 ? 8 : batch >= 3 ? 4 : batch == 2 ? 2 : 1;
+    while (s.bt > 1 && (size_t)(l->d.in + 1) * s.bt * 4 > (size_t)l->smem_optin) s.bt >>= 1;
+    const int nvec = l->d.kp / vec_of(l->dtype);
+    s.g = 4;
+    while (s.g < 32 && s.g * kSplitkUnroll < nvec) s.g <<= 1;
+    // Enough CTAs to cover the SMs a few times over, but no more x staging than needed.
+    const int64_t lanes = (int64_t)l->d.out * s.g;
+    s.threads = lanes >= (int64_t)l->sm_count * 4 * 256 ? 256 : 128;
+    const int groups = s.threads / s.g;
+    const int ctas_one_row_each = (l->d.out + groups - 1) / groups;
+    const int target = l->sm_count * 4;
+    s.rows_per_group = std::max(1, (ctas_one_row_each + target - 1) / target);
+    s.grid_x = (l->d.out + groups * s.rows_per_group - 1) / (groups * s.rows_per_group);
+    s.grid_y = (batch + s.bt - 1) / s.bt;
+    s.smem = (size_t)(l->d.in + 1) * s.bt * 4;
+    return s;
+}
+
+size_t batch_smem(const cfi_layer* l, int rt) {
+    const size_t es = l->dtype == CFI_BF16 ? 2 : 4;
+    const size_t xs = (((size_t)(l->d.cs + 1) * kBatchTile * es) + 15) & ~(size_t)15;
+    return xs + (size_t)kBatchTile * (rt | 1) * 4;
+}
+
+BatchShape batch_shape(const cfi_layer* l, int batch) {
+    BatchShape s{};
+    s.threads = 256;
+    const int rows_per_pass = (s.threads / 32) * (32 / (kBatchTile / 4));
+    s.grid_y = (batch + kBatchTile - 1) / kBatchTile;
+    // One wave of two CTAs per SM when the problem is small; otherwise tall row tiles, which amortise
+    // the x staging over more rows.
+    const int slots = std::max(1, (2 * l->sm_count) / s.grid_y);
+    int rt = (l->d.out + slots - 1) / slots;
+    rt = ((rt + rows_per_pass - 1) / rows_per_pass) * rows_per_pass;
+    rt = std::max(rows_per_pass, std::min(rt, 128));
+    while (rt > rows_per_pass && 2 * (batch_smem(l, rt) + 1024) > (size_t)228 * 1024) rt -= rows_per_pass;
+    s.rt = rt;
+    s.grid_x = (l->d.out + rt - 1) / rt;
+    s.smem = batch_smem(l, rt);
+    return s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host: launches
+// ------------------------------------------------------------------------------------------------
+template <typename K>
+cfi_status_t set_smem(K kernel, size_t bytes) {
+    if (bytes > 48 * 1024) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+            cudaGetLastError();
+            return CFI_ERR_SHAPE;
+        }
+    }
+    return CFI_OK;
+}
+
+template <typename VT, int BT, int G>
+cfi_status_t launch_splitk_g(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
+                             cudaStream_t st) {
+    auto kern = cfi_splitk_kernel<VT, BT, G>;
+    if (cfi_status_t e = set_smem(kern, s.smem)) return e;
+    kern<<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, x, y, batch, s.rows_per_group);
+    return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+}
+
+template <typename VT, int BT>
+cfi_status_t launch_splitk_bt(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
+                              cudaStream_t st) {
+    switch (s.g) {
+        case 4: return launch_splitk_g<VT, BT, 4>(l, s, x, y, batch, st);
+        case 8: return launch_splitk_g<VT, BT, 8>(l, s, x, y, batch, st);
+        case 16: return launch_splitk_g<VT, BT, 16>(l, s, x, y, batch, st);
+        case 32: return launch_splitk_g<VT, BT, 32>(l, s, x, y, batch, st);
+    }
+    return CFI_ERR_SHAPE;
+}
+
+template <typename VT>
+cfi_status_t launch_splitk(const cfi_layer* l, const SplitkShape& s, const void* x, void* y, int batch,
+                           cudaStream_t st) {
+    if (s.smem > (size_t)l->smem_optin) return CFI_ERR_SHAPE;
+    const VT* xx = static_cast<const VT*>(x);
+    VT* yy = static_cast<VT*>(y);
+    switch (s.bt) {
+        case 1: return launch_splitk_bt<VT, 1>(l, s, xx, yy, batch, st);
+        case 2: return launch_splitk_bt<VT, 2>(l, s, xx, yy, batch, st);
+        case 4: return launch_splitk_bt<VT, 4>(l, s, xx, yy, batch, st);
+        case 8: return launch_splitk_bt<VT, 8>(l, s, xx, yy, batch, st);
+    }
+    return CFI_ERR_SHAPE;
+}
+
+template <typename VT>
+cfi_status_t launch_batch(const cfi_layer* l, const BatchShape& s, const void* x, void* y, int batch,
+                          cudaStream_t st) {
+    if (s.smem > (size_t)l->smem_optin) return CFI_ERR_SHAPE;
+    auto kern = cfi_batch_kernel<VT>;
+    if (cfi_status_t e = set_smem(kern, s.smem)) return e;
+    kern<<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, static_cast<const VT*>(x), static_cast<VT*>(y),
+                                                              batch, s.rt);
+    return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+}
+
+template <typename VT>
+cfi_status_t launch_simple(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
+    const int64_t total = (int64_t)batch * l->d.out;
+    const int threads = 256;
+    const int64_t blocks = (total + threads - 1) / threads;
+    if (blocks > 0x7fffffffLL) return CFI_ERR_SHAPE;
+    cfi_simple_kernel<VT><<<(unsigned)blocks, threads, 0, st>>>(l->d, static_cast<const VT*>(x), static_cast<VT*>(y),
+                                                              batch);
+    return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+}
+
+int choose_variant(const cfi_layer* l, int batch) {
+    (void)l;
+    return batch <= 8 ? CFI_VARIANT_SPLITK : CFI_VARIANT_BATCH;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host: construction
+// ------------------------------------------------------------------------------------------------
+uint16_t bf16_bits_rne(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return (uint16_t)((u >> 16) | 0x0040u);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+float bf16_widen(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+template <typename T>
+cfi_status_t upload(cfi_layer* l, const std::vector<T>& host, const T** dev) {
+    void* p = nullptr;
+    const size_t bytes = std::max<size_t>(host.size() * sizeof(T), 16);
+    if (cudaMalloc(&p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_ALLOC;
+    }
+    l->allocs.push_back(p);
+    l->device_bytes += (int64_t)bytes;
+    if (!host.empty() && cudaMemcpy(p, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
+    *dev = static_cast<const T*>(p);
+    return CFI_OK;
+}
+
+void free_layer(cfi_layer* l) {
+    for (void* p : l->allocs) cudaFree(p);
+    if (l->stage_x) cudaFree(l->stage_x);
+    if (l->stage_y) cudaFree(l->stage_y);
+    delete l;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------------
+extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, const int32_t* active_rows,
+                                   const float* bias, int32_t n_active, int32_t k, int32_t in_features,
+                                   int32_t out_features, cfi_dtype_t dtype, cfi_act_t act, cfi_layer_t** layer) {
+    if (!layer) return CFI_ERR_NULL;
+    *layer = nullptr;
+    if (dtype != CFI_F32 && dtype != CFI_BF16) return CFI_ERR_DTYPE;
+    if (act != CFI_ACT_NONE && act != CFI_ACT_GELU_ERF) return CFI_ERR_DTYPE;
+    if (n_active < 0 || k < 0 || in_features < 0 || out_features < 0) return CFI_ERR_SHAPE;
+    if (n_active > out_features || k > in_features || in_features > (1 << 20)) return CFI_ERR_SHAPE;
+    if (n_active > 0 && k < 1) return CFI_ERR_SHAPE;
+    if (n_active > 0 && (!values || !indices || !active_rows)) return CFI_ERR_NULL;
+    const size_t nnz = (size_t)n_active * (size_t)k;
+    for (size_t i = 0; i < nnz; ++i)
+        if (indices[i] < 0 || indices[i] >= in_features) return CFI_ERR_INDEX_RANGE;
+
+    std::vector<int32_t> slot((size_t)out_features, -1);
+    for (int32_t r = 0; r < n_active; ++r) {
+        const int32_t o = active_rows[r];
+        if (o < 0 || o >= out_features || slot[o] != -1) return CFI_ERR_INDEX_RANGE;
+        slot[o] = r;
+    }
+
+    cfi_layer* l = new (std::nothrow) cfi_layer();
+    if (!l) return CFI_ERR_ALLOC;
+    cudaDeviceProp prop{};
+    if (cudaGetDevice(&l->device) != cudaSuccess || cudaGetDeviceProperties(&prop, l->device) != cudaSuccess) {
+        cudaGetLastError();
+        delete l;
+        return CFI_ERR_CUDA;
+    }
+    l->sm_count = prop.multiProcessorCount;
+    l->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    l->dtype = dtype;
+    DevLayer& d = l->d;
+    d.in = in_features, d.out = out_features, d.n_active = n_active, d.k = k, d.act = act;
+
+    try {
+        // Each row sorted by column (stable, so repeated columns keep the caller's order).
+        std::vector<int32_t> order((size_t)std::max(k, 1));
+        std::vector<float> v_sorted(nnz);
+        std::vector<int32_t> c_sorted(nnz);
+        for (int32_t r = 0; r < n_active; ++r) {
+            const size_t off = (size_t)r * k;
+            std::iota(order.begin(), order.begin() + k, 0);
+            std::stable_sort(order.begin(), order.begin() + k,
+                             [&](int32_t a, int32_t b) { return indices[off + a] < indices[off + b]; });
+            for (int32_t j = 0; j < k; ++j) {
+                float w = values[off + order[j]];
+                if (dtype == CFI_BF16) w = bf16_widen(bf16_bits_rne(w));
+                v_sorted[off + j] = w;
+                c_sorted[off + j] = indices[off + order[j]];
+            }
+        }
+
+        // ---- small-batch layout
+        const int vec = vec_of(dtype);
+        d.kp = ((k + vec - 1) / vec) * vec;
+        std::vector<int32_t> idx_p((size_t)n_active * d.kp, in_features);
+        cfi_status_t st = CFI_OK;
+        if (dtype == CFI_F32) {
+            std::vector<float> val_p((size_t)n_active * d.kp, 0.0f);
+            for (int32_t r = 0; r < n_active; ++r)
+                for (int32_t j = 0; j < k; ++j) {
+                    val_p[(size_t)r * d.kp + j] = v_sorted[(size_t)r * k + j];
+                    idx_p[(size_t)r * d.kp + j] = c_sorted[(size_t)r * k + j];
+                }
+            const float* p = nullptr;
+            st = upload(l, val_p, &p);
+            d.values = p;
+        } else {
+            std::vector<uint16_t> val_p((size_t)n_active * d.kp, (uint16_t)0);
+            for (int32_t r = 0; r < n_active; ++r)
+                for (int32_t j = 0; j < k; ++j) {
+                    val_p[(size_t)r * d.kp + j] = bf16_bits_rne(v_sorted[(size_t)r * k + j]);
+                    idx_p[(size_t)r * d.kp + j] = c_sorted[(size_t)r * k + j];
+                }
+            const uint16_t* p = nullptr;
+            st = upload(l, val_p, &p);
+            d.values = p;
+        }
+        if (st == CFI_OK) st = upload(l, idx_p, &d.indices);
+
+        // ---- large-batch layout
+        const int es = dtype == CFI_BF16 ? 2 : 4;
+        const int cs_max = std::max(8, (kSlabBytesBudget / (kBatchTile * es) - 1) & ~7);
+        d.n_slabs = std::max(1, (in_features + cs_max - 1) / cs_max);
+        d.cs = std::max(8, (((in_features + d.n_slabs - 1) / d.n_slabs) + 7) & ~7);
+        d.n_slabs = std::max(1, (in_features + d.cs - 1) / d.cs);
+        std::vector<int32_t> seg((size_t)n_active * (d.n_slabs + 1), 0);
+        int max_quads = 0;
+        for (int32_t r = 0; r < n_active; ++r) {
+            int q = 0, j = 0;
+            for (int s = 0; s < d.n_slabs; ++s) {
+                seg[(size_t)r * (d.n_slabs + 1) + s] = q;
+                int cnt = 0;
+                while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) ++j, ++cnt;
+                q += (cnt + 3) / 4;
+            }
+            seg[(size_t)r * (d.n_slabs + 1) + d.n_slabs] = q;
+            max_quads = std::max(max_quads, q);
+        }
+        d.stride_b = std::max(4, max_quads * 4);
+        std::vector<float> val_b((size_t)n_active * d.stride_b, 0.0f);
+        std::vector<int32_t> col_b((size_t)n_active * d.stride_b, d.cs);
+        for (int32_t r = 0; r < n_active; ++r) {
+            int j = 0;
+            for (int s = 0; s < d.n_slabs; ++s) {
+                size_t w = (size_t)r * d.stride_b + (size_t)seg[(size_t)r * (d.n_slabs + 1) + s] * 4;
+                while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) {
+                    val_b[w] = v_sorted[(size_t)r * k + j];
+                    col_b[w] = c_sorted[(size_t)r * k + j] - s * d.cs;
+                    ++w, ++j;
+                }
+            }
+        }
+        if (st == CFI_OK) st = upload(l, val_b, &d.values_b);
+        if (st == CFI_OK) st = upload(l, col_b, &d.cols_b);
+        if (st == CFI_OK) st = upload(l, seg, &d.seg);
+
+        std::vector<float> bias_h((size_t)out_features, 0.0f);
+        if (bias) std::copy(bias, bias + out_features, bias_h.begin());
+        if (st == CFI_OK) st = upload(l, bias_h, &d.bias);
+        if (st == CFI_OK) st = upload(l, slot, &d.slot);
+        std::vector<int32_t> zero(4, 0);
+        const int32_t* status = nullptr;
+        if (st == CFI_OK) st = upload(l, zero, &status);
+        d.status = const_cast<int32_t*>(status);
+        if (st != CFI_OK) {
+            free_layer(l);
+            return st;
+        }
+    } catch (const std::bad_alloc&) {
+        free_layer(l);
+        return CFI_ERR_ALLOC;
+    }
+    *layer = l;
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_destroy(cfi_layer_t* layer) {
+    if (!layer) return CFI_OK;
+    DeviceGuard g(layer->device);
+    free_layer(layer);
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_choose_variant(const cfi_layer_t* layer, int32_t batch, int32_t* variant) {
+    if (!layer || !variant) return CFI_ERR_NULL;
+    *variant = choose_variant(layer, batch);
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void* x, void* y, int32_t batch,
+                                            cfi_stream_t stream, cfi_variant_t variant) {
+    if (!layer) return CFI_ERR_NULL;
+    if (batch < 0) return CFI_ERR_SHAPE;
+    if (batch == 0 || layer->d.out == 0) return CFI_OK;
+    if (!y || (!x && layer->d.in > 0)) return CFI_ERR_NULL;
+    if (((uintptr_t)x | (uintptr_t)y) & 15u) return CFI_ERR_ALIGNMENT;
+    int v = variant;
+    if (v == CFI_VARIANT_AUTO) v = choose_variant(layer, batch);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const bool bf = layer->dtype == CFI_BF16;
+    switch (v) {
+        case CFI_VARIANT_SIMPLE:
+            return bf ? launch_simple<__nv_bfloat16>(layer, x, y, batch, st) : launch_simple<float>(layer, x, y, batch, st);
+        case CFI_VARIANT_SPLITK: {
+            const SplitkShape s = splitk_shape(layer, batch);
+            return bf ? launch_splitk<__nv_bfloat16>(layer, s, x, y, batch, st)
+                      : launch_splitk<float>(layer, s, x, y, batch, st);
+        }
+        case CFI_VARIANT_BATCH: {
+            const BatchShape s = batch_shape(layer, batch);
+            return bf ? launch_batch<__nv_bfloat16>(layer, s, x, y, batch, st)
+                      : launch_batch<float>(layer, s, x, y, batch, st);
+        }
+    }
+    return CFI_ERR_DTYPE;
+}
+
+extern "C" cfi_status_t cfi_forward(const cfi_layer_t* layer, const void* x, void* y, int32_t batch,
+                                    cfi_stream_t stream) {
+    return cfi_forward_variant(layer, x, y, batch, stream, CFI_VARIANT_AUTO);
+}
+
+extern "C" cfi_status_t cfi_forward_host(cfi_layer_t* layer, const void* x_host, void* y_host, int32_t batch,
+                                         cfi_stream_t stream) {
+    if (!layer) return CFI_ERR_NULL;
+    if (batch < 0) return CFI_ERR_SHAPE;
+    if (batch == 0) return CFI_OK;
+    if (!y_host || (!x_host && layer->d.in > 0)) return CFI_ERR_NULL;
+    DeviceGuard g(layer->device);
+    const size_t es = layer->dtype == CFI_BF16 ? 2 : 4;
+    if (batch > layer->staged_batch) {
+        if (layer->stage_x) cudaFree(layer->stage_x);
+        if (layer->stage_y) cudaFree(layer->stage_y);
+        layer->stage_x = layer->stage_y = nullptr;
+        layer->staged_batch = 0;
+        const size_t xb = std::max<size_t>((size_t)batch * layer->d.in * es, 16);
+        const size_t yb = std::max<size_t>((size_t)batch * layer->d.out * es, 16);
+        if (cudaMalloc(&layer->stage_x, xb) != cudaSuccess || cudaMalloc(&layer->stage_y, yb) != cudaSuccess) {
+            cudaGetLastError();
+            return CFI_ERR_ALLOC;
+        }
+        layer->staged_batch = batch;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const size_t xb = (size_t)batch * layer->d.in * es, yb = (size_t)batch * layer->d.out * es;
+    if (xb && cudaMemcpyAsync(layer->stage_x, x_host, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return CFI_ERR_CUDA;
+    if (cfi_status_t e = cfi_forward(layer, layer->stage_x, layer->stage_y, batch, stream)) return e;
+    if (yb && cudaMemcpyAsync(y_host, layer->stage_y, yb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return CFI_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+}
+
+extern "C" cfi_status_t cfi_layer_info(const cfi_layer_t* layer, cfi_layer_info_t* info) {
+    if (!layer || !info) return CFI_ERR_NULL;
+    const DevLayer& d = layer->d;
+    const int64_t vs = layer->dtype == CFI_BF16 ? 2 : 4;
+    info->in_features = d.in, info->out_features = d.out, info->n_active = d.n_active, info->k = d.k;
+    info->dtype = layer->dtype, info->act = d.act;
+    info->k_padded = d.kp;
+    info->batch_slab_columns = d.cs;
+    info->batch_row_stride = d.stride_b;
+    info->reserved = 0;
+    info->weight_bytes_splitk = (int64_t)d.n_active * d.kp * (vs + 4);
+    info->weight_bytes_batch = (int64_t)d.n_active * d.stride_b * 8;
+    info->device_bytes = layer->device_bytes;
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_device_status(const cfi_layer_t* layer, cfi_stream_t stream, int32_t* flag) {
+    if (!layer || !flag) return CFI_ERR_NULL;
+    DeviceGuard g(layer->device);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CFI_ERR_CUDA;
+    if (cudaMemcpy(flag, layer->d.status, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return CFI_ERR_CUDA;
+    return *flag ? CFI_ERR_DEVICE_FLAG : CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_stack_create(cfi_layer_t* const* layers, int32_t n_layers, int32_t max_batch,
+                                         cfi_stack_t** stack) {
+    if (!stack) return CFI_ERR_NULL;
+    *stack = nullptr;
+    if (!layers) return CFI_ERR_NULL;
+    if (n_layers < 1 || max_batch < 0) return CFI_ERR_SHAPE;
+    for (int i = 0; i < n_layers; ++i) {
+        if (!layers[i]) return CFI_ERR_NULL;
+        if (layers[i]->dtype != layers[0]->dtype || layers[i]->device != layers[0]->device) return CFI_ERR_DTYPE;
+        if (i && layers[i]->d.in != layers[i - 1]->d.out) return CFI_ERR_SHAPE;
+    }
+    cfi_stack* s = new (std::nothrow) cfi_stack();
+    if (!s) return CFI_ERR_ALLOC;
+    s->layers.assign(layers, layers + n_layers);
+    s->max_batch = max_batch;
+    s->dtype = layers[0]->dtype;
+    int widest = 0;
+    for (int i = 0; i + 1 < n_layers; ++i) widest = std::max(widest, layers[i]->d.out);
+    const size_t es = s->dtype == CFI_BF16 ? 2 : 4;
+    const size_t bytes = std::max<size_t>((size_t)max_batch * widest * es, 16);
+    DeviceGuard g(layers[0]->device);
+    for (int i = 0; i < 2; ++i)
+        if (cudaMalloc(&s->buf[i], bytes) != cudaSuccess) {
+            cudaGetLastError();
+            cfi_stack_destroy(s);
+            return CFI_ERR_ALLOC;
+        }
+    *stack = s;
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_stack_forward(const cfi_stack_t* stack, const void* x, void* y, int32_t batch,
+                                          cfi_stream_t stream) {
+    if (!stack) return CFI_ERR_NULL;
+    if (batch < 0) return CFI_ERR_SHAPE;
+    if (batch > stack->max_batch) return CFI_ERR_BUFFER_TOO_SMALL;
+    const void* cur = x;
+    const int n = (int)stack->layers.size();
+    for (int i = 0; i < n; ++i) {
+        void* dst = i + 1 == n ? y : stack->buf[i & 1];
+        if (cfi_status_t e = cfi_forward(stack->layers[i], cur, dst, batch, stream)) return e;
+        cur = dst;
+    }
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_stack_destroy(cfi_stack_t* stack) {
+    if (!stack) return CFI_OK;
+    for (int i = 0; i < 2; ++i)
+        if (stack->buf[i]) cudaFree(stack->buf[i]);
+    delete stack;
+    return CFI_OK;
+}
