@@ -1,0 +1,241 @@
+"""ctypes binding of the C-ABI library declared in include/cfi.h.
+
+Same names as the C entry points; this module only marshals arguments (numpy
+arrays for host data, torch tensors or raw integer addresses for device data)
+and turns a non-zero status into CfiError.  Every step of the forward runs in
+the library's CUDA kernels; there is no Python or CPU implementation behind
+these calls, and loading fails loudly if the shared library cannot be built or
+found.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+ACT_NONE, ACT_GELU = 0, 1
+VARIANT_AUTO, VARIANT_SIMPLE, VARIANT_SPLITK, VARIANT_BATCH = 0, 1, 2, 3
+_DTYPES = {"f32": F32, "fp32": F32, "float32": F32, "bf16": BF16, "bfloat16": BF16, F32: F32, BF16: BF16}
+_ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE, ACT_GELU: ACT_GELU}
+_VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, 0: 0, 1: 1, 2: 2, 3: 3}
+
+EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
+           "cfi_layer_info", "cfi_choose_variant", "cfi_device_status", "cfi_destroy",
+           "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy")
+
+
+class CfiError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {_lib.cfi_status_string(status).decode()}")
+
+
+class LayerInfo(ctypes.Structure):
+    _fields_ = [("in_features", ctypes.c_int32), ("out_features", ctypes.c_int32), ("n_active", ctypes.c_int32),
+                ("k", ctypes.c_int32), ("dtype", ctypes.c_int32), ("act", ctypes.c_int32),
+                ("k_padded", ctypes.c_int32), ("batch_slab_columns", ctypes.c_int32),
+                ("batch_row_stride", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("weight_bytes_splitk", ctypes.c_int64), ("weight_bytes_batch", ctypes.c_int64),
+                ("device_bytes", ctypes.c_int64)]
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path) or os.environ.get("CFI_REBUILD"):
+        path = _build.build()
+    lib = ctypes.CDLL(path)
+    vp, ci = ctypes.c_void_p, ctypes.c_int32
+    f32p, i32p, u8p = ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_uint8)
+    lib.cfi_status_string.restype = ctypes.c_char_p
+    lib.cfi_status_string.argtypes = [ctypes.c_int]
+    lib.cfi_pack.argtypes = [f32p, u8p, ci, ci, i32p, i32p, f32p, i32p, i32p]
+    lib.cfi_create.argtypes = [f32p, i32p, i32p, f32p, ci, ci, ci, ci, ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
+    lib.cfi_forward.argtypes = [vp, vp, vp, ci, vp]
+    lib.cfi_forward_variant.argtypes = [vp, vp, vp, ci, vp, ctypes.c_int]
+    lib.cfi_forward_host.argtypes = [vp, vp, vp, ci, vp]
+    lib.cfi_layer_info.argtypes = [vp, ctypes.POINTER(LayerInfo)]
+    lib.cfi_choose_variant.argtypes = [vp, ci, i32p]
+    lib.cfi_device_status.argtypes = [vp, vp, i32p]
+    lib.cfi_destroy.argtypes = [vp]
+    lib.cfi_stack_create.argtypes = [ctypes.POINTER(vp), ci, ci, ctypes.POINTER(vp)]
+    lib.cfi_stack_forward.argtypes = [vp, vp, vp, ci, vp]
+    lib.cfi_stack_destroy.argtypes = [vp]
+    for name in EXPORTS:
+        if name != "cfi_status_string":
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise CfiError(status, where)
+
+
+def _hp(a: Optional[np.ndarray], ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def _dev_ptr(t) -> int:
+    """Address of a device buffer: a torch CUDA tensor (contiguous) or an int."""
+    if isinstance(t, int):
+        return t
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def cfi_status_string(status: int) -> str:
+    return _lib.cfi_status_string(int(status)).decode()
+
+
+def cfi_pack(w_dense: np.ndarray, mask: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Dense masked weight -> (values [n_act,k] f32, indices [n_act,k] i32, active_rows [n_act] i32)."""
+    w = np.ascontiguousarray(w_dense, dtype=np.float32)
+    if w.ndim != 2:
+        raise ValueError("w_dense must be 2-D")
+    m = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    if m is not None and m.shape != w.shape:
+        raise ValueError("mask shape differs from w_dense")
+    out_f, in_f = w.shape
+    k, na = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_lib.cfi_pack(_hp(w, ctypes.c_float), _hp(m, ctypes.c_uint8), out_f, in_f, ctypes.byref(k),
+                         ctypes.byref(na), None, None, None), "cfi_pack")
+    values = np.empty((na.value, k.value), dtype=np.float32)
+    indices = np.empty((na.value, k.value), dtype=np.int32)
+    rows = np.empty((na.value,), dtype=np.int32)
+    _check(_lib.cfi_pack(_hp(w, ctypes.c_float), _hp(m, ctypes.c_uint8), out_f, in_f, ctypes.byref(k),
+                         ctypes.byref(na), _hp(values, ctypes.c_float), _hp(indices, ctypes.c_int32),
+                         _hp(rows, ctypes.c_int32)), "cfi_pack")
+    return values, indices, rows
+
+
+class Layer:
+    """Owner of one cfi_layer_t handle."""
+
+    def __init__(self, handle: int, in_features: int, out_features: int, dtype: int):
+        self.handle, self.in_features, self.out_features, self.dtype = handle, in_features, out_features, dtype
+
+    def close(self) -> None:
+        if self.handle:
+            _lib.cfi_destroy(self.handle)
+            self.handle = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def cfi_create(values, indices, active_rows, bias, in_features: int, out_features: int, dtype="f32",
+               act="none") -> Layer:
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    ix = np.ascontiguousarray(indices, dtype=np.int32)
+    ar = np.ascontiguousarray(active_rows, dtype=np.int32)
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    if v.shape != ix.shape or (v.ndim != 2 and v.size) or ar.ndim != 1:
+        raise ValueError("values/indices must be [n_active, k] and active_rows [n_active]")
+    n_active = ar.shape[0]
+    k = v.shape[1] if v.ndim == 2 else 0
+    if v.ndim == 2 and v.shape[0] != n_active:
+        raise ValueError("values has a different number of rows than active_rows")
+    if b is not None and b.shape != (out_features,):
+        raise ValueError("bias must be [out_features]")
+    h = ctypes.c_void_p()
+    _check(_lib.cfi_create(_hp(v, ctypes.c_float), _hp(ix, ctypes.c_int32), _hp(ar, ctypes.c_int32),
+                           _hp(b, ctypes.c_float), n_active, k, in_features, out_features, _DTYPES[dtype],
+                           _ACTS[act], ctypes.byref(h)), "cfi_create")
+    return Layer(h.value, in_features, out_features, _DTYPES[dtype])
+
+
+def cfi_forward(layer: Layer, x, y, batch: int, stream=None) -> None:
+    _check(_lib.cfi_forward(layer.handle, _dev_ptr(x), _dev_ptr(y), batch, _stream_handle(stream)), "cfi_forward")
+
+
+def cfi_forward_variant(layer: Layer, x, y, batch: int, stream=None, variant="auto") -> None:
+    _check(_lib.cfi_forward_variant(layer.handle, _dev_ptr(x), _dev_ptr(y), batch, _stream_handle(stream),
+                                    _VARIANTS[variant]), "cfi_forward_variant")
+
+
+def cfi_forward_host(layer: Layer, x_host, y_host, batch: int, stream=None) -> None:
+    """x_host / y_host: CPU torch tensors (pinned for asynchronous copies) or numpy arrays."""
+    xp = x_host.data_ptr() if hasattr(x_host, "data_ptr") else x_host.ctypes.data
+    yp = y_host.data_ptr() if hasattr(y_host, "data_ptr") else y_host.ctypes.data
+    _check(_lib.cfi_forward_host(layer.handle, xp, yp, batch, _stream_handle(stream)), "cfi_forward_host")
+
+
+def cfi_layer_info(layer: Layer) -> LayerInfo:
+    info = LayerInfo()
+    _check(_lib.cfi_layer_info(layer.handle, ctypes.byref(info)), "cfi_layer_info")
+    return info
+
+
+def cfi_choose_variant(layer: Layer, batch: int) -> int:
+    v = ctypes.c_int32(0)
+    _check(_lib.cfi_choose_variant(layer.handle, batch, ctypes.byref(v)), "cfi_choose_variant")
+    return v.value
+
+
+def cfi_device_status(layer: Layer, stream=None) -> int:
+    flag = ctypes.c_int32(0)
+    st = _lib.cfi_device_status(layer.handle, _stream_handle(stream), ctypes.byref(flag))
+    if st not in (0, 9):
+        raise CfiError(st, "cfi_device_status")
+    return flag.value
+
+
+def cfi_destroy(layer: Layer) -> None:
+    layer.close()
+
+
+class Stack:
+    def __init__(self, handle: int, layers: Sequence[Layer], max_batch: int):
+        self.handle, self.layers, self.max_batch = handle, list(layers), max_batch
+
+    def close(self) -> None:
+        if self.handle:
+            _lib.cfi_stack_destroy(self.handle)
+            self.handle = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def cfi_stack_create(layers: Sequence[Layer], max_batch: int) -> Stack:
+    arr = (ctypes.c_void_p * len(layers))(*[l.handle for l in layers])
+    h = ctypes.c_void_p()
+    _check(_lib.cfi_stack_create(arr, len(layers), max_batch, ctypes.byref(h)), "cfi_stack_create")
+    return Stack(h.value, layers, max_batch)
+
+
+def cfi_stack_forward(stack: Stack, x, y, batch: int, stream=None) -> None:
+    _check(_lib.cfi_stack_forward(stack.handle, _dev_ptr(x), _dev_ptr(y), batch, _stream_handle(stream)),
+           "cfi_stack_forward")
+
+
+def cfi_stack_destroy(stack: Stack) -> None:
+    stack.close()

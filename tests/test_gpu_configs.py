@@ -1,0 +1,46 @@
+"""The named workloads (ViT-B/16 MLP layer shapes, 80-99 % sparsity, batch 1-256) at full size, in the
+launch configuration the benchmark times (variant auto), against the oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2305_02299_b200 import inputs
+from parity import TOL, check_layer, device_layer, oracle_layer, run_device, scaled_error
+
+pytestmark = pytest.mark.gpu
+W = inputs.workloads()
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3_b1", "c3_b64", "c3_b256"])
+def test_vit_layer_configs(name):
+    w = W[name]
+    errs = check_layer(w.layer(), w.x(), "f32", variants=("auto", "splitk" if w.batch <= 64 else "batch"))
+    assert max(errs.values()) <= 1e-5
+
+
+@pytest.mark.parametrize("sp", [80, 90, 95, 99])
+def test_sparsity_sweep_4096(sp):
+    w = W[f"c4_s{sp}_b1"]
+    L = w.layer()
+    dl = device_layer(L)
+    packed = oracle.pack(L.w_dense, L.mask)
+    for B in (1, 16, 256):
+        x = w.x(batch=B)
+        y_ref, S = oracle_layer(L, x, packed=packed)
+        assert scaled_error(run_device(dl, x, "f32", "auto"), y_ref, S) <= 1e-5
+    dl.close()
+
+
+def test_vit_mlp_block_bf16_slice():
+    """One block of the bf16 MLP stack on a 788-row slice of its 50,432-row batch (per-layer, oracle inputs)."""
+    s = inputs.StackWorkload(blocks=1)
+    Ls, specs = s.layers(seed=0), s.layer_specs()
+    x = s.x(seed=0, batch=788)
+    cur = oracle.round_bf16(x)
+    for L, sp in zip(Ls, specs):
+        y_ref, S = oracle_layer(L, cur, "bf16", sp[4])
+        dl = device_layer(L, "bf16", sp[4])
+        y = run_device(dl, cur, "bf16")
+        assert scaled_error(y, y_ref, S) <= TOL["bf16"]
+        dl.close()
+        cur = oracle.round_bf16(y_ref.astype(np.float32))

@@ -1,0 +1,198 @@
+"""Parity of the CUDA forward (through the C-ABI) with the CPU oracle, element by element.
+
+Tolerance: max |y - y_oracle| / S <= 1e-5 (fp32) or 2e-2 (bf16 storage, fp32 accumulate), where
+S = |bias| + sum_j |w x| is the scale of the sum (a plain ratio to |y| is unbounded when terms cancel).
+Integer-valued cases must agree bit for bit whatever the summation order.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2305_02299_b200 import inputs
+from parity import TOL, check_layer, device_layer, oracle_layer, run_device, scaled_error, to_device, torch_dtype
+
+pytestmark = pytest.mark.gpu
+ALL = ("simple", "splitk", "batch", "auto")
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 5, 31, 32, 33, 77])
+@pytest.mark.parametrize("B", [1, 2, 3, 17])
+def test_fan_in_grid_fp32(k, B):
+    L = inputs.make_layer(101, 67, k, n_ablated=5, seed=k)
+    check_layer(L, inputs.make_x(B, 101, seed=B), "f32", variants=ALL)
+
+
+@pytest.mark.parametrize("B", [1, 2, 3, 8, 9, 17, 64, 65, 255, 256, 257])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_batch_grid(B, dtype):
+    L = inputs.make_layer(768, 200, 77, n_ablated=13, seed=2)
+    check_layer(L, inputs.make_x(B, 768, seed=B), dtype, variants=ALL)
+
+
+@pytest.mark.parametrize("in_f,out_f,k", [(1, 1, 1), (5, 3, 5), (9, 130, 4), (1000, 7, 307), (4096, 33, 819),
+                                          (2050, 300, 41), (333, 1025, 100)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_odd_shapes(in_f, out_f, k, dtype):
+    L = inputs.make_layer(in_f, out_f, k, n_ablated=out_f // 7, seed=in_f)
+    for B in (1, 5, 70):
+        check_layer(L, inputs.make_x(B, in_f, seed=3), dtype, variants=ALL)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("act", ["none", "gelu"])
+def test_gelu_and_ablated_rows(dtype, act):
+    import torch
+    L = inputs.make_layer(256, 96, 20, n_ablated=30, seed=4)
+    x = inputs.make_x(33, 256, seed=4)
+    y_ref, S = oracle_layer(L, x, dtype, act)
+    dl = device_layer(L, dtype, act)
+    for v in ALL:
+        y = run_device(dl, x, dtype, v)
+        assert scaled_error(y, y_ref, S) <= TOL[dtype]
+        # Ablated rows carry act(bias) only, identical for every batch row and rounded once to the storage type.
+        expect = torch.tensor(y_ref[0, L.ablated]).to(torch_dtype(dtype)).to(torch.float64).numpy()
+        got = y[:, L.ablated]
+        if act == "none":
+            assert np.array_equal(got, np.tile(expect, (33, 1)))
+        else:
+            assert np.all(got == got[0:1]) and np.allclose(got[0], expect, rtol=2 ** -7 if dtype == "bf16" else 1e-6, atol=1e-7)
+    dl.close()
+
+
+def test_all_rows_ablated_and_no_bias():
+    from paper_2305_02299_b200 import binding as cfi
+    dl = cfi.cfi_create(np.zeros((0, 0), np.float32), np.zeros((0, 0), np.int32), np.zeros((0,), np.int32),
+                        np.arange(6, dtype=np.float32), 10, 6)
+    for v in ALL:
+        y = run_device(dl, inputs.make_x(4, 10), "f32", v)
+        assert np.array_equal(y, np.tile(np.arange(6.0), (4, 1)))
+    dl.close()
+    L = inputs.make_layer(40, 12, 6, n_ablated=2, seed=1)
+    vv, ix, rows = cfi.cfi_pack(L.w_dense, L.mask)
+    dl = cfi.cfi_create(vv, ix, rows, None, 40, 12)          # Algorithm 1 as printed: no bias
+    x = inputs.make_x(3, 40, seed=1)
+    y_ref, S = oracle.forward(vv, ix, rows, None, 40, 12, x, want_scale=True)
+    for v in ALL:
+        y = run_device(dl, x, "f32", v)
+        assert np.all(y[:, L.ablated] == 0.0)
+        assert np.max(np.abs(y - y_ref)) <= 1e-5 * max(1.0, S.max())
+    dl.close()
+
+
+def test_batch_zero_launches_nothing():
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    L = inputs.make_layer(16, 8, 2, seed=0)
+    dl = device_layer(L)
+    y = torch.full((8,), 7.0, device="cuda")
+    cfi.cfi_forward(dl, torch.zeros(16, device="cuda"), y, 0)
+    torch.cuda.synchronize()
+    assert torch.all(y == 7.0)
+    assert cfi.cfi_device_status(dl) == 0
+    dl.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B", [1, 6, 40, 130])
+def test_exact_integer_arithmetic_is_bit_exact(dtype, B):
+    """Small-integer weights and inputs: every partial sum is exact in fp32 (and every output fits bf16
+    exactly), so any summation order and tiling must give the oracle's numbers bit for bit."""
+    L = inputs.make_layer(512, 150, 24, n_ablated=11, seed=7, integer_valued=True)
+    x = inputs.make_x(B, 512, seed=7, integer_valued=True, density=0.15 if dtype == "bf16" else 1.0)
+    y_ref, _ = oracle_layer(L, x, dtype)
+    if dtype == "bf16":
+        assert np.max(np.abs(y_ref)) <= 256          # integers up to 2^8 are exact in bf16
+    dl = device_layer(L, dtype)
+    for v in ALL:
+        assert np.array_equal(run_device(dl, x, dtype, v), y_ref), v
+    dl.close()
+
+
+def test_unsorted_and_duplicate_indices():
+    from paper_2305_02299_b200 import binding as cfi
+    rng = np.random.default_rng(0)
+    vals = rng.standard_normal((20, 9)).astype(np.float32)
+    idx = rng.integers(0, 30, size=(20, 9)).astype(np.int32)      # unsorted, with repeats
+    rows = rng.permutation(25)[:20].astype(np.int32)              # unsorted rows
+    bias = rng.standard_normal(25).astype(np.float32)
+    dl = cfi.cfi_create(vals, idx, rows, bias, 30, 25)
+    for B in (1, 4, 70):
+        x = inputs.make_x(B, 30, seed=B)
+        y_ref, S = oracle.forward(vals, idx, rows, bias, 30, 25, x, want_scale=True)
+        for v in ALL:
+            assert scaled_error(run_device(dl, x, "f32", v), y_ref, S) <= 1e-5
+    dl.close()
+
+
+def test_inf_in_unused_column_does_not_leak():
+    """A column no row reads may hold inf/NaN: padding entries must not touch real data."""
+    L = inputs.make_layer(64, 10, 3, seed=3)          # 30 of 64 columns used at most
+    unused = np.nonzero(L.mask.sum(axis=0) == 0)[0]
+    assert unused.size > 0
+    x = inputs.make_x(20, 64, seed=3)
+    x[:, unused] = np.inf
+    x[:, 0] = np.inf if 0 in unused else x[:, 0]
+    y_ref, S = oracle_layer(L, x)
+    dl = device_layer(L)
+    for v in ALL:
+        y = run_device(dl, x, "f32", v)
+        assert np.all(np.isfinite(y)) and scaled_error(y, y_ref, S) <= 1e-5
+    dl.close()
+
+
+def test_forward_host_matches_device_call():
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    L = inputs.make_layer(768, 300, 77, n_ablated=20, seed=6)
+    dl = device_layer(L)
+    for B in (3, 64, 10):                               # grows, then reuses the staging buffers
+        x = inputs.make_x(B, 768, seed=B)
+        xh = torch.from_numpy(x).pin_memory()
+        yh = torch.empty((B, 300), dtype=torch.float32).pin_memory()
+        cfi.cfi_forward_host(dl, xh, yh, B)
+        assert np.array_equal(yh.numpy().astype(np.float64), run_device(dl, x, "f32", "auto"))
+    dl.close()
+
+
+def test_misaligned_pointer_is_rejected():
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    dl = device_layer(inputs.make_layer(16, 8, 2, seed=0))
+    buf = torch.zeros(64, device="cuda")
+    with pytest.raises(cfi.CfiError) as e:
+        cfi.cfi_forward(dl, buf[1:17], buf[32:40], 1)
+    assert e.value.status == 10
+    dl.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_stack_matches_chained_oracle(dtype):
+    """MLP-shaped chain: per-layer comparison with oracle-supplied inputs, then the library's own chain."""
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    s = inputs.StackWorkload(blocks=2, d_model=96, d_hidden=384, k_up=10, k_down=38, batch=70)
+    Ls = s.layers(seed=1)
+    specs = s.layer_specs()
+    packed = [oracle.pack(L.w_dense, L.mask) for L in Ls]
+    o_layers = [(p[0], p[1], p[2], L.bias, sp[0], sp[1], sp[4]) for p, L, sp in zip(packed, Ls, specs)]
+    x = s.x(seed=1)
+    outs, exact, scales = oracle.stack_forward(o_layers, x, dtype=dtype)
+    dls = [device_layer(L, dtype, sp[4]) for L, sp in zip(Ls, specs)]
+    cur = oracle.round_bf16(x) if dtype == "bf16" else x
+    for i, dl in enumerate(dls):                        # teacher-forced: layer i gets the oracle's input
+        y = run_device(dl, cur, dtype)
+        assert scaled_error(y, exact[i], scales[i]) <= TOL[dtype], i
+        cur = outs[i].astype(np.float32)
+    st = cfi.cfi_stack_create(dls, 70)
+    y_d = torch.empty((70, 96), device="cuda", dtype=torch_dtype(dtype))
+    cfi.cfi_stack_forward(st, to_device(x, dtype), y_d, 70)
+    torch.cuda.synchronize()
+    y = y_d.to(torch.float64).cpu().numpy()
+    rel = np.linalg.norm(y - outs[-1]) / np.linalg.norm(outs[-1])
+    assert rel <= (1e-5 if dtype == "f32" else 3e-2), rel
+    with pytest.raises(cfi.CfiError) as e:
+        cfi.cfi_stack_forward(st, to_device(x, dtype), y_d, 71)
+    assert e.value.status == 5
+    st.close()
+    for dl in dls:
+        dl.close()
