@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the condensed constant-fan-in linear forward.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one cfi_forward over one batch of the headline workload: the 768 -> 3072, k = 77 (90 % sparse)
+fp32 layer at batch 256.  Prints ONE JSON line: effective GFLOP/s (2 * B * n_active * k / t), ms per step,
+the roofline object for the forward kernel, an end-to-end number with host buffers, the CPU oracle timed
+on this host as a reported baseline, and the batch-1 (online inference) numbers next to it.
+
+Timing: steps run as replays of a CUDA graph that holds the launches back to back, between CUDA events on
+the launching stream; consecutive steps use different replicas of the layer and of x / y whose total size
+exceeds twice the L2, so every step streams its operands from HBM.  With N > 1 (torchrun) every rank runs
+the same workload on its own GPU and its own batches (no exchange step exists in this path), the time is
+the maximum over ranks and the value the sum of all ranks' work.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2305_02299_b200 import inputs  # noqa: E402
+
+METRIC = "cfi_forward effective GFLOP/s (2*B*n_active*k/t), 768->3072 k=77 fp32, batch 256"
+FMA_LANES_PER_SM = 128      # fp32 FMA lanes per SM
+L2_BYTES_FALLBACK = 126 * 1024 * 1024
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def algorithmic_bytes(w: inputs.Workload, n_active: int, elem: int = 4) -> int:
+    """values + int32 indices once, x once, y once, bias and the active-row list."""
+    return n_active * w.k * (elem + 4) + w.batch * w.in_features * elem + w.batch * w.out_features * elem \
+        + w.out_features * 4 + n_active * 4
+
+
+def algorithmic_flops(w: inputs.Workload, n_active: int) -> int:
+    return 2 * w.batch * n_active * w.k
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while a region runs."""
+    _REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.max_mhz, self._stop, self._thr, self._h = None, threading.Event(), None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = int(vis.split(",")[index]) if vis and vis.split(",")[index].isdigit() else index
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+
+    def _once(self):
+        nv = self._nv
+        self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+        try:
+            mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+        except Exception:
+            mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+        for bit, name in self._REASONS.items():
+            if mask & bit:
+                self.reasons.add(name)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self._once()
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------------
+# device-side timing
+# --------------------------------------------------------------------------------------------------
+class Replicas:
+    """R independent copies of (layer, x, y) so that consecutive steps touch different memory."""
+
+    def __init__(self, w: inputs.Workload, cfi, torch, min_total_bytes: int, dtype: str = "f32", seed: int = 0,
+                 rank: int = 0, max_replicas: int = 64):
+        self.w, self.cfi, self.torch = w, cfi, torch
+        tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+        base = w.layer(seed=seed, replica=0)
+        v, ix, rows = cfi.cfi_pack(base.w_dense, base.mask)
+        self.n_active = int(rows.shape[0])
+        elem = 4 if dtype == "f32" else 2
+        self.bytes_per_step = algorithmic_bytes(w, self.n_active, elem)
+        per = self.bytes_per_step
+        self.R = int(max(2, min(max_replicas, -(-min_total_bytes // per))))
+        self.layers, self.x, self.y = [], [], []
+        rng = np.random.default_rng(1234 + rank)
+        for r in range(self.R):
+            # Same structure statistics, different numbers: permute rows of the base layer's condensed arrays
+            # (cheap) instead of drawing a fresh dense matrix per replica.
+            p = rng.permutation(self.n_active)
+            self.layers.append(cfi.cfi_create(v[p], ix[p], rows, base.bias, w.in_features, w.out_features,
+                                              dtype=dtype, act=w.act))
+            xr = w.x(seed=seed, replica=r + 100 * rank)
+            self.x.append(torch.from_numpy(xr).to("cuda", tdt).contiguous())
+            self.y.append(torch.empty((w.batch, w.out_features), device="cuda", dtype=tdt))
+        self.total_bytes = self.R * per
+
+    def step(self, i: int, variant: str = "auto"):
+        r = i % self.R
+        self.cfi.cfi_forward_variant(self.layers[r], self.x[r], self.y[r], self.w.batch, variant=variant)
+
+    def close(self):
+        for l in self.layers:
+            l.close()
+
+
+def time_steps(rep: Replicas, torch, steps: int, warmup: int, variant: str = "auto", graph_len: int = 1000,
+               barrier=None, sampler=None):
+    """Returns (seconds for exactly `steps` steps, launches).  Warm-up covers every replica at least once."""
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(max(warmup, 3)):
+            rep.step(i, variant)
+        for i in range(rep.R):
+            rep.step(i, variant)
+        stream.synchronize()
+        g_len = max(1, min(graph_len, steps))
+        n_replay, rem = divmod(steps, g_len)
+        graphs = []
+        for length in ([g_len] if n_replay else []) + ([rem] if rem else []):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(length):
+                    rep.step(i, variant)
+            graphs.append(g)
+        main = graphs[0] if n_replay else None
+        tail = graphs[-1] if rem else None
+        for g in graphs:            # one untimed replay each (graph upload)
+            g.replay()
+        stream.synchronize()
+        if barrier:
+            barrier()
+        torch.cuda.synchronize()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ctx = sampler if sampler is not None else _Null()
+        with ctx:
+            start.record(stream)
+            for _ in range(n_replay):
+                main.replay()
+            if tail is not None:
+                tail.replay()
+            end.record(stream)
+            end.synchronize()
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+    return start.elapsed_time(end) * 1e-3, steps
+
+
+class _Null:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        return False
+
+
+def time_e2e(rep: Replicas, torch, steps: int, warmup: int):
+    """Through cfi_forward_host: pinned host x -> device, forward, y -> pinned host, every step."""
+    w = rep.w
+    tdt = rep.x[0].dtype
+    xh = [rep.x[r].cpu().pin_memory() for r in range(min(rep.R, 8))]
+    yh = torch.empty((w.batch, w.out_features), dtype=tdt).pin_memory()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(max(3, warmup)):
+            rep.cfi.cfi_forward_host(rep.layers[i % rep.R], xh[i % len(xh)], yh, w.batch)
+        torch.cuda.synchronize()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(stream)
+        for i in range(steps):
+            rep.cfi.cfi_forward_host(rep.layers[i % rep.R], xh[i % len(xh)], yh, w.batch)
+        end.record(stream)
+        end.synchronize()
+    sec = start.elapsed_time(end) * 1e-3
+    return sec, xh[0].numel() * xh[0].element_size(), yh.numel() * yh.element_size()
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU oracle timing (reported baseline, and the --impl reference arm)
+# --------------------------------------------------------------------------------------------------
+def time_oracle(w: inputs.Workload, budget_s: float, sample_rows=None, repeats=None):
+    import oracle
+    L = w.layer(seed=0)
+    v, ix, rows = oracle.pack(L.w_dense, L.mask)
+    x = w.x(seed=0)
+    if sample_rows is None:
+        sample_rows = w.batch
+    xs = np.ascontiguousarray(x[:sample_rows])
+    call = lambda: oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, xs, act=w.act)
+    call()
+    t0 = time.perf_counter()
+    call()
+    one = time.perf_counter() - t0
+    if repeats is None:
+        repeats = int(max(5, min(2000, budget_s / max(one, 1e-6))))
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        call()
+        times.append(time.perf_counter() - t0)
+    flops = 2 * sample_rows * rows.shape[0] * w.k
+    return {"median_s": statistics.median(times), "flops": flops, "calls": repeats, "rows": sample_rows,
+            "cores": oracle.max_threads()}
+
+
+def run_reference(args, w):
+    """The oracle as it stands on the host cores; each step is one forward over a bounded sample of the batch."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    total = args.steps + args.warmup
+    L = w.layer(seed=0)
+    v, ix, rows = oracle.pack(L.w_dense, L.mask)
+    x = w.x(seed=0)
+    t0 = time.perf_counter()
+    oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, x[:8])
+    per_row = max((time.perf_counter() - t0) / 8, 1e-7)
+    sample = int(max(1, min(w.batch, (120.0 / max(total, 1)) / per_row)))
+    xs = np.ascontiguousarray(x[:sample])
+    for _ in range(args.warmup):
+        oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, xs)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, xs)
+    sec = time.perf_counter() - t0
+    gflops = 2 * sample * rows.shape[0] * w.k * args.steps / sec / 1e9
+    cores = oracle.max_threads()
+    desc = f"{sample} of {w.batch} batch rows per step, all {w.out_features} output rows"
+    line = {"impl": "reference", "metric": METRIC, "value": gflops, "unit": "GFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "in": w.in_features, "out": w.out_features, "k": w.k, "batch": w.batch,
+                       "sample": desc},
+            "cpu_baseline": {"value": gflops, "unit": "GFLOP/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": gflops, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--variant", default="auto")
+    ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
+    args = ap.parse_args()
+    W = inputs.workloads()
+    w = W[args.workload]
+
+    if args.impl == "reference":
+        args.steps = 20 if args.steps is None else args.steps
+        args.warmup = 3 if args.warmup is None else args.warmup
+        run_reference(args, w)
+        return
+    args.steps = 200000 if args.steps is None else args.steps
+    args.warmup = 20 if args.warmup is None else args.warmup
+
+    import torch
+    from paper_2305_02299_b200 import binding as cfi   # raises if the CUDA library is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    barrier = (lambda: dist.barrier()) if dist else None
+
+    peaks, peak_kind = measured_peaks()
+    props = torch.cuda.get_device_properties(local)
+    l2 = getattr(props, "L2_cache_size", None) or L2_BYTES_FALLBACK
+    sm_count = props.multi_processor_count
+
+    rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), rank=rank)
+    sampler = ClockSampler(local)
+    sec, launches = time_steps(rep, torch, args.steps, args.warmup, args.variant, barrier=barrier, sampler=sampler)
+    if dist:
+        t = torch.tensor([sec], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+    flops = algorithmic_flops(w, rep.n_active)
+    per_call = sec / args.steps
+    value = flops * world / per_call / 1e9
+
+    # End to end through the host-buffer entry point (each rank on its own GPU).
+    e2e_steps = int(min(args.steps, 2000))
+    e2e_sec, h2d, d2h = time_e2e(rep, torch, e2e_steps, 5)
+    if dist:
+        t = torch.tensor([e2e_sec], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_sec = float(t.item())
+    e2e_value = flops * world / (e2e_sec / e2e_steps) / 1e9
+
+    line = None
+    if rank == 0:
+        sm_max_mhz = float(peaks.get("sm_max_mhz", 1965.0))
+        fma_peak_tflops = sm_count * FMA_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
+        achieved_tflops = flops / per_call / 1e12
+        hbm_gbs = rep.bytes_per_step / per_call / 1e9
+        info = cfi.cfi_layer_info(rep.layers[0])
+        chosen = {1: "simple", 2: "splitk", 3: "batch"}[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
+        line = {
+            "metric": METRIC, "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": per_call * 1e3, "us_per_call": per_call * 1e6,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "in": w.in_features, "out": w.out_features, "k": w.k,
+                       "n_active": rep.n_active, "batch": w.batch, "variant": chosen if args.variant == "auto" else args.variant,
+                       "l2": f"inputs larger than L2: {rep.R} rotating replicas of layer+x+y, "
+                             f"{rep.total_bytes / 1e6:.0f} MB vs L2 {l2 / 1e6:.0f} MB",
+                       "timing": "CUDA-graph replays between CUDA events on the launching stream"},
+            "roofline": {"bound": "alu", "achieved": achieved_tflops, "peak": fma_peak_tflops, "unit": "TFLOP/s",
+                         "frac": achieved_tflops / fma_peak_tflops, "traffic": None,
+                         "peak_source": f"{sm_count} SMs x {FMA_LANES_PER_SM} fp32 FMA lanes x 2 x {sm_max_mhz:.0f} MHz",
+                         "kernel": "cfi_batch_kernel<float>" if chosen == "batch" else f"cfi_{chosen}_kernel",
+                         "hbm_achieved_gbs": hbm_gbs, "hbm_peak_gbs": peaks["hbm_gbs"],
+                         "hbm_frac": hbm_gbs / peaks["hbm_gbs"], "hbm_peak_source": f"{peak_kind} copy bandwidth",
+                         "algorithmic_bytes": rep.bytes_per_step, "algorithmic_flops": flops,
+                         "weight_bytes_streamed_per_batch_tile": int(info.weight_bytes_batch)},
+            "e2e": {"value": e2e_value, "unit": "GFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "us_per_call": e2e_sec / e2e_steps * 1e6, "steps": e2e_steps, "api": "cfi_forward_host"},
+            "gpu_launches": launches,
+            "clocks": sampler.summary(),
+        }
+    rep.close()
+
+    if rank == 0 and world == 1 and not args.no_extras:
+        line["batch1"] = batch1_leg(W, cfi, torch, l2, peaks, peak_kind)
+        cb = time_oracle(w, budget_s=15.0)
+        line["cpu_baseline"] = {"value": cb["flops"] / cb["median_s"] / 1e9, "unit": "GFLOP/s", "cores": cb["cores"],
+                                "kind": "oracle", "us_per_call": cb["median_s"] * 1e6,
+                                "sample": f"whole workload ({cb['rows']} batch rows), median of {cb['calls']} calls"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def batch1_leg(W, cfi, torch, l2, peaks, peak_kind):
+    """Online inference (batch 1): us per call and achieved fraction of the HBM roofline, cold (rotating
+    replicas larger than L2) and warm (one layer, L2-resident)."""
+    out = {}
+    for name in ("c1", "c3_b1", "c4_s80_b1", "c4_s90_b1"):
+        w = W[name]
+        rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), max_replicas=160)
+        info = cfi.cfi_layer_info(rep.layers[0])
+        streamed = int(info.weight_bytes_splitk) + (w.in_features + 2 * w.out_features) * 4
+        steps = 20000
+        sec, _ = time_steps(rep, torch, steps, 20)
+        cold = sec / steps
+        one = Replicas(w, cfi, torch, 0, max_replicas=2)
+        one.R = 1
+        sec, _ = time_steps(one, torch, steps, 20)
+        warm = sec / steps
+        one.close()
+        out[name] = {"us_per_call_cold": cold * 1e6, "us_per_call_warm": warm * 1e6,
+                     "algorithmic_bytes": rep.bytes_per_step, "streamed_bytes": streamed,
+                     "hbm_gbs_cold": rep.bytes_per_step / cold / 1e9,
+                     "hbm_frac_cold": rep.bytes_per_step / cold / 1e9 / peaks["hbm_gbs"],
+                     "hbm_peak_source": f"{peak_kind} copy bandwidth",
+                     "gflops_cold": algorithmic_flops(w, rep.n_active) / cold / 1e9,
+                     "replicas": rep.R, "replica_bytes_total": rep.total_bytes}
+        rep.close()
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -17,6 +17,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstdlib>
@@ -408,14 +409,21 @@ BatchShape batch_shape(const cfi_layer* l, int batch) {
 // ------------------------------------------------------------------------------------------------
 // host: launches
 // ------------------------------------------------------------------------------------------------
+// Opt in to more than 48 KB of dynamic shared memory.  The attribute is per kernel and per device, so the
+// largest value set so far is remembered per (instantiation, device) and the runtime is only called to raise it.
+constexpr int kMaxDevices = 64;
+
 template <typename K>
-cfi_status_t set_smem(K kernel, size_t bytes) {
-    if (bytes > 48 * 1024) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
-            cudaGetLastError();
-            return CFI_ERR_SHAPE;
-        }
+cfi_status_t set_smem(K kernel, size_t bytes, int device) {
+    static std::atomic<int> granted[kMaxDevices];
+    if (bytes <= 48 * 1024) return CFI_OK;
+    const bool tracked = device >= 0 && device < kMaxDevices;
+    if (tracked && granted[device].load(std::memory_order_relaxed) >= (int)bytes) return CFI_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_SHAPE;
     }
+    if (tracked) granted[device].store((int)bytes, std::memory_order_relaxed);
     return CFI_OK;
 }
 
@@ -423,7 +431,7 @@ template <typename VT, int BT, int G>
 cfi_status_t launch_splitk_g(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
                              cudaStream_t st) {
     auto kern = cfi_splitk_kernel<VT, BT, G>;
-    if (cfi_status_t e = set_smem(kern, s.smem)) return e;
+    if (cfi_status_t e = set_smem(kern, s.smem, l->device)) return e;
     kern<<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, x, y, batch, s.rows_per_group);
     return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
 }
@@ -443,7 +451,7 @@ cfi_status_t launch_splitk_bt(const cfi_layer* l, const SplitkShape& s, const VT
 template <typename VT>
 cfi_status_t launch_splitk(const cfi_layer* l, const SplitkShape& s, const void* x, void* y, int batch,
                            cudaStream_t st) {
-    if (s.smem > (size_t)l->smem_optin) return CFI_ERR_SHAPE;
+    if (s.smem > (size_t)l->smem_optin || s.grid_y > 65535) return CFI_ERR_SHAPE;
     const VT* xx = static_cast<const VT*>(x);
     VT* yy = static_cast<VT*>(y);
     switch (s.bt) {
@@ -458,9 +466,9 @@ cfi_status_t launch_splitk(const cfi_layer* l, const SplitkShape& s, const void*
 template <typename VT>
 cfi_status_t launch_batch(const cfi_layer* l, const BatchShape& s, const void* x, void* y, int batch,
                           cudaStream_t st) {
-    if (s.smem > (size_t)l->smem_optin) return CFI_ERR_SHAPE;
+    if (s.smem > (size_t)l->smem_optin || s.grid_y > 65535) return CFI_ERR_SHAPE;
     auto kern = cfi_batch_kernel<VT>;
-    if (cfi_status_t e = set_smem(kern, s.smem)) return e;
+    if (cfi_status_t e = set_smem(kern, s.smem, l->device)) return e;
     kern<<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, static_cast<const VT*>(x), static_cast<VT*>(y),
                                                               batch, s.rt);
     return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
