@@ -9,8 +9,8 @@
 //
 //   large-batch layout: columns are cut into slabs that fit shared memory; each row's entries are
 //     grouped by slab (sorting a row by column makes the groups contiguous), every group is padded
-//     to a multiple of 4, and columns are stored relative to the slab start.  seg[r][s] is the
-//     first 4-entry "quad" of row r in slab s.
+//     to a multiple of 4, and columns are stored relative to the slab start.  Entries are stored as
+//     32-byte "quads" (4 weights, 4 columns); seg[r][s] is the first quad of row r in slab s.
 #include "cfi.h"
 
 #include <cuda_bf16.h>
@@ -28,20 +28,20 @@
 
 namespace {
 
-constexpr int kBatchTile = 64;  // batch columns per CTA in the large-batch kernel
-constexpr int kSlabBytesBudget = 80 * 1024;
+constexpr int kBatchTile = 64;            // batch columns per CTA in the large-batch kernel
+constexpr int kBatchSmemBudget = 216 * 1024;  // what the large-batch kernel may use of the SM's shared memory
 
 struct DevLayer {
     const void* values;      // [n_active][kp]  fp32 or bf16
     const int32_t* indices;  // [n_active][kp]
-    const float* values_b;   // [n_active][stride_b]
-    const int32_t* cols_b;   // [n_active][stride_b] slab-relative column (cs = zero row)
-    const int32_t* seg;      // [n_active][n_slabs + 1] quad offsets
+    const void* wq_b;        // [n_active][stride_q] quads: 4 fp32 weights, then 4 int32 slab-relative columns
+                             //   (a pad entry has weight 0 and column cs, the staged zero column)
+    const int32_t* seg;      // [n_active][n_slabs + 1] first quad of every slab within the row
     const float* bias;       // [out]
     const int32_t* slot;     // [out] -> row of the condensed arrays, or -1 if ablated
     int32_t* status;
     int in, out, n_active, k, kp, act;
-    int cs, n_slabs, stride_b;
+    int cs, n_slabs, stride_q, maxq;  // slab width, slabs, quads per row, most quads of a row in one slab
 };
 
 }  // namespace
@@ -261,32 +261,75 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
 }
 
 // ------------------------------------------------------------------------------------------------
-// CFI_VARIANT_BATCH: large batch.  A CTA owns `rt` consecutive output rows x 64 batch columns.  Per
-// column slab it stages x transposed as xs[column][64] (so one column index yields 64 contiguous
-// batch values), then every 16-lane half-warp walks one row's entries of that slab: (weight, column)
-// are the same for the 16 lanes, each lane gathers its 4 batch values with one 16-byte (fp32) or
-// 8-byte (bf16) shared-memory load and does 4 FMAs.  Partial sums sit in ys[b][row] between slabs and
-// are written out row-contiguously at the end.
+// CFI_VARIANT_BATCH: large batch.  A CTA owns a tile of `rt` consecutive output rows x BT batch columns
+// and walks the columns of x slab by slab.
 //
-// Within a staged row the sixteen 4-value units are permuted by unit ^ (column & 15).  The staging
-// warp covers 8 consecutive columns x 4 batch rows (whole 32-byte sectors of x) and its stores then
-// fall into 32 different banks; the reading half-warp still sees each quarter in distinct banks.
+//   producer warps  read x[b0.., slab] (row-major, 16 bytes per lane, whole 128-byte lines per row) and
+//                   store it transposed into one of two shared-memory buffers xs[column][BT], so that a
+//                   single column index yields BT contiguous batch values;
+//   consumer warps  are split into row groups of BT/4 lanes.  A group owns `rph` rows of the tile and
+//                   keeps their partial sums in registers across slabs.  For every (slab, row) it copies
+//                   the row's quads of that slab (4 weights + 4 slab-relative columns = 32 bytes) into a
+//                   warp-private buffer with cp.async one item ahead, then per entry gathers its 4 batch
+//                   values with one 16-byte (fp32) or 8-byte (bf16) shared-memory load and does 4 FMAs.
+//
+// Producers and consumers hand the two x buffers back and forth with named barriers (FULL / EMPTY per
+// buffer).  At the end the sums go through shared memory once more so that y[b, o] is written in runs
+// of consecutive o.
+//
+// Within a staged column the BT/4 four-value units are permuted by unit ^ ((column / 4) & (BT/4 - 1)).
+// A staging warp reads 4 batch rows x 32 consecutive columns and its transposed stores then fall into
+// 32 different banks; a reading row group still sees consecutive units in distinct banks.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ int swz(int col, int unit) { return (col * (kBatchTile / 4) + (unit ^ (col & 15))) << 2; }
+constexpr int kProducerWarps = 4;
+constexpr int kMaxRowsPerGroup = 8;
+constexpr int kStageUnroll = 8;  // 16-byte (fp32) / 8-byte (bf16) x loads in flight per producer thread
 
-template <typename XT> struct SmemRow;
-template <> struct SmemRow<float> {
+enum : int { kBarFull0 = 1, kBarFull1 = 2, kBarEmpty0 = 3, kBarEmpty1 = 4 };
+
+__device__ __forceinline__ void bar_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(int id, int count) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <int BT>
+__device__ __forceinline__ int swz(int col, int unit) {
+    return (col * (BT / 4) + (unit ^ ((col >> 2) & (BT / 4 - 1)))) << 2;
+}
+
+__device__ __forceinline__ void load4(const float* p, float (&v)[4]) {
+    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = t.x, v[1] = t.y, v[2] = t.z, v[3] = t.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, __nv_bfloat16 (&v)[4]) {
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    *reinterpret_cast<uint2*>(v) = t;
+}
+
+template <typename XT, int BT> struct SmemRow;
+template <int BT> struct SmemRow<float, BT> {
     static __device__ __forceinline__ void fma4(float (&a)[4], const float* xs, int col, int ll, float w) {
-        const float4 v = *reinterpret_cast<const float4*>(xs + swz(col, ll));
+        const float4 v = *reinterpret_cast<const float4*>(xs + swz<BT>(col, ll));
         a[0] = fmaf(w, v.x, a[0]);
         a[1] = fmaf(w, v.y, a[1]);
         a[2] = fmaf(w, v.z, a[2]);
         a[3] = fmaf(w, v.w, a[3]);
     }
 };
-template <> struct SmemRow<__nv_bfloat16> {
+template <int BT> struct SmemRow<__nv_bfloat16, BT> {
     static __device__ __forceinline__ void fma4(float (&a)[4], const __nv_bfloat16* xs, int col, int ll, float w) {
-        const uint2 v = *reinterpret_cast<const uint2*>(xs + swz(col, ll));
+        const uint2 v = *reinterpret_cast<const uint2*>(xs + swz<BT>(col, ll));
         a[0] = fmaf(w, bf16_lo(v.x), a[0]);
         a[1] = fmaf(w, bf16_hi(v.x), a[1]);
         a[2] = fmaf(w, bf16_lo(v.y), a[2]);
@@ -294,59 +337,174 @@ template <> struct SmemRow<__nv_bfloat16> {
     }
 };
 
-template <typename VT>
-__global__ void cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch, int rt) {
-    constexpr int BT = kBatchTile, LPR = BT / 4, RPW = 32 / LPR;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    VT* xs = reinterpret_cast<VT*>(smem_raw);  // [(cs + 1)][BT], units swizzled
-    const int pitch = rt | 1;                  // odd: spreads banks
-    float* ys = reinterpret_cast<float*>(smem_raw + (((size_t)(L.cs + 1) * BT * sizeof(VT) + 15) & ~(size_t)15));
+// Shared-memory carve-up, identical on host and device.
+struct BatchSmem {
+    size_t xs_bytes;    // one x buffer
+    size_t meta_off;    // slot_s[rt] then seg_s[rt][n_slabs + 1]
+    size_t wbuf_off;    // [consumer warp][2 stages][rows per warp][maxq] quads of 32 bytes
+    size_t total;
+};
+__host__ __device__ inline BatchSmem batch_smem_layout(int cs, int n_slabs, int maxq, int elem, int bt, int rt,
+                                                       int consumer_warps) {
+    BatchSmem m;
+    m.xs_bytes = (((size_t)(cs + 1) * bt * elem) + 127) & ~(size_t)127;
+    m.meta_off = 2 * m.xs_bytes;
+    const size_t meta = (((size_t)rt * (n_slabs + 2) * 4) + 31) & ~(size_t)31;
+    m.wbuf_off = m.meta_off + meta;
+    m.total = m.wbuf_off + (size_t)consumer_warps * 2 * (128 / bt) * maxq * 32;
+    return m;
+}
 
-    const int tid = threadIdx.x, nthr = blockDim.x;
+template <typename VT, int BT>
+__global__ void __launch_bounds__(512, 1)
+cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch, int rph, int ncw) {
+    constexpr int LPR = BT / 4, RPW = 32 / LPR;  // lanes per row group, row groups per warp
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31;
+    const int ngroups = ncw * RPW, rt = ngroups * rph, S = L.n_slabs;
+    const BatchSmem lay = batch_smem_layout(L.cs, S, L.maxq, (int)sizeof(VT), BT, rt, ncw);
+    VT* xs0 = reinterpret_cast<VT*>(smem_raw);
+    VT* xs1 = reinterpret_cast<VT*>(smem_raw + lay.xs_bytes);
+    int32_t* slot_s = reinterpret_cast<int32_t*>(smem_raw + lay.meta_off);
+    int32_t* seg_s = slot_s + rt;  // [rt][S + 1]
     const int b0 = blockIdx.y * BT, nb = min(BT, batch - b0);
     const int o0 = blockIdx.x * rt, nrows = min(rt, L.out - o0);
-    const int lane = tid & 31, sub = lane / LPR, ll = lane % LPR;
-    const int row_step = (nthr >> 5) * RPW;
 
-    if (tid < BT) xs[(size_t)L.cs * BT + tid] = VT(0.0f);  // the zero row that pad entries point at
-
-    for (int s = 0; s < L.n_slabs; ++s) {
-        const int c0 = s * L.cs, ncol = min(L.cs, L.in - c0);
-        if (s) __syncthreads();  // everyone is done reading the previous slab
-        // Stage: element e <-> (column block of 8, batch block of 4, batch row in block, column in block).
-        const int total = ((ncol + 7) >> 3) * (BT / 4) * 32;
-        for (int e = tid; e < total; e += nthr) {
-            const int cl = e & 7, bl = (e >> 3) & 3, t = e >> 5;
-            const int bblk = t % (BT / 4), c = (t / (BT / 4)) * 8 + cl, b = bblk * 4 + bl;
-            if (c < ncol) xs[swz(c, bblk) + bl] = b < nb ? x[(size_t)(b0 + b) * L.in + c0 + c] : VT(0.0f);
-        }
-        __syncthreads();
-
-        for (int i = (tid >> 5) * RPW + sub; i < nrows; i += row_step) {
-            const int r = L.slot[o0 + i];
-            float acc[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[e] = s ? ys[(size_t)(4 * ll + e) * pitch + i] : 0.0f;
-            if (r >= 0) {
-                const int q0 = L.seg[(size_t)r * (L.n_slabs + 1) + s], q1 = L.seg[(size_t)r * (L.n_slabs + 1) + s + 1];
-                const float4* wq = reinterpret_cast<const float4*>(L.values_b + (size_t)r * L.stride_b);
-                const int4* cq = reinterpret_cast<const int4*>(L.cols_b + (size_t)r * L.stride_b);
-#pragma unroll 2
-                for (int q = q0; q < q1; ++q) {
-                    const float4 w = __ldg(wq + q);
-                    const int4 c = __ldg(cq + q);
-                    SmemRow<VT>::fma4(acc, xs, c.x, ll, w.x);
-                    SmemRow<VT>::fma4(acc, xs, c.y, ll, w.y);
-                    SmemRow<VT>::fma4(acc, xs, c.z, ll, w.z);
-                    SmemRow<VT>::fma4(acc, xs, c.w, ll, w.w);
-                }
-            }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) ys[(size_t)(4 * ll + e) * pitch + i] = acc[e];
-        }
+    // Tile metadata: which condensed row each output row is, and where its quads start in every slab.
+    for (int i = tid; i < rt; i += nthr) slot_s[i] = i < nrows ? L.slot[o0 + i] : -1;
+    for (int e = tid; e < rt * (S + 1); e += nthr) {
+        const int i = e / (S + 1), s = e - i * (S + 1);
+        const int r = i < nrows ? L.slot[o0 + i] : -1;
+        seg_s[e] = r >= 0 ? L.seg[(size_t)r * (S + 1) + s] : 0;
+    }
+    if (tid < BT) {  // the zero column that pad entries point at, in both buffers
+        xs0[(size_t)L.cs * BT + tid] = VT(0.0f);
+        xs1[(size_t)L.cs * BT + tid] = VT(0.0f);
     }
     __syncthreads();
-    // Epilogue: consecutive threads write consecutive output rows of one batch row.
+
+    float acc[kMaxRowsPerGroup][4];
+#pragma unroll
+    for (int j = 0; j < kMaxRowsPerGroup; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[j][e] = 0.0f;
+
+    if (warp >= ncw) {
+        // ---------------------------------------------------------------- producers
+        const int ptid = tid - ncw * 32, pthr = kProducerWarps * 32;
+        const bool vec_ok = (L.in & 3) == 0;
+        for (int s = 0; s < S; ++s) {
+            VT* xs = (s & 1) ? xs1 : xs0;
+            if (s >= 2) bar_sync((s & 1) ? kBarEmpty1 : kBarEmpty0, nthr);
+            const int c0 = s * L.cs, ncol = min(L.cs, L.in - c0);
+            // item e <-> (block of 32 columns, block of 4 batch rows, batch row in block, 4-column chunk).
+            const int total = ((ncol + 31) >> 5) * (BT / 4) * 32;
+            for (int e0 = ptid; e0 < total; e0 += pthr * kStageUnroll) {
+                VT v[kStageUnroll][4];
+#pragma unroll
+                for (int u = 0; u < kStageUnroll; ++u) {
+                    const int e = e0 + u * pthr;
+                    const int cl = e & 7, bl = (e >> 3) & 3, t = e >> 5;
+                    const int bblk = t % (BT / 4), c = ((t / (BT / 4)) * 8 + cl) * 4, b = bblk * 4 + bl;
+                    const VT* src = x + (size_t)(b0 + b) * L.in + c0 + c;
+                    if (e < total && b < nb && vec_ok && c + 3 < ncol) {
+                        load4(src, v[u]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            v[u][i] = (e < total && b < nb && c + i < ncol) ? src[i] : VT(0.0f);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kStageUnroll; ++u) {
+                    const int e = e0 + u * pthr;
+                    const int cl = e & 7, bl = (e >> 3) & 3, t = e >> 5;
+                    const int bblk = t % (BT / 4), c = ((t / (BT / 4)) * 8 + cl) * 4;
+                    if (e < total) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (c + i < ncol) xs[swz<BT>(c + i, bblk) + bl] = v[u][i];
+                    }
+                }
+            }
+            __threadfence_block();
+            bar_arrive((s & 1) ? kBarFull1 : kBarFull0, nthr);
+        }
+    } else {
+        // ---------------------------------------------------------------- consumers
+        const int sub = lane / LPR, ll = lane % LPR;
+        const int g = warp * RPW + sub;  // row group within the CTA; its rows are g, g + ngroups, ...
+        unsigned char* wbuf = smem_raw + lay.wbuf_off + (size_t)warp * 2 * RPW * L.maxq * 32;
+        const size_t stage_bytes = (size_t)RPW * L.maxq * 32;
+        const float4* wq = reinterpret_cast<const float4*>(L.wq_b);
+
+        // Copy the quads of item (slab s, row j of this group) into stage `st`; returns nothing, the
+        // group is committed even when empty so that every lane counts the same number of groups.
+        auto prefetch = [&](int s, int j, int st) {
+            const int i = g + j * ngroups;
+            const int r = slot_s[i];
+            if (r >= 0) {
+                const int q0 = seg_s[i * (S + 1) + s], q1 = seg_s[i * (S + 1) + s + 1];
+                const float4* src = wq + ((size_t)r * L.stride_q + q0) * 2;
+                unsigned char* dst = wbuf + st * stage_bytes + (size_t)sub * L.maxq * 32;
+                for (int ch = ll; ch < 2 * (q1 - q0); ch += LPR) cp_async16(dst + ch * 16, src + ch);
+            }
+            cp_async_commit();
+        };
+
+        prefetch(0, 0, 0);
+        int n = 0;
+        for (int s = 0; s < S; ++s) {
+            const VT* xs = (s & 1) ? xs1 : xs0;
+#pragma unroll
+            for (int j = 0; j < kMaxRowsPerGroup; ++j) {
+                if (j < rph) {
+                    __syncwarp();  // every lane is done reading the stage the next prefetch overwrites
+                    const int jn = j + 1 < rph ? j + 1 : 0, sn = j + 1 < rph ? s : s + 1;
+                    if (sn < S) {
+                        prefetch(sn, jn, (n + 1) & 1);
+                        cp_async_wait<1>();
+                    } else {
+                        cp_async_wait<0>();
+                    }
+                    __syncwarp();  // the other lanes' copies of this item are visible too
+                    if (j == 0) bar_sync((s & 1) ? kBarFull1 : kBarFull0, nthr);
+                    const int i = g + j * ngroups;
+                    if (slot_s[i] >= 0) {
+                        const int nq = seg_s[i * (S + 1) + s + 1] - seg_s[i * (S + 1) + s];
+                        const float4* wb = reinterpret_cast<const float4*>(wbuf + (n & 1) * stage_bytes +
+                                                                           (size_t)sub * L.maxq * 32);
+#pragma unroll 2
+                        for (int q = 0; q < nq; ++q) {
+                            const float4 w = wb[2 * q];
+                            const int4 c = *reinterpret_cast<const int4*>(wb + 2 * q + 1);
+                            SmemRow<VT, BT>::fma4(acc[j], xs, c.x, ll, w.x);
+                            SmemRow<VT, BT>::fma4(acc[j], xs, c.y, ll, w.y);
+                            SmemRow<VT, BT>::fma4(acc[j], xs, c.z, ll, w.z);
+                            SmemRow<VT, BT>::fma4(acc[j], xs, c.w, ll, w.w);
+                        }
+                    }
+                    ++n;
+                }
+            }
+            if (s + 2 < S) bar_arrive((s & 1) ? kBarEmpty1 : kBarEmpty0, nthr);
+        }
+    }
+    __syncthreads();  // all slabs consumed: the x buffers are free
+
+    // Epilogue: sums -> ys[b][row] in shared memory, then runs of consecutive output rows per batch row.
+    float* ys = reinterpret_cast<float*>(smem_raw);
+    const int pitch = rt | 1;
+    if (warp < ncw) {
+        const int sub = lane / LPR, ll = lane % LPR, g = warp * RPW + sub;
+#pragma unroll
+        for (int j = 0; j < kMaxRowsPerGroup; ++j)
+            if (j < rph) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) ys[(size_t)(4 * ll + e) * pitch + g + j * ngroups] = acc[j][e];
+            }
+    }
+    __syncthreads();
     for (int e = tid; e < nb * nrows; e += nthr) {
         const int b = e / nrows, i = e - b * nrows;
         const float v = ys[(size_t)b * pitch + i] + L.bias[o0 + i];
@@ -358,7 +516,7 @@ __global__ void cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __res
 // host: launch shapes
 // ------------------------------------------------------------------------------------------------
 struct SplitkShape { int bt, g, threads, rows_per_group, grid_x, grid_y; size_t smem; };
-struct BatchShape { int threads, rt, grid_x, grid_y; size_t smem; };
+struct BatchShape { int ncw, rph, threads, rt, grid_x, grid_y; size_t smem; bool ok; };
 
 int vec_of(int dtype) { return dtype == CFI_BF16 ? 8 : 4; }
 
@@ -382,44 +540,54 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     return s;
 }
 
-size_t batch_smem(const cfi_layer* l, int rt) {
-    const size_t es = l->dtype == CFI_BF16 ? 2 : 4;
-    const size_t xs = (((size_t)(l->d.cs + 1) * kBatchTile * es) + 15) & ~(size_t)15;
-    return xs + (size_t)kBatchTile * (rt | 1) * 4;
+size_t batch_smem(const cfi_layer* l, int ncw, int rph) {
+    const int es = l->dtype == CFI_BF16 ? 2 : 4;
+    const int rt = ncw * (128 / kBatchTile) * rph;
+    const BatchSmem m = batch_smem_layout(l->d.cs, l->d.n_slabs, l->d.maxq, es, kBatchTile, rt, ncw);
+    return std::max(m.total, (size_t)kBatchTile * (rt | 1) * 4);  // the epilogue's y tile reuses the start
 }
 
+// Tile shape: consumer warps (6..12) and rows per row group (1..8) give rt = 2 * ncw * rph rows per CTA.
+// Shared-memory traffic bounds this kernel, so the cost of a CTA is counted in 128-byte wavefronts:
+// gathers and weight reads per entry, the transposed staging of x, plus a fixed start-up; the grid runs
+// in waves of one CTA per SM.
 BatchShape batch_shape(const cfi_layer* l, int batch) {
-    BatchShape s{};
-    s.threads = 256;
-    const int rows_per_pass = (s.threads / 32) * (32 / (kBatchTile / 4));
-    s.grid_y = (batch + kBatchTile - 1) / kBatchTile;
-    // One wave of two CTAs per SM when the problem is small; otherwise tall row tiles, which amortise
-    // the x staging over more rows.
-    const int slots = std::max(1, (2 * l->sm_count) / s.grid_y);
-    int rt = (l->d.out + slots - 1) / slots;
-    rt = ((rt + rows_per_pass - 1) / rows_per_pass) * rows_per_pass;
-    rt = std::max(rows_per_pass, std::min(rt, 128));
-    while (rt > rows_per_pass && 2 * (batch_smem(l, rt) + 1024) > (size_t)228 * 1024) rt -= rows_per_pass;
-    s.rt = rt;
-    s.grid_x = (l->d.out + rt - 1) / rt;
-    s.smem = batch_smem(l, rt);
-    return s;
+    BatchShape best{};
+    best.ok = false;
+    double best_cost = 0;
+    const int es = l->dtype == CFI_BF16 ? 2 : 4;
+    const int grid_y = (batch + kBatchTile - 1) / kBatchTile;
+    const double per_entry = kBatchTile * es / 128.0 + 0.5, staging = (double)l->d.in * kBatchTile * es / 128.0;
+    for (int ncw = 6; ncw <= 12; ++ncw)
+        for (int rph = 1; rph <= kMaxRowsPerGroup; ++rph) {
+            const size_t smem = batch_smem(l, ncw, rph);
+            if (smem > (size_t)l->smem_optin) continue;
+            const int rt = ncw * (128 / kBatchTile) * rph;
+            const int64_t tiles = (int64_t)((l->d.out + rt - 1) / rt) * grid_y;
+            const int64_t waves = (tiles + l->sm_count - 1) / l->sm_count;
+            const double cost = (double)waves * ((double)rt * l->d.stride_q * 4 * per_entry + staging + 4000.0);
+            if (!best.ok || cost < best_cost * 0.999 || (cost < best_cost * 1.001 && ncw > best.ncw)) {
+                best = BatchShape{ncw, rph, (ncw + kProducerWarps) * 32, rt, (l->d.out + rt - 1) / rt, grid_y, smem, true};
+                best_cost = cost;
+            }
+        }
+    return best;
 }
 
 // ------------------------------------------------------------------------------------------------
 // host: launches
 // ------------------------------------------------------------------------------------------------
 // Opt in to more than 48 KB of dynamic shared memory.  The attribute is per kernel and per device, so the
-// largest value set so far is remembered per (instantiation, device) and the runtime is only called to raise it.
+// largest value set so far is remembered per (kernel, device) and the runtime is only called to raise it.
 constexpr int kMaxDevices = 64;
 
-template <typename K>
-cfi_status_t set_smem(K kernel, size_t bytes, int device) {
+template <auto Kernel>
+cfi_status_t set_smem(size_t bytes, int device) {
     static std::atomic<int> granted[kMaxDevices];
     if (bytes <= 48 * 1024) return CFI_OK;
     const bool tracked = device >= 0 && device < kMaxDevices;
     if (tracked && granted[device].load(std::memory_order_relaxed) >= (int)bytes) return CFI_OK;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+    if (cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
         cudaGetLastError();
         return CFI_ERR_SHAPE;
     }
@@ -430,9 +598,8 @@ cfi_status_t set_smem(K kernel, size_t bytes, int device) {
 template <typename VT, int BT, int G>
 cfi_status_t launch_splitk_g(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
                              cudaStream_t st) {
-    auto kern = cfi_splitk_kernel<VT, BT, G>;
-    if (cfi_status_t e = set_smem(kern, s.smem, l->device)) return e;
-    kern<<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, x, y, batch, s.rows_per_group);
+    if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, BT, G>>(s.smem, l->device)) return e;
+    cfi_splitk_kernel<VT, BT, G><<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, x, y, batch, s.rows_per_group);
     return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
 }
 
@@ -466,11 +633,10 @@ cfi_status_t launch_splitk(const cfi_layer* l, const SplitkShape& s, const void*
 template <typename VT>
 cfi_status_t launch_batch(const cfi_layer* l, const BatchShape& s, const void* x, void* y, int batch,
                           cudaStream_t st) {
-    if (s.smem > (size_t)l->smem_optin || s.grid_y > 65535) return CFI_ERR_SHAPE;
-    auto kern = cfi_batch_kernel<VT>;
-    if (cfi_status_t e = set_smem(kern, s.smem, l->device)) return e;
-    kern<<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, static_cast<const VT*>(x), static_cast<VT*>(y),
-                                                              batch, s.rt);
+    if (!s.ok || s.grid_y > 65535) return CFI_ERR_SHAPE;
+    if (cfi_status_t e = set_smem<cfi_batch_kernel<VT, kBatchTile>>(s.smem, l->device)) return e;
+    cfi_batch_kernel<VT, kBatchTile><<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(
+        l->d, static_cast<const VT*>(x), static_cast<VT*>(y), batch, s.rph, s.ncw);
     return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
 }
 
@@ -486,8 +652,8 @@ cfi_status_t launch_simple(const cfi_layer* l, const void* x, void* y, int batch
 }
 
 int choose_variant(const cfi_layer* l, int batch) {
-    (void)l;
-    return batch <= 8 ? CFI_VARIANT_SPLITK : CFI_VARIANT_BATCH;
+    if (batch <= 8) return CFI_VARIANT_SPLITK;
+    return batch_shape(l, batch).ok ? CFI_VARIANT_BATCH : CFI_VARIANT_SPLITK;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -632,41 +798,51 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
         }
         if (st == CFI_OK) st = upload(l, idx_p, &d.indices);
 
-        // ---- large-batch layout
+        // ---- large-batch layout: the fewest slabs (at least two when there is enough to pipeline) for which
+        // two x buffers, the tile metadata and the per-warp weight buffers of the largest tile fit.
         const int es = dtype == CFI_BF16 ? 2 : 4;
-        const int cs_max = std::max(8, (kSlabBytesBudget / (kBatchTile * es) - 1) & ~7);
-        d.n_slabs = std::max(1, (in_features + cs_max - 1) / cs_max);
-        d.cs = std::max(8, (((in_features + d.n_slabs - 1) / d.n_slabs) + 7) & ~7);
-        d.n_slabs = std::max(1, (in_features + d.cs - 1) / d.cs);
-        std::vector<int32_t> seg((size_t)n_active * (d.n_slabs + 1), 0);
-        int max_quads = 0;
-        for (int32_t r = 0; r < n_active; ++r) {
-            int q = 0, j = 0;
-            for (int s = 0; s < d.n_slabs; ++s) {
-                seg[(size_t)r * (d.n_slabs + 1) + s] = q;
-                int cnt = 0;
-                while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) ++j, ++cnt;
-                q += (cnt + 3) / 4;
+        std::vector<int32_t> seg;
+        for (int n_slabs = in_features >= 128 ? 2 : 1;; ++n_slabs) {
+            d.cs = std::max(8, (((in_features + n_slabs - 1) / n_slabs) + 7) & ~7);
+            d.n_slabs = std::max(1, (in_features + d.cs - 1) / d.cs);
+            seg.assign((size_t)n_active * (d.n_slabs + 1), 0);
+            int max_row_quads = 1, maxq = 1;
+            for (int32_t r = 0; r < n_active; ++r) {
+                int q = 0, j = 0;
+                for (int s = 0; s < d.n_slabs; ++s) {
+                    seg[(size_t)r * (d.n_slabs + 1) + s] = q;
+                    int cnt = 0;
+                    while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) ++j, ++cnt;
+                    q += (cnt + 3) / 4;
+                    maxq = std::max(maxq, (cnt + 3) / 4);
+                }
+                seg[(size_t)r * (d.n_slabs + 1) + d.n_slabs] = q;
+                max_row_quads = std::max(max_row_quads, q);
             }
-            seg[(size_t)r * (d.n_slabs + 1) + d.n_slabs] = q;
-            max_quads = std::max(max_quads, q);
+            d.stride_q = max_row_quads;
+            d.maxq = maxq;
+            const BatchSmem m = batch_smem_layout(d.cs, d.n_slabs, d.maxq, es, kBatchTile, 8 * 2 * 4, 8);
+            if (m.total <= (size_t)kBatchSmemBudget || d.cs <= 8) break;
         }
-        d.stride_b = std::max(4, max_quads * 4);
-        std::vector<float> val_b((size_t)n_active * d.stride_b, 0.0f);
-        std::vector<int32_t> col_b((size_t)n_active * d.stride_b, d.cs);
+        struct Quad { float w[4]; int32_t c[4]; };
+        std::vector<Quad> quads((size_t)n_active * d.stride_q);
+        for (auto& q : quads)
+            for (int e = 0; e < 4; ++e) q.w[e] = 0.0f, q.c[e] = d.cs;
         for (int32_t r = 0; r < n_active; ++r) {
             int j = 0;
             for (int s = 0; s < d.n_slabs; ++s) {
-                size_t w = (size_t)r * d.stride_b + (size_t)seg[(size_t)r * (d.n_slabs + 1) + s] * 4;
+                size_t w = (size_t)seg[(size_t)r * (d.n_slabs + 1) + s] * 4;
                 while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) {
-                    val_b[w] = v_sorted[(size_t)r * k + j];
-                    col_b[w] = c_sorted[(size_t)r * k + j] - s * d.cs;
+                    Quad& q = quads[(size_t)r * d.stride_q + w / 4];
+                    q.w[w % 4] = v_sorted[(size_t)r * k + j];
+                    q.c[w % 4] = c_sorted[(size_t)r * k + j] - s * d.cs;
                     ++w, ++j;
                 }
             }
         }
-        if (st == CFI_OK) st = upload(l, val_b, &d.values_b);
-        if (st == CFI_OK) st = upload(l, col_b, &d.cols_b);
+        const Quad* quads_dev = nullptr;
+        if (st == CFI_OK) st = upload(l, quads, &quads_dev);
+        d.wq_b = quads_dev;
         if (st == CFI_OK) st = upload(l, seg, &d.seg);
 
         std::vector<float> bias_h((size_t)out_features, 0.0f);
@@ -772,10 +948,10 @@ extern "C" cfi_status_t cfi_layer_info(const cfi_layer_t* layer, cfi_layer_info_
     info->dtype = layer->dtype, info->act = d.act;
     info->k_padded = d.kp;
     info->batch_slab_columns = d.cs;
-    info->batch_row_stride = d.stride_b;
+    info->batch_row_stride = d.stride_q * 4;
     info->reserved = 0;
     info->weight_bytes_splitk = (int64_t)d.n_active * d.kp * (vs + 4);
-    info->weight_bytes_batch = (int64_t)d.n_active * d.stride_b * 8;
+    info->weight_bytes_batch = (int64_t)d.n_active * d.stride_q * 32;
     info->device_bytes = layer->device_bytes;
     return CFI_OK;
 }
