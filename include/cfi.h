@@ -184,6 +184,29 @@ cfi_status_t cfi_stack_create(cfi_layer_t* const* layers, int32_t n_layers, int3
 cfi_status_t cfi_stack_forward(const cfi_stack_t* stack, const void* x, void* y, int32_t batch, cfi_stream_t stream);
 cfi_status_t cfi_stack_destroy(cfi_stack_t* stack);
 
+/*
+ * cfi_probe_device — measures, on the current device, the ceilings the forward kernels are judged against
+ * and that no vendor figure states: fp32 FMA rate (register-only chains on every SM), shared-memory load
+ * bandwidth (conflict-free 16-byte loads), L2 read bandwidth (every SM streaming a resident 16 MB buffer,
+ * and every SM streaming the same 768 KB, which is how the large-batch kernel reads x) and the time of an
+ * empty kernel launch in a stream.  Takes a few milliseconds; allocates and frees 16 MB; synchronises
+ * the device.  No counterpart in the paper: it reports timings only (Sec. 4.4, Fig. 4).
+ */
+typedef struct {
+    int32_t sm_count;
+    int32_t reserved;
+    int64_t l2_bytes;
+    int64_t smem_per_block_optin;
+    double sm_clock_mhz_nominal;
+    double fma_tflops;              /* 2 flops per FMA                                   */
+    double smem_load_gbs;           /* all SMs together                                  */
+    double l2_read_gbs;             /* distinct lines per SM at a time                   */
+    double l2_read_same_lines_gbs;  /* all SMs reading the same lines at the same time   */
+    double empty_launch_us;
+} cfi_device_probe_t;
+
+cfi_status_t cfi_probe_device(cfi_device_probe_t* probe);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,7 @@ _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, 0: 0, 1: 1, 2: 2, 
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_device_status", "cfi_destroy",
-           "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy")
+           "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_probe_device")
 
 
 class CfiError(RuntimeError):
@@ -42,6 +42,16 @@ class LayerInfo(ctypes.Structure):
                 ("batch_row_stride", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("weight_bytes_splitk", ctypes.c_int64), ("weight_bytes_batch", ctypes.c_int64),
                 ("device_bytes", ctypes.c_int64)]
+
+
+class DeviceProbe(ctypes.Structure):
+    _fields_ = [("sm_count", ctypes.c_int32), ("reserved", ctypes.c_int32), ("l2_bytes", ctypes.c_int64),
+                ("smem_per_block_optin", ctypes.c_int64), ("sm_clock_mhz_nominal", ctypes.c_double),
+                ("fma_tflops", ctypes.c_double), ("smem_load_gbs", ctypes.c_double), ("l2_read_gbs", ctypes.c_double),
+                ("l2_read_same_lines_gbs", ctypes.c_double), ("empty_launch_us", ctypes.c_double)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
 
 
 def library_path() -> str:
@@ -69,6 +79,7 @@ def _load() -> ctypes.CDLL:
     lib.cfi_stack_create.argtypes = [ctypes.POINTER(vp), ci, ci, ctypes.POINTER(vp)]
     lib.cfi_stack_forward.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_stack_destroy.argtypes = [vp]
+    lib.cfi_probe_device.argtypes = [ctypes.POINTER(DeviceProbe)]
     for name in EXPORTS:
         if name != "cfi_status_string":
             getattr(lib, name).restype = ctypes.c_int
@@ -239,3 +250,9 @@ def cfi_stack_forward(stack: Stack, x, y, batch: int, stream=None) -> None:
 
 def cfi_stack_destroy(stack: Stack) -> None:
     stack.close()
+
+
+def cfi_probe_device() -> DeviceProbe:
+    p = DeviceProbe()
+    _check(_lib.cfi_probe_device(ctypes.byref(p)), "cfi_probe_device")
+    return p

@@ -34,8 +34,9 @@ constexpr int kBatchSmemBudget = 216 * 1024;  // what the large-batch kernel may
 struct DevLayer {
     const void* values;      // [n_active][kp]  fp32 or bf16
     const int32_t* indices;  // [n_active][kp]
-    const void* wq_b;        // [n_active][stride_q] quads: 4 fp32 weights, then 4 int32 slab-relative columns
-                             //   (a pad entry has weight 0 and column cs, the staged zero column)
+    const void* wq_b;        // [n_active][stride_q] quads: 4 fp32 weights, then 4 int32 gather offsets: the byte
+                             //   offset of the slab-relative column in the staged slab with the bank permutation
+                             //   key folded in (a pad entry has weight 0 and points at column cs, all zero)
     const int32_t* seg;      // [n_active][n_slabs + 1] first quad of every slab within the row
     const float* bias;       // [out]
     const int32_t* slot;     // [out] -> row of the condensed arrays, or -1 if ablated
@@ -262,39 +263,42 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
 
 // ------------------------------------------------------------------------------------------------
 // CFI_VARIANT_BATCH: large batch.  A CTA owns a tile of `rt` consecutive output rows x BT batch columns
-// and walks the columns of x slab by slab.
+// and walks the columns of x slab by slab.  Two shared-memory buffers hold x slabs transposed,
+// xs[column][BT], so that one column index yields BT contiguous batch values.
 //
-//   producer warps  read x[b0.., slab] (row-major, 16 bytes per lane, whole 128-byte lines per row) and
-//                   store it transposed into one of two shared-memory buffers xs[column][BT], so that a
-//                   single column index yields BT contiguous batch values;
-//   consumer warps  are split into row groups of BT/4 lanes.  A group owns `rph` rows of the tile and
-//                   keeps their partial sums in registers across slabs.  For every (slab, row) it copies
-//                   the row's quads of that slab (4 weights + 4 slab-relative columns = 32 bytes) into a
-//                   warp-private buffer with cp.async one item ahead, then per entry gathers its 4 batch
-//                   values with one 16-byte (fp32) or 8-byte (bf16) shared-memory load and does 4 FMAs.
-//
-// Producers and consumers hand the two x buffers back and forth with named barriers (FULL / EMPTY per
-// buffer).  At the end the sums go through shared memory once more so that y[b, o] is written in runs
-// of consecutive o.
+// Warps are split into row groups of BT/4 lanes.  A group owns RPH rows of the tile and keeps their
+// partial sums in registers across slabs.  Work proceeds in items (slab s, row j of the group):
+//   - the row's quads of the NEXT item (4 weights + 4 gather offsets = 32 bytes each) are copied into a
+//     warp-private buffer with cp.async;
+//   - the thread's share of the NEXT slab of x is requested from global memory (16 bytes per lane, whole
+//     128-byte lines per batch row);
+//   - the current item is computed: per entry one 16-byte (fp32) or 8-byte (bf16) shared-memory gather
+//     of the lane's 4 batch values and 4 FMAs;
+//   - the x values requested above are stored, transposed, into the other buffer.
+// One __syncthreads per slab publishes the next buffer.  Global latency is thus hidden behind an item's
+// arithmetic by every warp, and no warp is reserved for data movement.  At the end the sums go through
+// shared memory once more so that y[b, o] is written in runs of consecutive o.
 //
 // Within a staged column the BT/4 four-value units are permuted by unit ^ ((column / 4) & (BT/4 - 1)).
 // A staging warp reads 4 batch rows x 32 consecutive columns and its transposed stores then fall into
-// 32 different banks; a reading row group still sees consecutive units in distinct banks.
+// 32 different banks; a reading row group still sees consecutive units in distinct banks.  The layer
+// stores, per entry, the byte offset of its column with the permutation key folded in, so a lane's
+// gather address is that offset XOR (its unit number * unit bytes).
+//
+// All shared-memory addresses are 32-bit byte offsets from the start of the dynamic shared memory.
 // ------------------------------------------------------------------------------------------------
-constexpr int kProducerWarps = 4;
 constexpr int kMaxRowsPerGroup = 8;
-constexpr int kStageUnroll = 8;  // 16-byte (fp32) / 8-byte (bf16) x loads in flight per producer thread
+constexpr int kStageUnroll = 8;   // x loads in flight per thread while staging the first slab
+constexpr int kStagePerItem = 4;  // x loads a thread can carry across one item
 
-enum : int { kBarFull0 = 1, kBarFull1 = 2, kBarEmpty0 = 3, kBarEmpty1 = 4 };
+// Dynamic shared memory as bytes; every extern __shared__ array starts at the same address.
+__device__ __forceinline__ unsigned char* smem_at(uint32_t off) {
+    extern __shared__ __align__(128) unsigned char smem_dyn[];
+    return smem_dyn + off;
+}
 
-__device__ __forceinline__ void bar_sync(int id, int count) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-__device__ __forceinline__ void bar_arrive(int id, int count) {
-    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+__device__ __forceinline__ void cp_async16(uint32_t smem_off, const void* gmem_src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_at(smem_off));
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -303,69 +307,94 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-template <int BT>
-__device__ __forceinline__ int swz(int col, int unit) {
-    return (col * (BT / 4) + (unit ^ ((col >> 2) & (BT / 4 - 1)))) << 2;
+// One gather + 4 FMAs.  addr = buffer offset + (entry's stored offset XOR the lane's unit offset).
+template <typename VT>
+__device__ __forceinline__ void fma4(float (&a)[4], uint32_t addr, float w);
+template <>
+__device__ __forceinline__ void fma4<float>(float (&a)[4], uint32_t addr, float w) {
+    const float4 v = *reinterpret_cast<const float4*>(smem_at(addr));
+    a[0] = fmaf(w, v.x, a[0]);
+    a[1] = fmaf(w, v.y, a[1]);
+    a[2] = fmaf(w, v.z, a[2]);
+    a[3] = fmaf(w, v.w, a[3]);
 }
-
-__device__ __forceinline__ void load4(const float* p, float (&v)[4]) {
-    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
-    v[0] = t.x, v[1] = t.y, v[2] = t.z, v[3] = t.w;
+template <>
+__device__ __forceinline__ void fma4<__nv_bfloat16>(float (&a)[4], uint32_t addr, float w) {
+    const uint2 v = *reinterpret_cast<const uint2*>(smem_at(addr));
+    a[0] = fmaf(w, bf16_lo(v.x), a[0]);
+    a[1] = fmaf(w, bf16_hi(v.x), a[1]);
+    a[2] = fmaf(w, bf16_lo(v.y), a[2]);
+    a[3] = fmaf(w, bf16_hi(v.y), a[3]);
 }
-__device__ __forceinline__ void load4(const __nv_bfloat16* p, __nv_bfloat16 (&v)[4]) {
-    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
-    *reinterpret_cast<uint2*>(v) = t;
-}
-
-template <typename XT, int BT> struct SmemRow;
-template <int BT> struct SmemRow<float, BT> {
-    static __device__ __forceinline__ void fma4(float (&a)[4], const float* xs, int col, int ll, float w) {
-        const float4 v = *reinterpret_cast<const float4*>(xs + swz<BT>(col, ll));
-        a[0] = fmaf(w, v.x, a[0]);
-        a[1] = fmaf(w, v.y, a[1]);
-        a[2] = fmaf(w, v.z, a[2]);
-        a[3] = fmaf(w, v.w, a[3]);
-    }
-};
-template <int BT> struct SmemRow<__nv_bfloat16, BT> {
-    static __device__ __forceinline__ void fma4(float (&a)[4], const __nv_bfloat16* xs, int col, int ll, float w) {
-        const uint2 v = *reinterpret_cast<const uint2*>(xs + swz<BT>(col, ll));
-        a[0] = fmaf(w, bf16_lo(v.x), a[0]);
-        a[1] = fmaf(w, bf16_hi(v.x), a[1]);
-        a[2] = fmaf(w, bf16_lo(v.y), a[2]);
-        a[3] = fmaf(w, bf16_hi(v.y), a[3]);
-    }
-};
 
 // Shared-memory carve-up, identical on host and device.
 struct BatchSmem {
-    size_t xs_bytes;    // one x buffer
-    size_t meta_off;    // slot_s[rt] then seg_s[rt][n_slabs + 1]
-    size_t wbuf_off;    // [consumer warp][2 stages][rows per warp][maxq] quads of 32 bytes
+    uint32_t xs_bytes;  // one x buffer
+    uint32_t meta_off;  // slot_s[rt] then seg_s[rt][n_slabs + 1]
+    uint32_t wbuf_off;  // [warp][2 stages][row groups per warp][maxq] quads of 32 bytes
     size_t total;
 };
 __host__ __device__ inline BatchSmem batch_smem_layout(int cs, int n_slabs, int maxq, int elem, int bt, int rt,
-                                                       int consumer_warps) {
+                                                       int warps) {
     BatchSmem m;
-    m.xs_bytes = (((size_t)(cs + 1) * bt * elem) + 127) & ~(size_t)127;
+    m.xs_bytes = (uint32_t)((((size_t)(cs + 1) * bt * elem) + 127) & ~(size_t)127);
     m.meta_off = 2 * m.xs_bytes;
-    const size_t meta = (((size_t)rt * (n_slabs + 2) * 4) + 31) & ~(size_t)31;
+    const uint32_t meta = (uint32_t)((((size_t)rt * (n_slabs + 2) * 4) + 31) & ~(size_t)31);
     m.wbuf_off = m.meta_off + meta;
-    m.total = m.wbuf_off + (size_t)consumer_warps * 2 * (128 / bt) * maxq * 32;
+    m.total = (size_t)m.wbuf_off + (size_t)warps * 2 * (128 / bt) * maxq * 32;
     return m;
 }
 
+// x staging.  A "warp item" wi is 4 batch rows x 32 consecutive columns of a slab: lane = (bl, cl) reads
+// the 4 columns c..c+3 of batch row 4 * bblk + bl, with bblk = wi % (BT/4) and c = 4 * (8 * (wi / (BT/4)) + cl),
+// and stores them to column c + i, unit bblk ^ key, element bl.  The 4 destination addresses differ by one
+// column pitch, so they share a base register.
 template <typename VT, int BT>
+struct Stager {
+    const VT* x;       // &x[b0 + bl][c0 + 4 * cl]  (row bl of the tile, this lane's first column in the slab)
+    size_t row4;       // 4 * in: distance between consecutive bblk
+    int in, cl, bl, nb, ncol;
+    bool vec_ok;
+    __device__ __forceinline__ bool load(int wi, int n_items, VT (&v)[4]) const {
+        const int bblk = wi % (BT / 4), c = ((wi / (BT / 4)) * 8 + cl) * 4, b = bblk * 4 + bl;
+        const VT* src = x + (size_t)bblk * row4 + (wi / (BT / 4)) * 32;
+        const bool live = wi < n_items && b < nb;
+        if (live && vec_ok && c + 3 < ncol) {
+            if constexpr (sizeof(VT) == 4) {
+                const float4 t = __ldg(reinterpret_cast<const float4*>(src));
+                v[0] = t.x, v[1] = t.y, v[2] = t.z, v[3] = t.w;
+            } else {
+                *reinterpret_cast<uint2*>(v) = __ldg(reinterpret_cast<const uint2*>(src));
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[i] = (live && c + i < ncol) ? src[i] : VT(0.0f);
+        }
+        return wi < n_items;
+    }
+    // xs_off: byte offset of the destination buffer.
+    __device__ __forceinline__ void store(int wi, uint32_t xs_off, const VT (&v)[4]) const {
+        const int bblk = wi % (BT / 4), c = ((wi / (BT / 4)) * 8 + cl) * 4;
+        const uint32_t base = xs_off + (uint32_t)sizeof(VT) * (uint32_t)(((c * (BT / 4) + (bblk ^ ((c >> 2) & (BT / 4 - 1)))) << 2) + bl);
+        if (c + 3 < ncol) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) *reinterpret_cast<VT*>(smem_at(base + i * BT * (uint32_t)sizeof(VT))) = v[i];
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (c + i < ncol) *reinterpret_cast<VT*>(smem_at(base + i * BT * (uint32_t)sizeof(VT))) = v[i];
+        }
+    }
+};
+
+template <typename VT, int BT, int RPH>
 __global__ void __launch_bounds__(512, 1)
-cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch, int rph, int ncw) {
+cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch) {
     constexpr int LPR = BT / 4, RPW = 32 / LPR;  // lanes per row group, row groups per warp
-    extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31;
-    const int ngroups = ncw * RPW, rt = ngroups * rph, S = L.n_slabs;
-    const BatchSmem lay = batch_smem_layout(L.cs, S, L.maxq, (int)sizeof(VT), BT, rt, ncw);
-    VT* xs0 = reinterpret_cast<VT*>(smem_raw);
-    VT* xs1 = reinterpret_cast<VT*>(smem_raw + lay.xs_bytes);
-    int32_t* slot_s = reinterpret_cast<int32_t*>(smem_raw + lay.meta_off);
+    const int nwarps = nthr >> 5, ngroups = nwarps * RPW, rt = ngroups * RPH, S = L.n_slabs;
+    const BatchSmem lay = batch_smem_layout(L.cs, S, L.maxq, (int)sizeof(VT), BT, rt, nwarps);
+    int32_t* slot_s = reinterpret_cast<int32_t*>(smem_at(lay.meta_off));
     int32_t* seg_s = slot_s + rt;  // [rt][S + 1]
     const int b0 = blockIdx.y * BT, nb = min(BT, batch - b0);
     const int o0 = blockIdx.x * rt, nrows = min(rt, L.out - o0);
@@ -378,136 +407,120 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
         seg_s[e] = r >= 0 ? L.seg[(size_t)r * (S + 1) + s] : 0;
     }
     if (tid < BT) {  // the zero column that pad entries point at, in both buffers
-        xs0[(size_t)L.cs * BT + tid] = VT(0.0f);
-        xs1[(size_t)L.cs * BT + tid] = VT(0.0f);
+        reinterpret_cast<VT*>(smem_at(0))[(size_t)L.cs * BT + tid] = VT(0.0f);
+        reinterpret_cast<VT*>(smem_at(lay.xs_bytes))[(size_t)L.cs * BT + tid] = VT(0.0f);
+    }
+
+    Stager<VT, BT> st;
+    st.in = L.in, st.cl = lane & 7, st.bl = lane >> 3, st.nb = nb, st.vec_ok = (L.in & 3) == 0;
+    st.row4 = (size_t)4 * L.in;
+    const VT* x_lane = x + (size_t)(b0 + st.bl) * L.in + 4 * st.cl;
+
+    // Slab 0: everybody stages, several requests in flight per thread.
+    {
+        st.x = x_lane, st.ncol = min(L.cs, L.in);
+        const int n_items = ((st.ncol + 31) >> 5) * (BT / 4);
+        for (int w0 = warp; w0 < n_items; w0 += nwarps * kStageUnroll) {
+            VT v[kStageUnroll][4];
+#pragma unroll
+            for (int u = 0; u < kStageUnroll; ++u) st.load(w0 + u * nwarps, n_items, v[u]);
+#pragma unroll
+            for (int u = 0; u < kStageUnroll; ++u)
+                if (w0 + u * nwarps < n_items) st.store(w0 + u * nwarps, 0u, v[u]);
+        }
     }
     __syncthreads();
 
-    float acc[kMaxRowsPerGroup][4];
+    const int sub = lane / LPR, ll = lane % LPR;
+    const uint32_t lane_key = (uint32_t)(ll * 4 * (int)sizeof(VT));
+    const int g = warp * RPW + sub;  // row group within the CTA; its rows are g, g + ngroups, ...
+    const uint32_t stage_bytes = (uint32_t)(RPW * L.maxq * 32);
+    const uint32_t wbuf = lay.wbuf_off + (uint32_t)warp * 2 * stage_bytes + (uint32_t)sub * L.maxq * 32;
+    const float4* wq = reinterpret_cast<const float4*>(L.wq_b);
+
+    // Copy the quads of item (slab s, row j of this group) into stage `st`.  The group is committed even
+    // when empty so that every lane counts the same number of groups.
+    auto prefetch = [&](int s, int j, int stage) {
+        const int i = g + j * ngroups;
+        const int r = slot_s[i];
+        if (r >= 0) {
+            const int q0 = seg_s[i * (S + 1) + s], q1 = seg_s[i * (S + 1) + s + 1];
+            const float4* src = wq + ((size_t)r * L.stride_q + q0) * 2;
+            const uint32_t dst = wbuf + stage * stage_bytes;
+            for (int ch = ll; ch < 2 * (q1 - q0); ch += LPR) cp_async16(dst + ch * 16, src + ch);
+        }
+        cp_async_commit();
+    };
+
+    float acc[RPH][4];
 #pragma unroll
-    for (int j = 0; j < kMaxRowsPerGroup; ++j)
+    for (int j = 0; j < RPH; ++j)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[j][e] = 0.0f;
 
-    if (warp >= ncw) {
-        // ---------------------------------------------------------------- producers
-        const int ptid = tid - ncw * 32, pthr = kProducerWarps * 32;
-        const bool vec_ok = (L.in & 3) == 0;
-        for (int s = 0; s < S; ++s) {
-            VT* xs = (s & 1) ? xs1 : xs0;
-            if (s >= 2) bar_sync((s & 1) ? kBarEmpty1 : kBarEmpty0, nthr);
-            const int c0 = s * L.cs, ncol = min(L.cs, L.in - c0);
-            // item e <-> (block of 32 columns, block of 4 batch rows, batch row in block, 4-column chunk).
-            const int total = ((ncol + 31) >> 5) * (BT / 4) * 32;
-            for (int e0 = ptid; e0 < total; e0 += pthr * kStageUnroll) {
-                VT v[kStageUnroll][4];
+    prefetch(0, 0, 0);
+    int n = 0;
+    for (int s = 0; s < S; ++s) {
+        const uint32_t xs_off = (s & 1) ? lay.xs_bytes : 0u, xs_next = (s & 1) ? 0u : lay.xs_bytes;
+        const int c0n = (s + 1) * L.cs;
+        st.ncol = s + 1 < S ? min(L.cs, L.in - c0n) : 0;
+        st.x = x_lane + c0n;
+        const int n_items = ((st.ncol + 31) >> 5) * (BT / 4);  // warp items of the next slab
 #pragma unroll
-                for (int u = 0; u < kStageUnroll; ++u) {
-                    const int e = e0 + u * pthr;
-                    const int cl = e & 7, bl = (e >> 3) & 3, t = e >> 5;
-                    const int bblk = t % (BT / 4), c = ((t / (BT / 4)) * 8 + cl) * 4, b = bblk * 4 + bl;
-                    const VT* src = x + (size_t)(b0 + b) * L.in + c0 + c;
-                    if (e < total && b < nb && vec_ok && c + 3 < ncol) {
-                        load4(src, v[u]);
-                    } else {
+        for (int j = 0; j < RPH; ++j) {
+            __syncwarp();  // every lane is done reading the stage the next prefetch overwrites
+            const int jn = j + 1 < RPH ? j + 1 : 0, sn = j + 1 < RPH ? s : s + 1;
+            if (sn < S) prefetch(sn, jn, (n + 1) & 1);
+            VT xv[kStagePerItem][4];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            v[u][i] = (e < total && b < nb && c + i < ncol) ? src[i] : VT(0.0f);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < kStageUnroll; ++u) {
-                    const int e = e0 + u * pthr;
-                    const int cl = e & 7, bl = (e >> 3) & 3, t = e >> 5;
-                    const int bblk = t % (BT / 4), c = ((t / (BT / 4)) * 8 + cl) * 4;
-                    if (e < total) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            if (c + i < ncol) xs[swz<BT>(c + i, bblk) + bl] = v[u][i];
-                    }
-                }
-            }
-            __threadfence_block();
-            bar_arrive((s & 1) ? kBarFull1 : kBarFull0, nthr);
-        }
-    } else {
-        // ---------------------------------------------------------------- consumers
-        const int sub = lane / LPR, ll = lane % LPR;
-        const int g = warp * RPW + sub;  // row group within the CTA; its rows are g, g + ngroups, ...
-        unsigned char* wbuf = smem_raw + lay.wbuf_off + (size_t)warp * 2 * RPW * L.maxq * 32;
-        const size_t stage_bytes = (size_t)RPW * L.maxq * 32;
-        const float4* wq = reinterpret_cast<const float4*>(L.wq_b);
-
-        // Copy the quads of item (slab s, row j of this group) into stage `st`; returns nothing, the
-        // group is committed even when empty so that every lane counts the same number of groups.
-        auto prefetch = [&](int s, int j, int st) {
+            for (int u = 0; u < kStagePerItem; ++u) st.load(warp + (j * kStagePerItem + u) * nwarps, n_items, xv[u]);
+            if (sn < S) cp_async_wait<1>();
+            else cp_async_wait<0>();
+            __syncwarp();  // the other lanes' copies of this item are visible too
             const int i = g + j * ngroups;
-            const int r = slot_s[i];
-            if (r >= 0) {
-                const int q0 = seg_s[i * (S + 1) + s], q1 = seg_s[i * (S + 1) + s + 1];
-                const float4* src = wq + ((size_t)r * L.stride_q + q0) * 2;
-                unsigned char* dst = wbuf + st * stage_bytes + (size_t)sub * L.maxq * 32;
-                for (int ch = ll; ch < 2 * (q1 - q0); ch += LPR) cp_async16(dst + ch * 16, src + ch);
-            }
-            cp_async_commit();
-        };
-
-        prefetch(0, 0, 0);
-        int n = 0;
-        for (int s = 0; s < S; ++s) {
-            const VT* xs = (s & 1) ? xs1 : xs0;
-#pragma unroll
-            for (int j = 0; j < kMaxRowsPerGroup; ++j) {
-                if (j < rph) {
-                    __syncwarp();  // every lane is done reading the stage the next prefetch overwrites
-                    const int jn = j + 1 < rph ? j + 1 : 0, sn = j + 1 < rph ? s : s + 1;
-                    if (sn < S) {
-                        prefetch(sn, jn, (n + 1) & 1);
-                        cp_async_wait<1>();
-                    } else {
-                        cp_async_wait<0>();
-                    }
-                    __syncwarp();  // the other lanes' copies of this item are visible too
-                    if (j == 0) bar_sync((s & 1) ? kBarFull1 : kBarFull0, nthr);
-                    const int i = g + j * ngroups;
-                    if (slot_s[i] >= 0) {
-                        const int nq = seg_s[i * (S + 1) + s + 1] - seg_s[i * (S + 1) + s];
-                        const float4* wb = reinterpret_cast<const float4*>(wbuf + (n & 1) * stage_bytes +
-                                                                           (size_t)sub * L.maxq * 32);
+            if (slot_s[i] >= 0) {
+                const int nq = seg_s[i * (S + 1) + s + 1] - seg_s[i * (S + 1) + s];
+                const uint32_t wb = wbuf + (n & 1) * stage_bytes;
 #pragma unroll 2
-                        for (int q = 0; q < nq; ++q) {
-                            const float4 w = wb[2 * q];
-                            const int4 c = *reinterpret_cast<const int4*>(wb + 2 * q + 1);
-                            SmemRow<VT, BT>::fma4(acc[j], xs, c.x, ll, w.x);
-                            SmemRow<VT, BT>::fma4(acc[j], xs, c.y, ll, w.y);
-                            SmemRow<VT, BT>::fma4(acc[j], xs, c.z, ll, w.z);
-                            SmemRow<VT, BT>::fma4(acc[j], xs, c.w, ll, w.w);
-                        }
-                    }
-                    ++n;
+                for (int q = 0; q < nq; ++q) {
+                    const float4 w = *reinterpret_cast<const float4*>(smem_at(wb + q * 32));
+                    const int4 c = *reinterpret_cast<const int4*>(smem_at(wb + q * 32 + 16));
+                    fma4<VT>(acc[j], xs_off + ((uint32_t)c.x ^ lane_key), w.x);
+                    fma4<VT>(acc[j], xs_off + ((uint32_t)c.y ^ lane_key), w.y);
+                    fma4<VT>(acc[j], xs_off + ((uint32_t)c.z ^ lane_key), w.z);
+                    fma4<VT>(acc[j], xs_off + ((uint32_t)c.w ^ lane_key), w.w);
                 }
             }
-            if (s + 2 < S) bar_arrive((s & 1) ? kBarEmpty1 : kBarEmpty0, nthr);
+#pragma unroll
+            for (int u = 0; u < kStagePerItem; ++u) {
+                const int wi = warp + (j * kStagePerItem + u) * nwarps;
+                if (wi < n_items) st.store(wi, xs_next, xv[u]);
+            }
+            ++n;
         }
+        // Whatever of the next slab the row items did not cover.
+        for (int w0 = warp + RPH * kStagePerItem * nwarps; w0 < n_items; w0 += nwarps * kStagePerItem) {
+            VT xv[kStagePerItem][4];
+#pragma unroll
+            for (int u = 0; u < kStagePerItem; ++u) st.load(w0 + u * nwarps, n_items, xv[u]);
+#pragma unroll
+            for (int u = 0; u < kStagePerItem; ++u)
+                if (w0 + u * nwarps < n_items) st.store(w0 + u * nwarps, xs_next, xv[u]);
+        }
+        __syncthreads();  // next slab is complete, and nobody reads this slab's buffer any more
     }
-    __syncthreads();  // all slabs consumed: the x buffers are free
 
     // Epilogue: sums -> ys[b][row] in shared memory, then runs of consecutive output rows per batch row.
-    float* ys = reinterpret_cast<float*>(smem_raw);
+    float* ys = reinterpret_cast<float*>(smem_at(0));
     const int pitch = rt | 1;
-    if (warp < ncw) {
-        const int sub = lane / LPR, ll = lane % LPR, g = warp * RPW + sub;
 #pragma unroll
-        for (int j = 0; j < kMaxRowsPerGroup; ++j)
-            if (j < rph) {
+    for (int j = 0; j < RPH; ++j)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) ys[(size_t)(4 * ll + e) * pitch + g + j * ngroups] = acc[j][e];
-            }
-    }
+        for (int e = 0; e < 4; ++e) ys[(4 * ll + e) * pitch + g + j * ngroups] = acc[j][e];
     __syncthreads();
     for (int e = tid; e < nb * nrows; e += nthr) {
         const int b = e / nrows, i = e - b * nrows;
-        const float v = ys[(size_t)b * pitch + i] + L.bias[o0 + i];
+        const float v = ys[b * pitch + i] + L.bias[o0 + i];
         from_f32(&y[(size_t)(b0 + b) * L.out + o0 + i], activate(v, L.act));
     }
 }
@@ -516,7 +529,7 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 // host: launch shapes
 // ------------------------------------------------------------------------------------------------
 struct SplitkShape { int bt, g, threads, rows_per_group, grid_x, grid_y; size_t smem; };
-struct BatchShape { int ncw, rph, threads, rt, grid_x, grid_y; size_t smem; bool ok; };
+struct BatchShape { int warps, rph, threads, rt, grid_x, grid_y; size_t smem; bool ok; };
 
 int vec_of(int dtype) { return dtype == CFI_BF16 ? 8 : 4; }
 
@@ -540,14 +553,14 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     return s;
 }
 
-size_t batch_smem(const cfi_layer* l, int ncw, int rph) {
+size_t batch_smem(const cfi_layer* l, int warps, int rph) {
     const int es = l->dtype == CFI_BF16 ? 2 : 4;
-    const int rt = ncw * (128 / kBatchTile) * rph;
-    const BatchSmem m = batch_smem_layout(l->d.cs, l->d.n_slabs, l->d.maxq, es, kBatchTile, rt, ncw);
+    const int rt = warps * (128 / kBatchTile) * rph;
+    const BatchSmem m = batch_smem_layout(l->d.cs, l->d.n_slabs, l->d.maxq, es, kBatchTile, rt, warps);
     return std::max(m.total, (size_t)kBatchTile * (rt | 1) * 4);  // the epilogue's y tile reuses the start
 }
 
-// Tile shape: consumer warps (6..12) and rows per row group (1..8) give rt = 2 * ncw * rph rows per CTA.
+// Tile shape: warps (6..16) and rows per row group (1..8) give rt = 2 * warps * rph rows per CTA.
 // Shared-memory traffic bounds this kernel, so the cost of a CTA is counted in 128-byte wavefronts:
 // gathers and weight reads per entry, the transposed staging of x, plus a fixed start-up; the grid runs
 // in waves of one CTA per SM.
@@ -558,16 +571,16 @@ BatchShape batch_shape(const cfi_layer* l, int batch) {
     const int es = l->dtype == CFI_BF16 ? 2 : 4;
     const int grid_y = (batch + kBatchTile - 1) / kBatchTile;
     const double per_entry = kBatchTile * es / 128.0 + 0.5, staging = (double)l->d.in * kBatchTile * es / 128.0;
-    for (int ncw = 6; ncw <= 12; ++ncw)
+    for (int warps = 6; warps <= 16; ++warps)
         for (int rph = 1; rph <= kMaxRowsPerGroup; ++rph) {
-            const size_t smem = batch_smem(l, ncw, rph);
+            const size_t smem = batch_smem(l, warps, rph);
             if (smem > (size_t)l->smem_optin) continue;
-            const int rt = ncw * (128 / kBatchTile) * rph;
+            const int rt = warps * (128 / kBatchTile) * rph;
             const int64_t tiles = (int64_t)((l->d.out + rt - 1) / rt) * grid_y;
             const int64_t waves = (tiles + l->sm_count - 1) / l->sm_count;
             const double cost = (double)waves * ((double)rt * l->d.stride_q * 4 * per_entry + staging + 4000.0);
-            if (!best.ok || cost < best_cost * 0.999 || (cost < best_cost * 1.001 && ncw > best.ncw)) {
-                best = BatchShape{ncw, rph, (ncw + kProducerWarps) * 32, rt, (l->d.out + rt - 1) / rt, grid_y, smem, true};
+            if (!best.ok || cost < best_cost * 0.999 || (cost < best_cost * 1.001 && warps > best.warps)) {
+                best = BatchShape{warps, rph, warps * 32, rt, (l->d.out + rt - 1) / rt, grid_y, smem, true};
                 best_cost = cost;
             }
         }
@@ -630,14 +643,30 @@ cfi_status_t launch_splitk(const cfi_layer* l, const SplitkShape& s, const void*
     return CFI_ERR_SHAPE;
 }
 
+template <typename VT, int RPH>
+cfi_status_t launch_batch_rph(const cfi_layer* l, const BatchShape& s, const VT* x, VT* y, int batch, cudaStream_t st) {
+    if (cfi_status_t e = set_smem<cfi_batch_kernel<VT, kBatchTile, RPH>>(s.smem, l->device)) return e;
+    cfi_batch_kernel<VT, kBatchTile, RPH><<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, x, y, batch);
+    return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+}
+
 template <typename VT>
 cfi_status_t launch_batch(const cfi_layer* l, const BatchShape& s, const void* x, void* y, int batch,
                           cudaStream_t st) {
     if (!s.ok || s.grid_y > 65535) return CFI_ERR_SHAPE;
-    if (cfi_status_t e = set_smem<cfi_batch_kernel<VT, kBatchTile>>(s.smem, l->device)) return e;
-    cfi_batch_kernel<VT, kBatchTile><<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(
-        l->d, static_cast<const VT*>(x), static_cast<VT*>(y), batch, s.rph, s.ncw);
-    return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+    const VT* xx = static_cast<const VT*>(x);
+    VT* yy = static_cast<VT*>(y);
+    switch (s.rph) {
+        case 1: return launch_batch_rph<VT, 1>(l, s, xx, yy, batch, st);
+        case 2: return launch_batch_rph<VT, 2>(l, s, xx, yy, batch, st);
+        case 3: return launch_batch_rph<VT, 3>(l, s, xx, yy, batch, st);
+        case 4: return launch_batch_rph<VT, 4>(l, s, xx, yy, batch, st);
+        case 5: return launch_batch_rph<VT, 5>(l, s, xx, yy, batch, st);
+        case 6: return launch_batch_rph<VT, 6>(l, s, xx, yy, batch, st);
+        case 7: return launch_batch_rph<VT, 7>(l, s, xx, yy, batch, st);
+        case 8: return launch_batch_rph<VT, 8>(l, s, xx, yy, batch, st);
+    }
+    return CFI_ERR_SHAPE;
 }
 
 template <typename VT>
@@ -821,13 +850,13 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
             }
             d.stride_q = max_row_quads;
             d.maxq = maxq;
-            const BatchSmem m = batch_smem_layout(d.cs, d.n_slabs, d.maxq, es, kBatchTile, 8 * 2 * 4, 8);
+            const BatchSmem m = batch_smem_layout(d.cs, d.n_slabs, d.maxq, es, kBatchTile, 128, 8);
             if (m.total <= (size_t)kBatchSmemBudget || d.cs <= 8) break;
         }
         struct Quad { float w[4]; int32_t c[4]; };
         std::vector<Quad> quads((size_t)n_active * d.stride_q);
         for (auto& q : quads)
-            for (int e = 0; e < 4; ++e) q.w[e] = 0.0f, q.c[e] = d.cs;
+            for (int e = 0; e < 4; ++e) q.w[e] = 0.0f, q.c[e] = d.cs * kBatchTile * es;
         for (int32_t r = 0; r < n_active; ++r) {
             int j = 0;
             for (int s = 0; s < d.n_slabs; ++s) {
@@ -835,7 +864,8 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                 while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) {
                     Quad& q = quads[(size_t)r * d.stride_q + w / 4];
                     q.w[w % 4] = v_sorted[(size_t)r * k + j];
-                    q.c[w % 4] = c_sorted[(size_t)r * k + j] - s * d.cs;
+                    const int col = c_sorted[(size_t)r * k + j] - s * d.cs;
+                    q.c[w % 4] = col * kBatchTile * es + ((col >> 2) & (kBatchTile / 4 - 1)) * 4 * es;
                     ++w, ++j;
                 }
             }
