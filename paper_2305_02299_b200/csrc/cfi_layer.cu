@@ -37,7 +37,7 @@ struct DevLayer {
     const void* wq_b;        // [n_active][stride_q] quads: 4 fp32 weights, then 4 int32 gather offsets: the byte
                              //   offset of the slab-relative column in the staged slab with the bank permutation
                              //   key folded in (a pad entry has weight 0 and points at column cs, all zero)
-    const int32_t* seg;      // [n_active][n_slabs + 1] first quad of every slab within the row
+    const int32_t* seg;      // [out][n_slabs + 1] first quad of every slab within the output row's condensed row
     const float* bias;       // [out]
     const int32_t* slot;     // [out] -> row of the condensed arrays, or -1 if ablated
     int32_t* status;
@@ -270,26 +270,25 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
 // partial sums in registers across slabs.  Work proceeds in items (slab s, row j of the group):
 //   - the row's quads of the NEXT item (4 weights + 4 gather offsets = 32 bytes each) are copied into a
 //     warp-private buffer with cp.async;
-//   - the thread's share of the NEXT slab of x is requested from global memory (16 bytes per lane, whole
-//     128-byte lines per batch row);
+//   - the thread's share of the NEXT slab of x, a 4 x 4 block, is requested from global memory (16 bytes
+//     per lane and batch row, whole 128-byte lines per row and warp);
 //   - the current item is computed: per entry one 16-byte (fp32) or 8-byte (bf16) shared-memory gather
 //     of the lane's 4 batch values and 4 FMAs;
-//   - the x values requested above are stored, transposed, into the other buffer.
+//   - the block requested above is transposed in registers and stored into the other buffer.
 // One __syncthreads per slab publishes the next buffer.  Global latency is thus hidden behind an item's
 // arithmetic by every warp, and no warp is reserved for data movement.  At the end the sums go through
 // shared memory once more so that y[b, o] is written in runs of consecutive o.
 //
 // Within a staged column the BT/4 four-value units are permuted by unit ^ ((column / 4) & (BT/4 - 1)).
-// A staging warp reads 4 batch rows x 32 consecutive columns and its transposed stores then fall into
-// 32 different banks; a reading row group still sees consecutive units in distinct banks.  The layer
+// The staging stores (one unit per lane) then fall into distinct banks within every quarter warp, and a
+// reading row group still sees consecutive units in distinct banks.  The layer
 // stores, per entry, the byte offset of its column with the permutation key folded in, so a lane's
 // gather address is that offset XOR (its unit number * unit bytes).
 //
 // All shared-memory addresses are 32-bit byte offsets from the start of the dynamic shared memory.
 // ------------------------------------------------------------------------------------------------
 constexpr int kMaxRowsPerGroup = 8;
-constexpr int kStageUnroll = 8;   // x loads in flight per thread while staging the first slab
-constexpr int kStagePerItem = 4;  // x loads a thread can carry across one item
+constexpr int kStageUnroll = 2;  // 4 x 4 blocks (4 loads each) in flight per thread outside the row items
 
 // Dynamic shared memory as bytes; every extern __shared__ array starts at the same address.
 __device__ __forceinline__ unsigned char* smem_at(uint32_t off) {
@@ -330,7 +329,7 @@ __device__ __forceinline__ void fma4<__nv_bfloat16>(float (&a)[4], uint32_t addr
 // Shared-memory carve-up, identical on host and device.
 struct BatchSmem {
     uint32_t xs_bytes;  // one x buffer
-    uint32_t meta_off;  // slot_s[rt] then seg_s[rt][n_slabs + 1]
+    uint32_t meta_off;  // slot_s[rt], bias_s[rt], seg_s[rt][n_slabs + 1]
     uint32_t wbuf_off;  // [warp][2 stages][row groups per warp][maxq] quads of 32 bytes
     size_t total;
 };
@@ -339,50 +338,68 @@ __host__ __device__ inline BatchSmem batch_smem_layout(int cs, int n_slabs, int 
     BatchSmem m;
     m.xs_bytes = (uint32_t)((((size_t)(cs + 1) * bt * elem) + 127) & ~(size_t)127);
     m.meta_off = 2 * m.xs_bytes;
-    const uint32_t meta = (uint32_t)((((size_t)rt * (n_slabs + 2) * 4) + 31) & ~(size_t)31);
+    const uint32_t meta = (uint32_t)((((size_t)rt * (n_slabs + 3) * 4) + 31) & ~(size_t)31);
     m.wbuf_off = m.meta_off + meta;
     m.total = (size_t)m.wbuf_off + (size_t)warps * 2 * (128 / bt) * maxq * 32;
     return m;
 }
 
-// x staging.  A "warp item" wi is 4 batch rows x 32 consecutive columns of a slab: lane = (bl, cl) reads
-// the 4 columns c..c+3 of batch row 4 * bblk + bl, with bblk = wi % (BT/4) and c = 4 * (8 * (wi / (BT/4)) + cl),
-// and stores them to column c + i, unit bblk ^ key, element bl.  The 4 destination addresses differ by one
-// column pitch, so they share a base register.
+// x staging.  A "warp block" wb is 16 batch rows x 32 consecutive columns of a slab.  Lane = (cl, uq): it reads
+// the 4 columns c..c+3 (c = 32 * (wb / (BT/16)) + 4 * cl) of the 4 batch rows of unit u, one 16-byte (fp32) or
+// 8-byte (bf16) load per row, transposes the 4 x 4 block in registers and writes column c + j's 4 batch values
+// with one 16-byte / 8-byte store to unit u ^ key(c).  Per load instruction a warp reads 128 contiguous bytes
+// of 4 batch rows; per store instruction every quarter (fp32) or half (bf16) of the warp hits distinct banks.
 template <typename VT, int BT>
 struct Stager {
-    const VT* x;       // &x[b0 + bl][c0 + 4 * cl]  (row bl of the tile, this lane's first column in the slab)
-    size_t row4;       // 4 * in: distance between consecutive bblk
-    int in, cl, bl, nb, ncol;
+    const VT* x;   // &x[b0][c0]: first batch row of the tile, first column of the slab
+    int in, cl, uq, nb, ncol;
     bool vec_ok;
-    __device__ __forceinline__ bool load(int wi, int n_items, VT (&v)[4]) const {
-        const int bblk = wi % (BT / 4), c = ((wi / (BT / 4)) * 8 + cl) * 4, b = bblk * 4 + bl;
-        const VT* src = x + (size_t)bblk * row4 + (wi / (BT / 4)) * 32;
-        const bool live = wi < n_items && b < nb;
-        if (live && vec_ok && c + 3 < ncol) {
-            if constexpr (sizeof(VT) == 4) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(src));
-                v[0] = t.x, v[1] = t.y, v[2] = t.z, v[3] = t.w;
-            } else {
-                *reinterpret_cast<uint2*>(v) = __ldg(reinterpret_cast<const uint2*>(src));
-            }
-        } else {
+    struct alignas(16) Block { VT v[4][4]; };  // [batch row in unit][column in chunk]
+
+    __device__ __forceinline__ int unit_of(int wb) const { return ((uq & 1) * 8 + (uq >> 1) * 4 + (wb & 3)) & (BT / 4 - 1); }
+
+    __device__ __forceinline__ void load(int wb, int n_blocks, Block& blk) const {
+        static_assert(BT == 64, "lane mapping assumes 16 units per staged column");
+        const int u = unit_of(wb), c = ((wb >> 2) * 8 + cl) * 4;
+        const bool live = wb < n_blocks;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) v[i] = (live && c + i < ncol) ? src[i] : VT(0.0f);
+        for (int i = 0; i < 4; ++i) {
+            const int b = 4 * u + i;
+            const VT* src = x + (size_t)b * in + c;
+            if (live && b < nb && vec_ok && c + 3 < ncol) {
+                if constexpr (sizeof(VT) == 4) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(src));
+                    blk.v[i][0] = t.x, blk.v[i][1] = t.y, blk.v[i][2] = t.z, blk.v[i][3] = t.w;
+                } else {
+                    *reinterpret_cast<uint2*>(blk.v[i]) = __ldg(reinterpret_cast<const uint2*>(src));
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) blk.v[i][j] = (live && b < nb && c + j < ncol) ? src[j] : VT(0.0f);
+            }
         }
-        return wi < n_items;
     }
     // xs_off: byte offset of the destination buffer.
-    __device__ __forceinline__ void store(int wi, uint32_t xs_off, const VT (&v)[4]) const {
-        const int bblk = wi % (BT / 4), c = ((wi / (BT / 4)) * 8 + cl) * 4;
-        const uint32_t base = xs_off + (uint32_t)sizeof(VT) * (uint32_t)(((c * (BT / 4) + (bblk ^ ((c >> 2) & (BT / 4 - 1)))) << 2) + bl);
-        if (c + 3 < ncol) {
+    __device__ __forceinline__ void store(int wb, uint32_t xs_off, const Block& blk) const {
+        const int u = unit_of(wb), c = ((wb >> 2) * 8 + cl) * 4;
+        constexpr uint32_t unit_bytes = 4 * sizeof(VT), col_bytes = BT * sizeof(VT);
+        const uint32_t base = xs_off + (uint32_t)c * col_bytes + (uint32_t)(u ^ ((c >> 2) & (BT / 4 - 1))) * unit_bytes;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) *reinterpret_cast<VT*>(smem_at(base + i * BT * (uint32_t)sizeof(VT))) = v[i];
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (c + i < ncol) *reinterpret_cast<VT*>(smem_at(base + i * BT * (uint32_t)sizeof(VT))) = v[i];
+        for (int j = 0; j < 4; ++j) {
+            if (c + j < ncol) {
+                if constexpr (sizeof(VT) == 4) {
+                    *reinterpret_cast<float4*>(smem_at(base + j * col_bytes)) =
+                        make_float4(blk.v[0][j], blk.v[1][j], blk.v[2][j], blk.v[3][j]);
+                } else {
+                    const uint32_t* w0 = reinterpret_cast<const uint32_t*>(blk.v[0]);
+                    const uint32_t* w1 = reinterpret_cast<const uint32_t*>(blk.v[1]);
+                    const uint32_t* w2 = reinterpret_cast<const uint32_t*>(blk.v[2]);
+                    const uint32_t* w3 = reinterpret_cast<const uint32_t*>(blk.v[3]);
+                    const uint32_t sel = (j & 1) ? 0x7632u : 0x5410u;
+                    *reinterpret_cast<uint2*>(smem_at(base + j * col_bytes)) =
+                        make_uint2(__byte_perm(w0[j >> 1], w1[j >> 1], sel), __byte_perm(w2[j >> 1], w3[j >> 1], sel));
+                }
+            }
         }
     }
 };
@@ -395,38 +412,37 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
     const int nwarps = nthr >> 5, ngroups = nwarps * RPW, rt = ngroups * RPH, S = L.n_slabs;
     const BatchSmem lay = batch_smem_layout(L.cs, S, L.maxq, (int)sizeof(VT), BT, rt, nwarps);
     int32_t* slot_s = reinterpret_cast<int32_t*>(smem_at(lay.meta_off));
-    int32_t* seg_s = slot_s + rt;  // [rt][S + 1]
+    float* bias_s = reinterpret_cast<float*>(slot_s + rt);
+    int32_t* seg_s = slot_s + 2 * rt;  // [rt][S + 1]
     const int b0 = blockIdx.y * BT, nb = min(BT, batch - b0);
     const int o0 = blockIdx.x * rt, nrows = min(rt, L.out - o0);
 
-    // Tile metadata: which condensed row each output row is, and where its quads start in every slab.
-    for (int i = tid; i < rt; i += nthr) slot_s[i] = i < nrows ? L.slot[o0 + i] : -1;
-    for (int e = tid; e < rt * (S + 1); e += nthr) {
-        const int i = e / (S + 1), s = e - i * (S + 1);
-        const int r = i < nrows ? L.slot[o0 + i] : -1;
-        seg_s[e] = r >= 0 ? L.seg[(size_t)r * (S + 1) + s] : 0;
+    // Tile metadata: which condensed row each output row is, where its quads start in every slab, its bias.
+    for (int i = tid; i < rt; i += nthr) {
+        slot_s[i] = i < nrows ? L.slot[o0 + i] : -1;
+        bias_s[i] = i < nrows ? L.bias[o0 + i] : 0.0f;
     }
+    for (int e = tid; e < rt * (S + 1); e += nthr) seg_s[e] = e < nrows * (S + 1) ? L.seg[(size_t)o0 * (S + 1) + e] : 0;
     if (tid < BT) {  // the zero column that pad entries point at, in both buffers
         reinterpret_cast<VT*>(smem_at(0))[(size_t)L.cs * BT + tid] = VT(0.0f);
         reinterpret_cast<VT*>(smem_at(lay.xs_bytes))[(size_t)L.cs * BT + tid] = VT(0.0f);
     }
 
     Stager<VT, BT> st;
-    st.in = L.in, st.cl = lane & 7, st.bl = lane >> 3, st.nb = nb, st.vec_ok = (L.in & 3) == 0;
-    st.row4 = (size_t)4 * L.in;
-    const VT* x_lane = x + (size_t)(b0 + st.bl) * L.in + 4 * st.cl;
+    st.in = L.in, st.cl = lane & 7, st.uq = lane >> 3, st.nb = nb, st.vec_ok = (L.in & 3) == 0;
+    const VT* x_tile = x + (size_t)b0 * L.in;
 
-    // Slab 0: everybody stages, several requests in flight per thread.
+    // Slab 0: everybody stages, kStageUnroll blocks (4 loads each) in flight per thread.
     {
-        st.x = x_lane, st.ncol = min(L.cs, L.in);
-        const int n_items = ((st.ncol + 31) >> 5) * (BT / 4);
-        for (int w0 = warp; w0 < n_items; w0 += nwarps * kStageUnroll) {
-            VT v[kStageUnroll][4];
+        st.x = x_tile, st.ncol = min(L.cs, L.in);
+        const int n_blocks = ((st.ncol + 31) >> 5) * (BT / 16);
+        for (int w0 = warp; w0 < n_blocks; w0 += nwarps * kStageUnroll) {
+            typename Stager<VT, BT>::Block blk[kStageUnroll];
 #pragma unroll
-            for (int u = 0; u < kStageUnroll; ++u) st.load(w0 + u * nwarps, n_items, v[u]);
+            for (int u = 0; u < kStageUnroll; ++u) st.load(w0 + u * nwarps, n_blocks, blk[u]);
 #pragma unroll
             for (int u = 0; u < kStageUnroll; ++u)
-                if (w0 + u * nwarps < n_items) st.store(w0 + u * nwarps, 0u, v[u]);
+                if (w0 + u * nwarps < n_blocks) st.store(w0 + u * nwarps, 0u, blk[u]);
         }
     }
     __syncthreads();
@@ -464,16 +480,15 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
         const uint32_t xs_off = (s & 1) ? lay.xs_bytes : 0u, xs_next = (s & 1) ? 0u : lay.xs_bytes;
         const int c0n = (s + 1) * L.cs;
         st.ncol = s + 1 < S ? min(L.cs, L.in - c0n) : 0;
-        st.x = x_lane + c0n;
-        const int n_items = ((st.ncol + 31) >> 5) * (BT / 4);  // warp items of the next slab
+        st.x = x_tile + c0n;
+        const int n_blocks = ((st.ncol + 31) >> 5) * (BT / 16);  // warp blocks of the next slab
 #pragma unroll
         for (int j = 0; j < RPH; ++j) {
             __syncwarp();  // every lane is done reading the stage the next prefetch overwrites
             const int jn = j + 1 < RPH ? j + 1 : 0, sn = j + 1 < RPH ? s : s + 1;
             if (sn < S) prefetch(sn, jn, (n + 1) & 1);
-            VT xv[kStagePerItem][4];
-#pragma unroll
-            for (int u = 0; u < kStagePerItem; ++u) st.load(warp + (j * kStagePerItem + u) * nwarps, n_items, xv[u]);
+            typename Stager<VT, BT>::Block xv;  // this item's share of the next slab
+            st.load(warp + j * nwarps, n_blocks, xv);
             if (sn < S) cp_async_wait<1>();
             else cp_async_wait<0>();
             __syncwarp();  // the other lanes' copies of this item are visible too
@@ -491,37 +506,38 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
                     fma4<VT>(acc[j], xs_off + ((uint32_t)c.w ^ lane_key), w.w);
                 }
             }
-#pragma unroll
-            for (int u = 0; u < kStagePerItem; ++u) {
-                const int wi = warp + (j * kStagePerItem + u) * nwarps;
-                if (wi < n_items) st.store(wi, xs_next, xv[u]);
-            }
+            if (warp + j * nwarps < n_blocks) st.store(warp + j * nwarps, xs_next, xv);
             ++n;
         }
         // Whatever of the next slab the row items did not cover.
-        for (int w0 = warp + RPH * kStagePerItem * nwarps; w0 < n_items; w0 += nwarps * kStagePerItem) {
-            VT xv[kStagePerItem][4];
+        for (int w0 = warp + RPH * nwarps; w0 < n_blocks; w0 += nwarps * kStageUnroll) {
+            typename Stager<VT, BT>::Block blk[kStageUnroll];
 #pragma unroll
-            for (int u = 0; u < kStagePerItem; ++u) st.load(w0 + u * nwarps, n_items, xv[u]);
+            for (int u = 0; u < kStageUnroll; ++u) st.load(w0 + u * nwarps, n_blocks, blk[u]);
 #pragma unroll
-            for (int u = 0; u < kStagePerItem; ++u)
-                if (w0 + u * nwarps < n_items) st.store(w0 + u * nwarps, xs_next, xv[u]);
+            for (int u = 0; u < kStageUnroll; ++u)
+                if (w0 + u * nwarps < n_blocks) st.store(w0 + u * nwarps, xs_next, blk[u]);
         }
         __syncthreads();  // next slab is complete, and nobody reads this slab's buffer any more
     }
 
-    // Epilogue: sums -> ys[b][row] in shared memory, then runs of consecutive output rows per batch row.
+    // Epilogue: bias + activation, then through shared memory (ys[b][row]) so that y is written in runs of
+    // consecutive output rows per batch row.
     float* ys = reinterpret_cast<float*>(smem_at(0));
     const int pitch = rt | 1;
+    float bias_r[RPH];
+#pragma unroll
+    for (int j = 0; j < RPH; ++j) bias_r[j] = bias_s[g + j * ngroups];
+    __syncthreads();  // bias_s is read; the y tile may now overwrite any part of shared memory
 #pragma unroll
     for (int j = 0; j < RPH; ++j)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) ys[(4 * ll + e) * pitch + g + j * ngroups] = acc[j][e];
+        for (int e = 0; e < 4; ++e) ys[(4 * ll + e) * pitch + g + j * ngroups] = activate(acc[j][e] + bias_r[j], L.act);
     __syncthreads();
-    for (int e = tid; e < nb * nrows; e += nthr) {
-        const int b = e / nrows, i = e - b * nrows;
-        const float v = ys[b * pitch + i] + L.bias[o0 + i];
-        from_f32(&y[(size_t)(b0 + b) * L.out + o0 + i], activate(v, L.act));
+    const int per_b = nrows;
+    for (int b = warp; b < nb; b += nwarps) {
+        VT* yrow = y + (size_t)(b0 + b) * L.out + o0;
+        for (int i = lane; i < per_b; i += 32) from_f32(&yrow[i], ys[b * pitch + i]);
     }
 }
 
@@ -873,7 +889,13 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
         const Quad* quads_dev = nullptr;
         if (st == CFI_OK) st = upload(l, quads, &quads_dev);
         d.wq_b = quads_dev;
-        if (st == CFI_OK) st = upload(l, seg, &d.seg);
+        // The kernel looks the quad offsets up by output row: ablated rows get an all-zero line.
+        std::vector<int32_t> seg_o((size_t)out_features * (d.n_slabs + 1), 0);
+        for (int32_t o = 0; o < out_features; ++o)
+            if (slot[o] >= 0)
+                std::copy(seg.begin() + (size_t)slot[o] * (d.n_slabs + 1), seg.begin() + (size_t)(slot[o] + 1) * (d.n_slabs + 1),
+                          seg_o.begin() + (size_t)o * (d.n_slabs + 1));
+        if (st == CFI_OK) st = upload(l, seg_o, &d.seg);
 
         std::vector<float> bias_h((size_t)out_features, 0.0f);
         if (bias) std::copy(bias, bias + out_features, bias_h.begin());
