@@ -185,6 +185,34 @@ cfi_status_t cfi_stack_forward(const cfi_stack_t* stack, const void* x, void* y,
 cfi_status_t cfi_stack_destroy(cfi_stack_t* stack);
 
 /*
+ * cfi_stack_forward_static — the chain of cfi_stack_forward for callers that must not allocate device
+ * memory: code running where cudaMalloc is off limits (a real-time or latency-critical serving loop that
+ * may not take the allocator's locks or implicit synchronisation, a process working under a fixed memory
+ * budget handed out at start-up, a plug-in whose host forbids allocations after initialisation).  The paper
+ * has no counterpart of this entry point; it exists for deployment only.
+ *
+ * Nothing is created or destroyed: the layers are passed directly, and the intermediate activations live
+ * in one fixed 8 MiB device array that is part of the library image (every GPU that loads the library
+ * holds these 8 MiB until the process exits).  The array is split into two 4 MiB halves used alternately,
+ * so the call requires
+ *
+ *     batch * max_i(out_features of layer i, i < n_layers - 1) * sizeof(dtype)  <=  4 MiB
+ *
+ * and returns CFI_ERR_BUFFER_TOO_SMALL otherwise (a single layer needs no intermediate and always fits).
+ * Arguments and checks are those of cfi_stack_create + cfi_stack_forward: layers must chain and share
+ * dtype and device; x and y are caller-owned device buffers, 16-byte aligned.  The work is enqueued on
+ * `stream` without synchronising.  No cudaMalloc / cudaFree and no allocating library call is made.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that first
+ * call outside any stream capture.  All calls in the process share the one array: two calls whose kernels
+ * can overlap on the GPU (different streams) race on it and must be ordered by the caller.  The array keeps
+ * whatever the last call left; nothing needs clearing, because every layer overwrites all batch * out
+ * values it hands to the next.
+ */
+cfi_status_t cfi_stack_forward_static(cfi_layer_t* const* layers, int32_t n_layers, const void* x, void* y,
+                                      int32_t batch, cfi_stream_t stream);
+
+/*
  * cfi_probe_device — measures, on the current device, the ceilings the forward kernels are judged against
  * and that no vendor figure states: fp32 FMA rate (register-only chains on every SM), shared-memory load
  * bandwidth (conflict-free 16-byte loads), L2 read bandwidth (every SM streaming a resident 16 MB buffer,

@@ -26,7 +26,8 @@ _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, 0: 0, 1: 1, 2: 2, 
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_device_status", "cfi_destroy",
-           "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_probe_device")
+           "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static",
+           "cfi_probe_device")
 
 
 class CfiError(RuntimeError):
@@ -79,6 +80,7 @@ def _load() -> ctypes.CDLL:
     lib.cfi_stack_create.argtypes = [ctypes.POINTER(vp), ci, ci, ctypes.POINTER(vp)]
     lib.cfi_stack_forward.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_stack_destroy.argtypes = [vp]
+    lib.cfi_stack_forward_static.argtypes = [ctypes.POINTER(vp), ci, vp, vp, ci, vp]
     lib.cfi_probe_device.argtypes = [ctypes.POINTER(DeviceProbe)]
     for name in EXPORTS:
         if name != "cfi_status_string":
@@ -250,6 +252,17 @@ def cfi_stack_forward(stack: Stack, x, y, batch: int, stream=None) -> None:
 
 def cfi_stack_destroy(stack: Stack) -> None:
     stack.close()
+
+
+def cfi_stack_forward_static(layers: Sequence[Layer], x, y, batch: int, stream=None) -> None:
+    """Chain of layers with the intermediates in the library's fixed 8 MiB device array: no allocation.
+
+    For callers that may not call cudaMalloc (see include/cfi.h).  batch * widest intermediate * element size
+    must not exceed 4 MiB; calls that can overlap on the GPU race on the shared array.
+    """
+    arr = (ctypes.c_void_p * len(layers))(*[l.handle for l in layers])
+    _check(_lib.cfi_stack_forward_static(arr, len(layers), _dev_ptr(x), _dev_ptr(y), batch, _stream_handle(stream)),
+           "cfi_stack_forward_static")
 
 
 def cfi_probe_device() -> DeviceProbe:

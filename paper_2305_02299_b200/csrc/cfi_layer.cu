@@ -1070,3 +1070,58 @@ extern "C" cfi_status_t cfi_stack_destroy(cfi_stack_t* stack) {
     delete stack;
     return CFI_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Chain of layers without any allocation: the intermediates live in a fixed device array.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticScratchBytes = (size_t)8 << 20;  // two halves of 4 MiB, used alternately
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch per device.  In host code the array's name only stands for the symbol;
+// the address a kernel can use has to be asked for, with the owning device current.
+std::atomic<unsigned char*> g_static_scratch_addr[kMaxDevices];
+
+cfi_status_t static_scratch(int device, unsigned char** base) {
+    if (device < 0 || device >= kMaxDevices) return CFI_ERR_SHAPE;
+    unsigned char* p = g_static_scratch_addr[device].load(std::memory_order_acquire);
+    if (!p) {
+        void* sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, g_static_scratch) != cudaSuccess || !sym) {
+            cudaGetLastError();
+            return CFI_ERR_CUDA;
+        }
+        p = static_cast<unsigned char*>(sym);
+        g_static_scratch_addr[device].store(p, std::memory_order_release);
+    }
+    *base = p;
+    return CFI_OK;
+}
+
+}  // namespace
+
+extern "C" cfi_status_t cfi_stack_forward_static(cfi_layer_t* const* layers, int32_t n_layers, const void* x, void* y,
+                                                 int32_t batch, cfi_stream_t stream) {
+    if (!layers) return CFI_ERR_NULL;
+    if (n_layers < 1 || batch < 0) return CFI_ERR_SHAPE;
+    size_t widest = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        if (!layers[i]) return CFI_ERR_NULL;
+        if (layers[i]->dtype != layers[0]->dtype || layers[i]->device != layers[0]->device) return CFI_ERR_DTYPE;
+        if (i && layers[i]->d.in != layers[i - 1]->d.out) return CFI_ERR_SHAPE;
+        if (i + 1 < n_layers) widest = std::max(widest, (size_t)layers[i]->d.out);
+    }
+    const size_t es = layers[0]->dtype == CFI_BF16 ? 2 : 4;
+    if ((size_t)batch * widest * es > kStaticScratchBytes / 2) return CFI_ERR_BUFFER_TOO_SMALL;
+    DeviceGuard g(layers[0]->device);
+    unsigned char* base = nullptr;
+    if (cfi_status_t e = static_scratch(layers[0]->device, &base)) return e;
+    const void* cur = x;
+    for (int i = 0; i < n_layers; ++i) {
+        void* dst = i + 1 == n_layers ? y : base + (size_t)(i & 1) * (kStaticScratchBytes / 2);
+        if (cfi_status_t e = cfi_forward(layers[i], cur, dst, batch, stream)) return e;
+        cur = dst;
+    }
+    return CFI_OK;
+}
