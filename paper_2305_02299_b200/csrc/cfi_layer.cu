@@ -95,7 +95,10 @@ __global__ void cfi_simple_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
         const VT* w = reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp;
         const int32_t* ix = L.indices + (size_t)r * L.kp;
         const VT* xr = x + (size_t)b * L.in;
-        for (int j = 0; j < L.k; ++j) s = fmaf(to_f32(w[j]), to_f32(xr[ix[j]]), s);
+        for (int j = 0; j < L.kp; ++j) {  // pad entries (column == in) may sit anywhere in the row
+            const int c = ix[j];
+            if (c < L.in) s = fmaf(to_f32(w[j]), to_f32(xr[c]), s);
+        }
     }
     from_f32(&y[t], activate(s + L.bias[o], L.act));
 }
@@ -171,19 +174,42 @@ __device__ __forceinline__ void gather_fma(float (&acc)[BT], const float* xs, in
     }
 }
 
-constexpr int kSplitkUnroll = 4;  // 16-byte vector pairs in flight per lane
+// Programmatic dependent launch.  Every forward kernel lets its successor in the stream start early
+// (pdl_launch_dependents at its top) and itself touches x and y only after pdl_wait, which returns once the
+// predecessor has completed and its writes are visible.  What a kernel does before pdl_wait (reading the
+// layer's weights, indices and tables, which no kernel writes) therefore overlaps the predecessor's tail.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-template <typename VT, int BT, int G>
+// U = 16-byte vector pairs (weights + indices) in flight per lane: 4, or 8 for long rows so that a whole
+// row is requested at once.
+template <typename VT, int BT, int G, int U>
 __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch,
                                   int rows_per_group) {
     extern __shared__ __align__(16) float xs_f32[];  // [(in + 1)][BT]
     float* xs = xs_f32;
     using CK = Chunk<VT>;
-    constexpr int U = kSplitkUnroll;
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int b0 = blockIdx.y * BT;
     const int nb = min(BT, batch - b0);
+    const int groups = nthr / G, g = tid / G, lg = tid % G;
+    const int nvec = L.kp / CK::VEC;
+    const bool dense_rows = L.n_active == L.out;  // no ablated row: output row o is condensed row o
+    int o = blockIdx.x * (groups * rows_per_group) + g;
+    int r = o < L.out ? (dense_rows ? o : L.slot[o]) : -1;
 
+    // The first vectors of the first row depend neither on x nor on the kernel before this one: they are
+    // requested first, so the weight stream is in flight while x is awaited and staged.
+    CK ck[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int v = lg + u * G;
+        ck[u].load(L.values, L.indices, (size_t)max(r, 0) * L.kp, v, r >= 0 && v < nvec, L.in);
+    }
+    float bias = o < L.out ? L.bias[o] : 0.0f;
+
+    pdl_wait();
     // Stage the CTA's x rows, widened to fp32, transposed to [column][b].
     if (BT == 1 && sizeof(VT) == 4 && (L.in & 3) == 0) {
         const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(x) + (size_t)b0 * L.in);
@@ -200,20 +226,6 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
         }
     }
     if (tid < BT) xs[(size_t)L.in * BT + tid] = 0.0f;
-
-    const int groups = nthr / G, g = tid / G, lg = tid % G;
-    const int nvec = L.kp / CK::VEC;
-    int o = blockIdx.x * (groups * rows_per_group) + g;
-    int r = o < L.out ? L.slot[o] : -1;
-
-    // The first vectors of the first row do not depend on x: issue them before the barrier so the
-    // weight stream and the x staging are in flight together.
-    CK ck[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-        const int v = lg + u * G;
-        ck[u].load(L.values, L.indices, (size_t)max(r, 0) * L.kp, v, r >= 0 && v < nvec, L.in);
-    }
     __syncthreads();
 
     for (int i = 0;;) {
@@ -236,6 +248,20 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
                 }
             }
         }
+        const int o_done = o;
+        const float bias_done = bias;
+        // The next row's first vectors and bias are requested before this row's reduction and store.
+        const bool more = ++i < rows_per_group;
+        if (more) {
+            o += groups;
+            r = o < L.out ? (dense_rows ? o : L.slot[o]) : -1;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int v = lg + u * G;
+                ck[u].load(L.values, L.indices, (size_t)max(r, 0) * L.kp, v, r >= 0 && v < nvec, L.in);
+            }
+            bias = o < L.out ? L.bias[o] : 0.0f;
+        }
         // Finish the k-sum across the G lanes of the group.
 #pragma unroll
         for (int b = 0; b < BT; ++b) {
@@ -244,20 +270,12 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
             for (int m = G >> 1; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
             acc[b] = v;
         }
-        if (lg == 0 && o < L.out) {
-            const float bias = L.bias[o];
+        if (lg == 0 && o_done < L.out) {
 #pragma unroll
             for (int b = 0; b < BT; ++b)
-                if (b < nb) from_f32(&y[(size_t)(b0 + b) * L.out + o], activate(acc[b] + bias, L.act));
+                if (b < nb) from_f32(&y[(size_t)(b0 + b) * L.out + o_done], activate(acc[b] + bias_done, L.act));
         }
-        if (++i >= rows_per_group) break;
-        o += groups;
-        r = o < L.out ? L.slot[o] : -1;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int v = lg + u * G;
-            ck[u].load(L.values, L.indices, (size_t)max(r, 0) * L.kp, v, r >= 0 && v < nvec, L.in);
-        }
+        if (!more) break;
     }
 }
 
@@ -544,24 +562,33 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 // ------------------------------------------------------------------------------------------------
 // host: launch shapes
 // ------------------------------------------------------------------------------------------------
-struct SplitkShape { int bt, g, threads, rows_per_group, grid_x, grid_y; size_t smem; };
+struct SplitkShape { int bt, g, u, threads, rows_per_group, grid_x, grid_y; size_t smem; };
 struct BatchShape { int warps, rph, threads, rt, grid_x, grid_y; size_t smem; bool ok; };
 
 int vec_of(int dtype) { return dtype == CFI_BF16 ? 8 : 4; }
+
+// Lanes that share a row in the split-k kernel: the smallest power of two for which 4 vectors per lane cover
+// the row, at most a warp.  The small-batch layout orders a row's entries for this number (order_for_banks).
+int splitk_lanes_per_row(int nvec) {
+    int g = 4;
+    while (g < 32 && g * 4 < nvec) g <<= 1;
+    return g;
+}
 
 SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     SplitkShape s{};
     s.bt = batch >= 8 ? 8 : batch >= 3 ? 4 : batch == 2 ? 2 : 1;
     while (s.bt > 1 && (size_t)(l->d.in + 1) * s.bt * 4 > (size_t)l->smem_optin) s.bt >>= 1;
     const int nvec = l->d.kp / vec_of(l->dtype);
-    s.g = 4;
-    while (s.g < 32 && s.g * kSplitkUnroll < nvec) s.g <<= 1;
-    // Enough CTAs to cover the SMs a few times over, but no more x staging than needed.
+    s.g = splitk_lanes_per_row(nvec);
+    s.u = nvec > s.g * 4 ? 8 : 4;  // long rows: request the whole row (up to 8 vectors per lane) at once
+    // Enough CTAs to cover the SMs several times over (each CTA stages x for itself, and many small CTAs
+    // keep more independent requests in flight), but not more x staging than that needs.
     const int64_t lanes = (int64_t)l->d.out * s.g;
-    s.threads = lanes >= (int64_t)l->sm_count * 4 * 256 ? 256 : 128;
+    s.threads = lanes >= (int64_t)l->sm_count * 8 * 256 ? 256 : 128;
     const int groups = s.threads / s.g;
     const int ctas_one_row_each = (l->d.out + groups - 1) / groups;
-    const int target = l->sm_count * 4;
+    const int target = l->sm_count * 8;
     s.rows_per_group = std::max(1, (ctas_one_row_each + target - 1) / target);
     s.grid_x = (l->d.out + groups * s.rows_per_group - 1) / (groups * s.rows_per_group);
     s.grid_y = (batch + s.bt - 1) / s.bt;
@@ -624,12 +651,38 @@ cfi_status_t set_smem(size_t bytes, int device) {
     return CFI_OK;
 }
 
+// Launch with programmatic stream serialisation allowed: the kernel may start before its predecessor in the
+// stream has finished (see pdl_wait in the kernels).
+template <typename... KArgs, typename... Args>
+cfi_status_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
+    return CFI_OK;
+}
+
 template <typename VT, int BT, int G>
 cfi_status_t launch_splitk_g(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
                              cudaStream_t st) {
-    if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, BT, G>>(s.smem, l->device)) return e;
-    cfi_splitk_kernel<VT, BT, G><<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, x, y, batch, s.rows_per_group);
-    return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+    if (s.u == 8) {
+        if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, BT, G, 8>>(s.smem, l->device)) return e;
+        return launch_pdl(cfi_splitk_kernel<VT, BT, G, 8>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch,
+                          s.rows_per_group);
+    }
+    if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, BT, G, 4>>(s.smem, l->device)) return e;
+    return launch_pdl(cfi_splitk_kernel<VT, BT, G, 4>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch,
+                      s.rows_per_group);
 }
 
 template <typename VT, int BT>
@@ -749,6 +802,40 @@ cfi_status_t upload(cfi_layer* l, const std::vector<T>& host, const T** dev) {
     return CFI_OK;
 }
 
+// Order of a row's entries in the small-batch layout.  The `lanes` lanes that share a row read vector
+// v = lane + lanes * t of the row and gather its element e in the same instruction, so the entries at
+// positions vec * (lane + lanes * t) + e, lane = 0..lanes-1, hit shared memory together.  Entries are dealt
+// to these sets so that a set's columns fall into different banks (column mod 32 for one batch row) as far
+// as the row allows, lanes ascending with the bank so that aligned sub-groups differ in the low bits too.
+// cols: the row's k columns; place[j] receives the position (< kp) of entry j; pad positions stay free.
+void order_for_banks(const int32_t* cols, int k, int kp, int vec, int lanes, int32_t* place) {
+    std::vector<int32_t> by_bank[32];
+    for (int j = 0; j < k; ++j) by_bank[cols[j] & 31].push_back(j);
+    const int nvec = kp / vec;
+    int left = k;
+    int order[32], chosen[32];
+    for (int t = 0; t * lanes < nvec && left > 0; ++t) {
+        const int width = std::min(lanes, nvec - t * lanes);  // lanes that have a vector in this round
+        for (int e = 0; e < vec && left > 0; ++e) {
+            // Fullest banks first; one entry per bank while enough banks are non-empty.
+            std::iota(order, order + 32, 0);
+            std::stable_sort(order, order + 32, [&](int a, int b) { return by_bank[a].size() > by_bank[b].size(); });
+            const int quota = std::min(width, left);  // sets are filled in order; pads collect at the row's end
+            int n_chosen = 0;
+            for (int pass = 0; n_chosen < quota; ++pass)
+                for (int q = 0; q < 32 && n_chosen < quota; ++q)
+                    if ((int)by_bank[order[q]].size() > pass) chosen[n_chosen++] = order[q];
+            std::sort(chosen, chosen + n_chosen);
+            for (int i = 0; i < n_chosen; ++i) {
+                const int j = by_bank[chosen[i]].back();
+                by_bank[chosen[i]].pop_back();
+                place[j] = vec * (i + lanes * t) + e;
+                --left;
+            }
+        }
+    }
+}
+
 void free_layer(cfi_layer* l) {
     for (void* p : l->allocs) cudaFree(p);
     if (l->stage_x) cudaFree(l->stage_x);
@@ -818,25 +905,31 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
         // ---- small-batch layout
         const int vec = vec_of(dtype);
         d.kp = ((k + vec - 1) / vec) * vec;
+        std::vector<int32_t> place((size_t)std::max(d.kp, 1));  // position in the padded row of sorted entry j
+        const int lanes = splitk_lanes_per_row(std::max(1, d.kp / vec));
         std::vector<int32_t> idx_p((size_t)n_active * d.kp, in_features);
         cfi_status_t st = CFI_OK;
         if (dtype == CFI_F32) {
             std::vector<float> val_p((size_t)n_active * d.kp, 0.0f);
-            for (int32_t r = 0; r < n_active; ++r)
+            for (int32_t r = 0; r < n_active; ++r) {
+                order_for_banks(&c_sorted[(size_t)r * k], k, d.kp, vec, lanes, place.data());
                 for (int32_t j = 0; j < k; ++j) {
-                    val_p[(size_t)r * d.kp + j] = v_sorted[(size_t)r * k + j];
-                    idx_p[(size_t)r * d.kp + j] = c_sorted[(size_t)r * k + j];
+                    val_p[(size_t)r * d.kp + place[j]] = v_sorted[(size_t)r * k + j];
+                    idx_p[(size_t)r * d.kp + place[j]] = c_sorted[(size_t)r * k + j];
                 }
+            }
             const float* p = nullptr;
             st = upload(l, val_p, &p);
             d.values = p;
         } else {
             std::vector<uint16_t> val_p((size_t)n_active * d.kp, (uint16_t)0);
-            for (int32_t r = 0; r < n_active; ++r)
+            for (int32_t r = 0; r < n_active; ++r) {
+                order_for_banks(&c_sorted[(size_t)r * k], k, d.kp, vec, lanes, place.data());
                 for (int32_t j = 0; j < k; ++j) {
-                    val_p[(size_t)r * d.kp + j] = bf16_bits_rne(v_sorted[(size_t)r * k + j]);
-                    idx_p[(size_t)r * d.kp + j] = c_sorted[(size_t)r * k + j];
+                    val_p[(size_t)r * d.kp + place[j]] = bf16_bits_rne(v_sorted[(size_t)r * k + j]);
+                    idx_p[(size_t)r * d.kp + place[j]] = c_sorted[(size_t)r * k + j];
                 }
+            }
             const uint16_t* p = nullptr;
             st = upload(l, val_p, &p);
             d.values = p;
