@@ -426,6 +426,7 @@ template <typename VT, int BT, int RPH>
 __global__ void __launch_bounds__(512, 1)
 cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch) {
     constexpr int LPR = BT / 4, RPW = 32 / LPR;  // lanes per row group, row groups per warp
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31;
     const int nwarps = nthr >> 5, ngroups = nwarps * RPW, rt = ngroups * RPH, S = L.n_slabs;
     const BatchSmem lay = batch_smem_layout(L.cs, S, L.maxq, (int)sizeof(VT), BT, rt, nwarps);
@@ -450,7 +451,9 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
     st.in = L.in, st.cl = lane & 7, st.uq = lane >> 3, st.nb = nb, st.vec_ok = (L.in & 3) == 0;
     const VT* x_tile = x + (size_t)b0 * L.in;
 
-    // Slab 0: everybody stages, kStageUnroll blocks (4 loads each) in flight per thread.
+    // Slab 0: everybody stages, kStageUnroll blocks (4 loads each) in flight per thread.  x (and later y) may
+    // belong to the kernel before this one, so this is where its completion is awaited.
+    pdl_wait();
     {
         st.x = x_tile, st.ncol = min(L.cs, L.in);
         const int n_blocks = ((st.ncol + 31) >> 5) * (BT / 16);
@@ -715,8 +718,7 @@ cfi_status_t launch_splitk(const cfi_layer* l, const SplitkShape& s, const void*
 template <typename VT, int RPH>
 cfi_status_t launch_batch_rph(const cfi_layer* l, const BatchShape& s, const VT* x, VT* y, int batch, cudaStream_t st) {
     if (cfi_status_t e = set_smem<cfi_batch_kernel<VT, kBatchTile, RPH>>(s.smem, l->device)) return e;
-    cfi_batch_kernel<VT, kBatchTile, RPH><<<dim3(s.grid_x, s.grid_y), s.threads, s.smem, st>>>(l->d, x, y, batch);
-    return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
+    return launch_pdl(cfi_batch_kernel<VT, kBatchTile, RPH>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch);
 }
 
 template <typename VT>
