@@ -386,10 +386,66 @@ def main():
         line["cpu_baseline"] = {"value": cb["flops"] / cb["median_s"] / 1e9, "unit": "GFLOP/s", "cores": cb["cores"],
                                 "kind": "oracle", "us_per_call": cb["median_s"] * 1e6,
                                 "sample": f"whole workload ({cb['rows']} batch rows), median of {cb['calls']} calls"}
+        line["context"] = context_leg(w, torch)
+        line["stack_c5"] = stack_leg(cfi, torch, peaks, sm_count)
     if rank == 0:
         print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
+
+
+def _time_torch(fn, torch, iters=200):
+    for _ in range(10):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(iters):
+        fn()
+    b.record()
+    b.synchronize()
+    return a.elapsed_time(b) * 1e-3 / iters
+
+
+def context_leg(w, torch):
+    """Library routines on the same masked weights, as context (not a target): cuBLAS dense through
+    torch.matmul on the full masked weight, cuSPARSE CSR through torch's sparse matmul.  Warm (one layer),
+    eager launches, batch of the headline workload and batch 1."""
+    L = w.layer(seed=0)
+    wd = torch.from_numpy(L.w_dense * L.mask).cuda()
+    csr = wd.to_sparse_csr()
+    out = {}
+    for batch in (w.batch, 1):
+        x = torch.from_numpy(w.x(seed=0, batch=batch)).cuda()
+        xt = x.t().contiguous()
+        out[f"b{batch}"] = {"cublas_dense_us": _time_torch(lambda: torch.matmul(x, wd.t()), torch) * 1e6,
+                            "cusparse_csr_us": _time_torch(lambda: torch.matmul(csr, xt), torch) * 1e6}
+    out["note"] = "torch.matmul (cuBLAS fp32, TF32 off) and torch CSR matmul (cuSPARSE), warm, eager; paper: 1.7x / 13.0x " \
+                  "faster than dense / CSR at batch 256 on a Titan V, 3.4x / 2.5x on a Xeon W-2145 at batch 1"
+    return out
+
+
+def stack_leg(cfi, torch, peaks, sm_count):
+    """The bf16 MLP stack (12 blocks of 768 -> 3072 GELU -> 768, 5 % of rows ablated, 50,432 rows)."""
+    s = inputs.StackWorkload()
+    layers, flops, bytes_ = [], 0, 0
+    for L, sp in zip(s.layers(seed=0), s.layer_specs()):
+        v, ix, rows = cfi.cfi_pack(L.w_dense, L.mask)
+        layers.append(cfi.cfi_create(v, ix, rows, L.bias, sp[0], sp[1], dtype="bf16", act=sp[4]))
+        flops += 2 * s.batch * rows.shape[0] * sp[2]
+        bytes_ += rows.shape[0] * sp[2] * 6 + s.batch * (sp[0] + sp[1]) * 2 + sp[1] * 4
+    stack = cfi.cfi_stack_create(layers, s.batch)
+    x = torch.from_numpy(s.x(seed=0)).to("cuda", torch.bfloat16)
+    y = torch.empty((s.batch, s.d_model), device="cuda", dtype=torch.bfloat16)
+    sec = _time_torch(lambda: cfi.cfi_stack_forward(stack, x, y, s.batch), torch, iters=5)
+    stack.close()
+    for l in layers:
+        l.close()
+    fma_peak = sm_count * FMA_LANES_PER_SM * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+    return {"ms_per_pass": sec * 1e3, "layers": len(layers), "rows": s.batch, "dtype": "bf16",
+            "effective_tflops": flops / sec / 1e12, "fma_frac": flops / sec / 1e12 / fma_peak,
+            "algorithmic_bytes": bytes_, "hbm_frac": bytes_ / sec / 1e9 / peaks["hbm_gbs"],
+            "l2": "activations of one layer (388 MB) exceed L2"}
 
 
 def batch1_leg(W, cfi, torch, l2, peaks, peak_kind):
