@@ -355,7 +355,7 @@ def main():
         achieved_tflops = flops / per_call / 1e12
         hbm_gbs = rep.bytes_per_step / per_call / 1e9
         info = cfi.cfi_layer_info(rep.layers[0])
-        chosen = {1: "simple", 2: "splitk", 3: "batch"}[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
+        chosen = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
         line = {
             "metric": METRIC, "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": per_call * 1e3, "us_per_call": per_call * 1e6,

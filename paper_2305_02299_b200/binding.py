@@ -19,10 +19,10 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 ACT_NONE, ACT_GELU = 0, 1
-VARIANT_AUTO, VARIANT_SIMPLE, VARIANT_SPLITK, VARIANT_BATCH = 0, 1, 2, 3
+VARIANT_AUTO, VARIANT_SIMPLE, VARIANT_SPLITK, VARIANT_BATCH, VARIANT_DENSE_TC = 0, 1, 2, 3, 4
 _DTYPES = {"f32": F32, "fp32": F32, "float32": F32, "bf16": BF16, "bfloat16": BF16, F32: F32, BF16: BF16}
 _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE, ACT_GELU: ACT_GELU}
-_VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, 0: 0, 1: 1, 2: 2, 3: 3}
+_VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_device_status", "cfi_destroy",

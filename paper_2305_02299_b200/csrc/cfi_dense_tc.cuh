@@ -1,0 +1,218 @@
+// CFI_VARIANT_DENSE_TC: large batch, bf16 storage, on the tensor cores.
+//
+// Included by cfi_layer.cu inside its unnamed namespace (it uses DevLayer, activate, smem_at and the
+// pdl_* helpers defined there).
+//
+// The paper notes that a layer trained with SRigL can be run either from the condensed arrays or as a
+// dense layer over the kept neurons, with the same weights (Sec. 4.4, last paragraph), and that the dense
+// form wins at larger batch.  On B200 this is where that happens: the gather formulation is held to
+// about a fifth of the fp32 FMA rate by shared-memory bandwidth, while a dense bf16 contraction on the
+// 5th-generation tensor cores is more than twenty times faster than the FMA pipes, so at 90 % sparsity
+// ten times the flops still finish several times sooner.  The layer keeps a dense bf16 copy of its
+// weight, Wd[out_pad][in] (zero rows for ablated and padding rows), and the forward is
+//
+//     y[b, o] = act( bias[o] + sum_c x[b, c] * Wd[o, c] )          fp32 accumulation of exact products,
+//
+// i.e. the same numbers as the condensed forms up to the order of the additions.
+//
+// One CTA computes a 128 (batch) x 128 (output rows) tile:
+//   warp 0, one lane   TMA producer: per 64-column block of x and Wd one 128 x 64 bf16 box each
+//                      (cp.async.bulk.tensor, 128-byte swizzle) into a 3-stage ring, completion on mbarriers;
+//   warp 1, one lane   issues tcgen05.mma (cta_group::1, kind::f16, M = N = 128, K = 16 per instruction,
+//                      both operands K-major from shared memory), accumulator in 128 columns of tensor
+//                      memory; tcgen05.commit hands ring slots back and finally signals the epilogue;
+//   warps 2..5         epilogue: tcgen05.ld the accumulator (one batch row per thread), add bias, apply the
+//                      activation, round to bf16, pass through shared memory (the drained ring) and write
+//                      y in 256-byte runs per batch row.
+// Two CTAs fit an SM (97 KB of shared memory, 128 of 512 tensor-memory columns each), so one CTA's
+// epilogue overlaps the other's main loop.
+//
+// Every mbarrier wait is bounded.  If one expires the thread records code 2 in the layer's status word and
+// leaves its role's loop; all roles still meet at the final barrier, tensor memory is freed and the kernel
+// returns.
+
+#include <cuda.h>  // CUtensorMap and the enums of cuTensorMapEncodeTiled (types only; the entry point is looked up at run time)
+
+constexpr int kTcM = 128, kTcN = 128, kTcK = 64, kTcStages = 3, kTcThreads = 192;
+constexpr uint32_t kTcStageBytes = (kTcM + kTcN) * kTcK * 2;  // 32 KB
+constexpr uint32_t kTcSpinLimit = 1u << 22;
+constexpr size_t kTcSmemBytes = 1024 + kTcStages * kTcStageBytes + 1024;
+
+__device__ __forceinline__ uint32_t smem_u32(uint32_t off) { return (uint32_t)__cvta_generic_to_shared(smem_at(off)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
+// Returns false if the phase with this parity did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, uint32_t limit) {
+    for (uint32_t it = 0; it < limit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(mbar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t mbar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(mbar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile stored as rows of 128 bytes with the 128-byte
+// swizzle (what the TMA box above produces): groups of 8 rows are 1024 bytes apart (stride offset), the
+// leading offset is not used by swizzled K-major layouts, descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr_bytes & 0x3FFFFu) >> 4);  // start address, bits [0,14)
+    d |= (uint64_t)1 << 16;                               // leading byte offset (unused here), bits [16,30)
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                               // version, bits [46,48)
+    d |= (uint64_t)2 << 61;                               // 128-byte swizzle, bits [61,64)
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = 128, M = 128.
+constexpr uint32_t kTcInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcN >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(kTcInstrDesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t mbar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Shared memory (offsets from the first 1024-byte boundary): the ring, then barriers and small tables.
+//   ring      kTcStages x [A 128 x 64 bf16 | B 128 x 64 bf16]; after the main loop its first 32 KB hold the y tile
+//   +0        full[kTcStages], +32 empty[kTcStages], +64 accumulator barrier, +72 tensor-memory base address
+//   +128      bias of the tile's 128 output rows
+__global__ void __launch_bounds__(kTcThreads, 2)
+cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                    __nv_bfloat16* __restrict__ y, int batch) {
+    pdl_launch_dependents();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t base = ((smem_u32(0) + 1023u) & ~1023u) - smem_u32(0);  // offset of the first 1024-byte boundary
+    const uint32_t ring = base, ctl = base + kTcStages * kTcStageBytes;
+    const uint32_t full0 = smem_u32(ctl), empty0 = smem_u32(ctl + 32), accum = smem_u32(ctl + 64);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_at(ctl + 72));
+    float* bias_s = reinterpret_cast<float*>(smem_at(ctl + 128));
+    const int m0 = blockIdx.y * kTcM, n0 = blockIdx.x * kTcN;
+    const int k_blocks = (L.in + kTcK - 1) / kTcK;
+
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accum, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {  // one warp allocates the accumulator's 128 columns of tensor memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(ctl + 72)), "r"(128u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid >= 64) {
+        const int n = n0 + tid - 64;
+        bias_s[tid - 64] = n < L.out ? L.bias[n] : 0.0f;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // x and y may belong to the kernel before this one
+    bool ok = true;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % kTcStages;
+            if (kb >= kTcStages) ok = mbar_wait(empty0 + 8 * s, (uint32_t)(kb / kTcStages - 1) & 1u, kTcSpinLimit);
+            if (!ok) break;
+            const uint32_t a_dst = smem_u32(ring + s * kTcStageBytes), b_dst = a_dst + kTcM * kTcK * 2;
+            mbar_expect_tx(full0 + 8 * s, kTcStageBytes);
+            tma_load_2d(a_dst, &map_x, full0 + 8 * s, kb * kTcK, m0);
+            tma_load_2d(b_dst, &map_w, full0 + 8 * s, kb * kTcK, n0);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------------------------------------------------------- MMA issuer
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % kTcStages;
+            ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / kTcStages) & 1u, kTcSpinLimit);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = smem_u32(ring + s * kTcStageBytes), b_addr = a_addr + kTcM * kTcK * 2;
+            const uint64_t da = umma_desc_k_sw128(a_addr), db = umma_desc_k_sw128(b_addr);
+#pragma unroll
+            for (int k = 0; k < kTcK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzled row
+                umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), (kb | k) != 0 ? 1u : 0u);
+            umma_commit(empty0 + 8 * s);  // the slot is free once these MMAs have read it
+        }
+        if (ok) umma_commit(accum);  // the accumulator is complete once every MMA issued so far has finished
+    } else if (warp >= 2) {
+        // ---------------------------------------------------------------- epilogue
+        ok = mbar_wait(accum, 0u, kTcSpinLimit);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int q = warp & 3;           // a warp may read the tensor-memory lanes 32 q .. 32 q + 31
+        const int row = 32 * q + lane;    // batch row of the tile held by this thread
+        if (ok) {
+            // y tile in shared memory: 128 rows x 256 bytes, 16-byte chunks permuted by chunk ^ (row & 15).
+#pragma unroll 1
+            for (int c = 0; c < kTcN; c += 16) {
+                uint32_t v[16];
+                tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                uint32_t packed[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float lo = activate(__uint_as_float(v[2 * e]) + bias_s[c + 2 * e], L.act);
+                    const float hi = activate(__uint_as_float(v[2 * e + 1]) + bias_s[c + 2 * e + 1], L.act);
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+                    packed[e] = *reinterpret_cast<const uint32_t*>(&p);
+                }
+                const int ch = c >> 3;  // 16-byte chunk index of columns c .. c+7; the next one holds c+8 .. c+15
+                *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + (((ch) ^ (row & 15)) << 4))) =
+                    make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + (((ch + 1) ^ (row & 15)) << 4))) =
+                    make_uint4(packed[4], packed[5], packed[6], packed[7]);
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");  // the four epilogue warps only
+        if (ok) {
+            const int et = tid - 64;  // 0..127: 16 threads per row, 8 rows per pass
+            for (int r = et >> 4; r < kTcM; r += 8) {
+                const int ch = et & 15, m = m0 + r, n = n0 + 8 * ch;
+                if (m < batch && n < L.out) {
+                    const uint4 val = *reinterpret_cast<const uint4*>(smem_at(ring + r * 256 + ((ch ^ (r & 15)) << 4)));
+                    *reinterpret_cast<uint4*>(y + (size_t)m * L.out + n) = val;
+                }
+            }
+        }
+    }
+    if (!ok) atomicExch(L.status, 2);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(128u) : "memory");
+    }
+}

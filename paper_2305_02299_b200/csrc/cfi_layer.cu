@@ -13,6 +13,7 @@
 //     32-byte "quads" (4 weights, 4 columns); seg[r][s] is the first quad of row r in slab s.
 #include "cfi.h"
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -55,6 +56,11 @@ struct cfi_layer {
     void* stage_x = nullptr;
     void* stage_y = nullptr;
     int staged_batch = 0;
+    // Tensor-core variant (bf16 layers whose shapes TMA can address): dense copy of the weight and its tensor map.
+    const void* w_dense = nullptr;
+    int out_pad = 0;
+    bool tc_ok = false;
+    CUtensorMap map_w{};
 };
 
 struct cfi_stack {
@@ -562,6 +568,8 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
     }
 }
 
+#include "cfi_dense_tc.cuh"
+
 // ------------------------------------------------------------------------------------------------
 // host: launch shapes
 // ------------------------------------------------------------------------------------------------
@@ -751,8 +759,54 @@ cfi_status_t launch_simple(const cfi_layer* l, const void* x, void* y, int batch
     return cudaGetLastError() == cudaSuccess ? CFI_OK : CFI_ERR_CUDA;
 }
 
+// cuTensorMapEncodeTiled is a driver entry point; it is looked up once through the runtime so that the library
+// does not link against the driver directly.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static std::atomic<void*> cached{nullptr};
+    void* fn = cached.load(std::memory_order_acquire);
+    if (!fn) {
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        cached.store(fn, std::memory_order_release);
+    }
+    return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
+// Tensor map of a row-major bf16 matrix [rows][cols] read in boxes of 128 rows x 64 columns with the 128-byte
+// swizzle; out-of-range elements read as zero.  Needs a 16-byte aligned base and cols % 8 == 0.
+bool encode_bf16_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || rows == 0 || cols == 0 || (cols & 7) || ((uintptr_t)base & 15)) return false;
+    const cuuint64_t dims[2] = {cols, rows}, strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcK, (cuuint32_t)kTcM}, elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
+    if (!l->tc_ok || l->dtype != CFI_BF16) return CFI_ERR_SHAPE;
+    const int grid_x = (l->d.out + kTcN - 1) / kTcN, grid_y = (batch + kTcM - 1) / kTcM;
+    if (grid_y > 65535) return CFI_ERR_SHAPE;
+    CUtensorMap map_x;
+    if (!encode_bf16_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in)) return CFI_ERR_SHAPE;
+    if (cfi_status_t e = set_smem<cfi_dense_tc_kernel>(kTcSmemBytes, l->device)) return e;
+    return launch_pdl(cfi_dense_tc_kernel, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d, map_x, l->map_w,
+                      static_cast<__nv_bfloat16*>(y), batch);
+}
+
 int choose_variant(const cfi_layer* l, int batch) {
     if (batch <= 8) return CFI_VARIANT_SPLITK;
+    // bf16 at large batch: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
+    // (10 TFLOP/s effective for the gather against several hundred dense); below a full 128-row tile it does not pay.
+    if (l->tc_ok && batch >= 96) return CFI_VARIANT_DENSE_TC;
     return batch_shape(l, batch).ok ? CFI_VARIANT_BATCH : CFI_VARIANT_SPLITK;
 }
 
@@ -992,6 +1046,24 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                           seg_o.begin() + (size_t)o * (d.n_slabs + 1));
         if (st == CFI_OK) st = upload(l, seg_o, &d.seg);
 
+        // ---- dense bf16 copy for the tensor-core variant (zero rows for ablated and padding rows)
+        if (dtype == CFI_BF16 && in_features >= 8 && (in_features & 7) == 0 && (out_features & 7) == 0 && out_features > 0 &&
+            (size_t)out_features * in_features <= ((size_t)1 << 31)) {
+            l->out_pad = ((out_features + kTcN - 1) / kTcN) * kTcN;
+            std::vector<uint16_t> wd((size_t)l->out_pad * in_features, (uint16_t)0);
+            bool repeated = false;  // a column kept twice in one row cannot be one dense entry without re-rounding
+            for (int32_t r = 0; r < n_active; ++r)
+                for (int32_t j = 0; j < k; ++j) {
+                    const int32_t c = c_sorted[(size_t)r * k + j];
+                    repeated = repeated || (j > 0 && c == c_sorted[(size_t)r * k + j - 1]);
+                    wd[(size_t)active_rows[r] * in_features + c] = bf16_bits_rne(v_sorted[(size_t)r * k + j]);
+                }
+            const uint16_t* wd_dev = nullptr;
+            if (st == CFI_OK) st = upload(l, wd, &wd_dev);
+            l->w_dense = wd_dev;
+            l->tc_ok = st == CFI_OK && !repeated && encode_bf16_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features);
+        }
+
         std::vector<float> bias_h((size_t)out_features, 0.0f);
         if (bias) std::copy(bias, bias + out_features, bias_h.begin());
         if (st == CFI_OK) st = upload(l, bias_h, &d.bias);
@@ -1044,6 +1116,8 @@ extern "C" cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void
             return bf ? launch_splitk<__nv_bfloat16>(layer, s, x, y, batch, st)
                       : launch_splitk<float>(layer, s, x, y, batch, st);
         }
+        case CFI_VARIANT_DENSE_TC:
+            return launch_dense_tc(layer, x, y, batch, st);
         case CFI_VARIANT_BATCH: {
             const BatchShape s = batch_shape(layer, batch);
             return bf ? launch_batch<__nv_bfloat16>(layer, s, x, y, batch, st)
