@@ -21,9 +21,9 @@
 //   warp 1, one lane   issues tcgen05.mma (cta_group::1, kind::f16, M = N = 128, K = 16 per instruction,
 //                      both operands K-major from shared memory), accumulator in 128 columns of tensor
 //                      memory; tcgen05.commit hands ring slots back and finally signals the epilogue;
-//   warps 2..5         epilogue: tcgen05.ld the accumulator (one batch row per thread), add bias, apply the
-//                      activation, round to bf16, pass through shared memory (the drained ring) and write
-//                      y in 256-byte runs per batch row.
+//   warps 2..9         epilogue: tcgen05.ld the accumulator (one batch row and half of the 128 columns per
+//                      thread), add bias, apply the activation, round to bf16, pass through shared memory
+//                      (the drained ring) and write y in 256-byte runs per batch row.
 // Two CTAs fit an SM (97 KB of shared memory, 128 of 512 tensor-memory columns each), so one CTA's
 // epilogue overlaps the other's main loop.
 //
@@ -33,7 +33,8 @@
 
 #include <cuda.h>  // CUtensorMap and the enums of cuTensorMapEncodeTiled (types only; the entry point is looked up at run time)
 
-constexpr int kTcM = 128, kTcN = 128, kTcK = 64, kTcStages = 3, kTcThreads = 192;
+constexpr int kTcM = 128, kTcN = 128, kTcK = 64, kTcStages = 3;
+constexpr int kTcEpilogueWarps = 8, kTcThreads = 64 + 32 * kTcEpilogueWarps;
 constexpr uint32_t kTcStageBytes = (kTcM + kTcN) * kTcK * 2;  // 32 KB
 constexpr uint32_t kTcSpinLimit = 1u << 22;
 constexpr size_t kTcSmemBytes = 1024 + kTcStages * kTcStageBytes + 1024;
@@ -101,6 +102,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "memory");
 }
 
+// Activation for the epilogue.  GELU is v * Phi(v) with Phi = (1 + erf(v / sqrt 2)) / 2; erf is evaluated with the
+// rational-times-Gaussian formula of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7, far inside a
+// bf16 result), and the two signs of v are kept apart so that the small tail is not obtained by cancellation.
+__device__ __forceinline__ float activate_tc(float v, int act) {
+    if (act != CFI_ACT_GELU_ERF) return v;
+    const float z = fabsf(v) * 0.70710678118654752f;
+    const float t = __frcp_rn(fmaf(0.3275911f, z, 1.0f));
+    float p = fmaf(1.061405429f, t, -1.453152027f);
+    p = fmaf(p, t, 1.421413741f);
+    p = fmaf(p, t, -0.284496736f);
+    p = fmaf(p, t, 0.254829592f);
+    const float tail = 0.5f * p * t * __expf(-z * z);  // (1 - erf(z)) / 2
+    return v * (v < 0.0f ? tail : 1.0f - tail);
+}
+
 // Shared memory (offsets from the first 1024-byte boundary): the ring, then barriers and small tables.
 //   ring      kTcStages x [A 128 x 64 bf16 | B 128 x 64 bf16]; after the main loop its first 32 KB hold the y tile
 //   +0        full[kTcStages], +32 empty[kTcStages], +64 accumulator barrier, +72 tensor-memory base address
@@ -131,7 +147,7 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (tid >= 64) {
+    if (tid >= 64 && tid < 64 + kTcN) {
         const int n = n0 + tid - 64;
         bias_s[tid - 64] = n < L.out ? L.bias[n] : 0.0f;
     }
@@ -172,34 +188,40 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
         // ---------------------------------------------------------------- epilogue
         ok = mbar_wait(accum, 0u, kTcSpinLimit);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int q = warp & 3;           // a warp may read the tensor-memory lanes 32 q .. 32 q + 31
-        const int row = 32 * q + lane;    // batch row of the tile held by this thread
+        const int q = warp & 3;            // a warp may read the tensor-memory lanes 32 q .. 32 q + 31
+        const int half = (warp - 2) >> 2;  // two warps share a lane quarter and split the 128 columns
+        const int row = 32 * q + lane;     // batch row of the tile held by this thread
         if (ok) {
             // y tile in shared memory: 128 rows x 256 bytes, 16-byte chunks permuted by chunk ^ (row & 15).
 #pragma unroll 1
-            for (int c = 0; c < kTcN; c += 16) {
-                uint32_t v[16];
-                tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
+            for (int c = 64 * half; c < 64 * half + 64; c += 32) {
+                uint32_t v[2][16];
+                tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v[0]);
+                tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(c + 16), v[1]);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                uint32_t packed[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float lo = activate(__uint_as_float(v[2 * e]) + bias_s[c + 2 * e], L.act);
-                    const float hi = activate(__uint_as_float(v[2 * e + 1]) + bias_s[c + 2 * e + 1], L.act);
-                    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
-                    packed[e] = *reinterpret_cast<const uint32_t*>(&p);
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t packed[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int col = c + 16 * h + 2 * e;
+                        const float lo = activate_tc(__uint_as_float(v[h][2 * e]) + bias_s[col], L.act);
+                        const float hi = activate_tc(__uint_as_float(v[h][2 * e + 1]) + bias_s[col + 1], L.act);
+                        const __nv_bfloat162 p2 = __floats2bfloat162_rn(lo, hi);
+                        packed[e] = *reinterpret_cast<const uint32_t*>(&p2);
+                    }
+                    const int ch = (c + 16 * h) >> 3;  // 16-byte chunk of columns .. +7; the next one holds +8 .. +15
+                    *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + ((ch ^ (row & 15)) << 4))) =
+                        make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + (((ch + 1) ^ (row & 15)) << 4))) =
+                        make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
-                const int ch = c >> 3;  // 16-byte chunk index of columns c .. c+7; the next one holds c+8 .. c+15
-                *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + (((ch) ^ (row & 15)) << 4))) =
-                    make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + (((ch + 1) ^ (row & 15)) << 4))) =
-                    make_uint4(packed[4], packed[5], packed[6], packed[7]);
             }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");  // the four epilogue warps only
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kTcEpilogueWarps) : "memory");  // the epilogue warps only
         if (ok) {
-            const int et = tid - 64;  // 0..127: 16 threads per row, 8 rows per pass
-            for (int r = et >> 4; r < kTcM; r += 8) {
+            const int et = tid - 64;  // 16 threads per row, 16 rows per pass
+            for (int r = et >> 4; r < kTcM; r += 2 * kTcEpilogueWarps) {
                 const int ch = et & 15, m = m0 + r, n = n0 + 8 * ch;
                 if (m < batch && n < L.out) {
                     const uint4 val = *reinterpret_cast<const uint4*>(smem_at(ring + r * 256 + ((ch ^ (r & 15)) << 4)));
