@@ -296,6 +296,8 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--variant", default="auto")
     ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
+    ap.add_argument("--stack-only", type=int, default=0, metavar="ROWS",
+                    help="run only the bf16 MLP stack leg on ROWS batch rows (for profiling) and print its JSON")
     args = ap.parse_args()
     W = inputs.workloads()
     w = W[args.workload]
@@ -310,6 +312,13 @@ def main():
 
     import torch
     from paper_2305_02299_b200 import binding as cfi   # raises if the CUDA library is missing
+
+    if args.stack_only:
+        torch.cuda.set_device(0)
+        peaks, _ = measured_peaks()
+        print(json.dumps(stack_leg(cfi, torch, peaks, torch.cuda.get_device_properties(0).multi_processor_count,
+                                   rows=args.stack_only, blocks=1)))
+        return
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -425,9 +434,9 @@ def context_leg(w, torch):
     return out
 
 
-def stack_leg(cfi, torch, peaks, sm_count):
+def stack_leg(cfi, torch, peaks, sm_count, rows=None, blocks=12):
     """The bf16 MLP stack (12 blocks of 768 -> 3072 GELU -> 768, 5 % of rows ablated, 50,432 rows)."""
-    s = inputs.StackWorkload()
+    s = inputs.StackWorkload(blocks=blocks) if rows is None else inputs.StackWorkload(blocks=blocks, batch=rows)
     layers, flops, bytes_ = [], 0, 0
     for L, sp in zip(s.layers(seed=0), s.layer_specs()):
         v, ix, rows = cfi.cfi_pack(L.w_dense, L.mask)

@@ -102,25 +102,33 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "memory");
 }
 
-// Activation for the epilogue.  GELU is v * Phi(v) with Phi = (1 + erf(v / sqrt 2)) / 2; erf is evaluated with the
-// rational-times-Gaussian formula of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7, far inside a
-// bf16 result), and the two signs of v are kept apart so that the small tail is not obtained by cancellation.
-__device__ __forceinline__ float activate_tc(float v, int act) {
-    if (act != CFI_ACT_GELU_ERF) return v;
-    const float z = fabsf(v) * 0.70710678118654752f;
-    const float t = __frcp_rn(fmaf(0.3275911f, z, 1.0f));
-    float p = fmaf(1.061405429f, t, -1.453152027f);
-    p = fmaf(p, t, 1.421413741f);
-    p = fmaf(p, t, -0.284496736f);
-    p = fmaf(p, t, 0.254829592f);
-    const float tail = 0.5f * p * t * __expf(-z * z);  // (1 - erf(z)) / 2
-    return v * (v < 0.0f ? tail : 1.0f - tail);
+// Activation for the epilogue, chosen at compile time.  GELU is v * Phi(v) with Phi = (1 + erf(v / sqrt 2)) / 2;
+// erf is evaluated with the rational-times-Gaussian formula of Abramowitz & Stegun 7.1.26 (absolute error
+// below 1.5e-7, far inside a bf16 result), with the factors 1/sqrt 2 and 1/2 folded into its constants, and
+// the two signs of v are kept apart so that the small tail is not obtained by cancellation.
+template <int ACT>
+__device__ __forceinline__ float activate_tc(float v) {
+    if constexpr (ACT != CFI_ACT_GELU_ERF) {
+        return v;
+    } else {
+        float t;  // 1 / (1 + 0.3275911 |v| / sqrt 2)
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(fabsf(v), 0.23164189f, 1.0f)));
+        float p = fmaf(0.5307027145f, t, -0.7265760135f);  // half the published coefficients
+        p = fmaf(p, t, 0.7107068705f);
+        p = fmaf(p, t, -0.142248368f);
+        p = fmaf(p, t, 0.127414796f);
+        float e;  // exp(-v^2 / 2) = 2^(-v^2 * log2(e) / 2)
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(v * v * -0.72134752f));
+        const float m = v * (p * t * e);  // v * (1 - erf(|v| / sqrt 2)) / 2
+        return v < 0.0f ? m : v - m;
+    }
 }
 
 // Shared memory (offsets from the first 1024-byte boundary): the ring, then barriers and small tables.
 //   ring      kTcStages x [A 128 x 64 bf16 | B 128 x 64 bf16]; after the main loop its first 32 KB hold the y tile
 //   +0        full[kTcStages], +32 empty[kTcStages], +64 accumulator barrier, +72 tensor-memory base address
 //   +128      bias of the tile's 128 output rows
+template <int ACT>
 __global__ void __launch_bounds__(kTcThreads, 2)
 cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                     __nv_bfloat16* __restrict__ y, int batch) {
@@ -203,12 +211,15 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
                 for (int h = 0; h < 2; ++h) {
                     uint32_t packed[8];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const int col = c + 16 * h + 2 * e;
-                        const float lo = activate_tc(__uint_as_float(v[h][2 * e]) + bias_s[col], L.act);
-                        const float hi = activate_tc(__uint_as_float(v[h][2 * e + 1]) + bias_s[col + 1], L.act);
-                        const __nv_bfloat162 p2 = __floats2bfloat162_rn(lo, hi);
-                        packed[e] = *reinterpret_cast<const uint32_t*>(&p2);
+                    for (int e4 = 0; e4 < 4; ++e4) {
+                        const float4 bv = *reinterpret_cast<const float4*>(bias_s + c + 16 * h + 4 * e4);
+                        const float r0 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 0]) + bv.x);
+                        const float r1 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 1]) + bv.y);
+                        const float r2 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 2]) + bv.z);
+                        const float r3 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 3]) + bv.w);
+                        const __nv_bfloat162 p01 = __floats2bfloat162_rn(r0, r1), p23 = __floats2bfloat162_rn(r2, r3);
+                        packed[2 * e4] = *reinterpret_cast<const uint32_t*>(&p01);
+                        packed[2 * e4 + 1] = *reinterpret_cast<const uint32_t*>(&p23);
                     }
                     const int ch = (c + 16 * h) >> 3;  // 16-byte chunk of columns .. +7; the next one holds +8 .. +15
                     *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + ((ch ^ (row & 15)) << 4))) =

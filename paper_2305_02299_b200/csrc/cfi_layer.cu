@@ -797,9 +797,14 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
     if (grid_y > 65535) return CFI_ERR_SHAPE;
     CUtensorMap map_x;
     if (!encode_bf16_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in)) return CFI_ERR_SHAPE;
-    if (cfi_status_t e = set_smem<cfi_dense_tc_kernel>(kTcSmemBytes, l->device)) return e;
-    return launch_pdl(cfi_dense_tc_kernel, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d, map_x, l->map_w,
-                      static_cast<__nv_bfloat16*>(y), batch);
+    if (l->d.act == CFI_ACT_GELU_ERF) {
+        if (cfi_status_t e = set_smem<cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>>(kTcSmemBytes, l->device)) return e;
+        return launch_pdl(cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d,
+                          map_x, l->map_w, static_cast<__nv_bfloat16*>(y), batch);
+    }
+    if (cfi_status_t e = set_smem<cfi_dense_tc_kernel<CFI_ACT_NONE>>(kTcSmemBytes, l->device)) return e;
+    return launch_pdl(cfi_dense_tc_kernel<CFI_ACT_NONE>, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d, map_x,
+                      l->map_w, static_cast<__nv_bfloat16*>(y), batch);
 }
 
 int choose_variant(const cfi_layer* l, int batch) {
