@@ -1,0 +1,188 @@
+// CFI_VARIANT_DENSE_TC for fp32 layers: the dense contraction on the tensor cores in split TF32.
+//
+// Included by cfi_layer.cu after cfi_dense_tc.cuh (it reuses that file's mbarrier, TMA, descriptor and
+// tensor-memory helpers).
+//
+// A TF32 operand keeps 11 significant bits of an fp32 number, which alone would miss the 1e-5 tolerance of
+// the fp32 layer by two orders of magnitude.  Each operand is therefore split into two TF32-exact parts,
+//
+//     a = a_hi + a_lo + r,   a_hi = a with the low 13 mantissa bits cleared,   a_lo = (a - a_hi) likewise cleared,
+//
+// so that |r| < 2^-21 |a|, and the product is taken as  x_hi w_hi + x_hi w_lo + x_lo w_hi  (three MMAs, fp32
+// accumulation in tensor memory).  What is dropped (x_lo w_lo and the two remainders) is below 2^-19 of the
+// term, fifty times inside the tolerance.  Because both parts are exactly representable in TF32, the result
+// does not depend on how the tensor core would convert a general fp32 operand.
+//
+// The layer keeps one dense fp32 copy of its weight, Wd[out_pad][in].  Per 32-column block of K:
+//   warp 0, one lane   TMA: a 128 x 32 box of x and a 64 x 32 box of Wd (fp32, 128-byte swizzle) into a ring slot;
+//   warps 2..9         split both boxes in shared memory, hi in place and lo into the slot's second half (the
+//                      split is element-wise, so the swizzled layout is untouched), make the writes visible to
+//                      the tensor core (fence.proxy.async) and arrive on the slot's "ready" barrier;
+//   warp 1, one lane   4 K-steps x 3 tcgen05.mma (kind::tf32, M = 128, N = 64, K = 8), then tcgen05.commit
+//                      frees the slot;
+// and after the last block warps 2..9 run the epilogue: tcgen05.ld, bias, activation, y tile through shared
+// memory, 256-byte runs per batch row.  All mbarrier waits are bounded (status code 2), as in the bf16 kernel.
+
+constexpr int kTfM = 128, kTfN = 64, kTfK = 32, kTfStages = 3;
+constexpr int kTfWorkerWarps = 8, kTfThreads = 64 + 32 * kTfWorkerWarps;
+constexpr uint32_t kTfABytes = kTfM * kTfK * 4, kTfBBytes = kTfN * kTfK * 4;   // 16 KB, 8 KB
+constexpr uint32_t kTfStageBytes = 2 * (kTfABytes + kTfBBytes);                // raw/hi then lo: 48 KB
+constexpr size_t kTfSmemBytes = 1024 + kTfStages * kTfStageBytes + 1024;
+
+// fp32 accumulate, tf32 x tf32, both K-major, N = 64, M = 128.
+constexpr uint32_t kTfInstrDesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTfN >> 3) << 17) | ((uint32_t)(kTfM >> 4) << 24);
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(kTfInstrDesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+}
+
+// hi = v with the 13 low mantissa bits cleared; lo = the same of (v - hi).  Both are exact TF32 numbers.
+__device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
+    hi = __uint_as_float(__float_as_uint(v) & 0xFFFFE000u);
+    lo = __uint_as_float(__float_as_uint(v - hi) & 0xFFFFE000u);
+}
+
+// Shared memory from the first 1024-byte boundary: kTfStages slots of [A hi | B hi | A lo | B lo]; then
+//   +0 full[3], +32 ready[3], +64 empty[3], +96 accumulator barrier, +104 tensor-memory base, +128 bias[64].
+__global__ void __launch_bounds__(kTfThreads, 1)
+cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                      float* __restrict__ y, int batch) {
+    pdl_launch_dependents();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t base = ((smem_u32(0) + 1023u) & ~1023u) - smem_u32(0);
+    const uint32_t ring = base, ctl = base + kTfStages * kTfStageBytes;
+    const uint32_t full0 = smem_u32(ctl), ready0 = smem_u32(ctl + 32), empty0 = smem_u32(ctl + 64), accum = smem_u32(ctl + 96);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_at(ctl + 104));
+    float* bias_s = reinterpret_cast<float*>(smem_at(ctl + 128));
+    const int m0 = blockIdx.y * kTfM, n0 = blockIdx.x * kTfN;
+    const int k_blocks = (L.in + kTfK - 1) / kTfK;
+
+    if (tid == 0) {
+        for (int s = 0; s < kTfStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(ready0 + 8 * s, 32 * kTfWorkerWarps);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accum, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(ctl + 104)), "r"(64u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid >= 64 && tid < 64 + kTfN) {
+        const int n = n0 + tid - 64;
+        bias_s[tid - 64] = n < L.out ? L.bias[n] : 0.0f;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // x and y may belong to the kernel before this one
+    bool ok = true;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % kTfStages;
+            if (kb >= kTfStages) ok = mbar_wait(empty0 + 8 * s, (uint32_t)(kb / kTfStages - 1) & 1u, kTcSpinLimit);
+            if (!ok) break;
+            const uint32_t a_dst = smem_u32(ring + s * kTfStageBytes), b_dst = a_dst + kTfABytes;
+            mbar_expect_tx(full0 + 8 * s, kTfABytes + kTfBBytes);
+            tma_load_2d(a_dst, &map_x, full0 + 8 * s, kb * kTfK, m0);
+            tma_load_2d(b_dst, &map_w, full0 + 8 * s, kb * kTfK, n0);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------------------------------------------------------- MMA issuer
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % kTfStages;
+            ok = mbar_wait(ready0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_hi = smem_u32(ring + s * kTfStageBytes), b_hi = a_hi + kTfABytes;
+            const uint32_t a_lo = a_hi + kTfABytes + kTfBBytes, b_lo = a_lo + kTfABytes;
+            const uint64_t dah = umma_desc_k_sw128(a_hi), dbh = umma_desc_k_sw128(b_hi);
+            const uint64_t dal = umma_desc_k_sw128(a_lo), dbl = umma_desc_k_sw128(b_lo);
+#pragma unroll
+            for (int k = 0; k < kTfK / 8; ++k) {  // 8 fp32 = 32 bytes further along K inside the swizzled row
+                const uint64_t off = (uint64_t)(2 * k);
+                umma_tf32(tmem_base, dal + off, dbh + off, (kb | k) != 0 ? 1u : 0u);  // small terms first
+                umma_tf32(tmem_base, dah + off, dbl + off, 1u);
+                umma_tf32(tmem_base, dah + off, dbh + off, 1u);
+            }
+            umma_commit(empty0 + 8 * s);
+        }
+        if (ok) umma_commit(accum);
+    } else if (warp >= 2) {
+        // ---------------------------------------------------------------- split, then epilogue
+        const int wt = tid - 64;  // 0..255
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % kTfStages;
+            ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
+            if (!ok) break;
+            const uint32_t hi_off = ring + s * kTfStageBytes, lo_off = hi_off + kTfABytes + kTfBBytes;
+#pragma unroll 2
+            for (uint32_t e = wt * 16u; e < kTfABytes + kTfBBytes; e += 32u * kTfWorkerWarps * 16u) {
+                float4 v = *reinterpret_cast<const float4*>(smem_at(hi_off + e)), h, l;
+                split_tf32(v.x, h.x, l.x);
+                split_tf32(v.y, h.y, l.y);
+                split_tf32(v.z, h.z, l.z);
+                split_tf32(v.w, h.w, l.w);
+                *reinterpret_cast<float4*>(smem_at(hi_off + e)) = h;
+                *reinterpret_cast<float4*>(smem_at(lo_off + e)) = l;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
+            mbar_arrive(ready0 + 8 * s);
+        }
+        if (ok) ok = mbar_wait(accum, 0u, kTcSpinLimit);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int q = warp & 3;            // tensor-memory lanes 32 q .. 32 q + 31
+        const int half = (warp - 2) >> 2;  // two warps share a lane quarter and split the 64 columns
+        const int row = 32 * q + lane;
+        if (ok) {
+            // y tile in shared memory: 128 rows x 256 bytes (64 fp32), 16-byte chunks permuted by chunk ^ (row & 15).
+            uint32_t v[2][16];
+            tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * half), v[0]);
+            tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * half + 16), v[1]);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int e4 = 0; e4 < 4; ++e4) {
+                    const int col = 32 * half + 16 * h + 4 * e4;
+                    const float4 bv = *reinterpret_cast<const float4*>(bias_s + col);
+                    float4 r;
+                    r.x = activate(__uint_as_float(v[h][4 * e4 + 0]) + bv.x, L.act);
+                    r.y = activate(__uint_as_float(v[h][4 * e4 + 1]) + bv.y, L.act);
+                    r.z = activate(__uint_as_float(v[h][4 * e4 + 2]) + bv.z, L.act);
+                    r.w = activate(__uint_as_float(v[h][4 * e4 + 3]) + bv.w, L.act);
+                    *reinterpret_cast<float4*>(smem_at(ring + row * 256 + (((col >> 2) ^ (row & 15)) << 4))) = r;
+                }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kTfWorkerWarps) : "memory");
+        if (ok) {
+            for (int r = wt >> 4; r < kTfM; r += 2 * kTfWorkerWarps) {  // 16 threads per row, 16 rows per pass
+                const int ch = wt & 15, m = m0 + r, n = n0 + 4 * ch;
+                if (m < batch && n < L.out) {
+                    const float4 val = *reinterpret_cast<const float4*>(smem_at(ring + r * 256 + ((ch ^ (r & 15)) << 4)));
+                    *reinterpret_cast<float4*>(y + (size_t)m * L.out + n) = val;
+                }
+            }
+        }
+    }
+    if (!ok) atomicExch(L.status, 2);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(64u) : "memory");
+    }
+}

@@ -569,6 +569,7 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 }
 
 #include "cfi_dense_tc.cuh"
+#include "cfi_dense_tf32.cuh"
 
 // ------------------------------------------------------------------------------------------------
 // host: launch shapes
@@ -779,24 +780,35 @@ EncodeTiledFn encode_tiled_fn() {
     return reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-// Tensor map of a row-major bf16 matrix [rows][cols] read in boxes of 128 rows x 64 columns with the 128-byte
-// swizzle; out-of-range elements read as zero.  Needs a 16-byte aligned base and cols % 8 == 0.
-bool encode_bf16_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols) {
+// Tensor map of a row-major bf16 or fp32 matrix [rows][cols] read in boxes of box_rows rows x 128 bytes of columns
+// with the 128-byte swizzle; out-of-range elements read as zero.  Needs a 16-byte aligned base and row pitch.
+bool encode_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, int elem_bytes, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn || rows == 0 || cols == 0 || (cols & 7) || ((uintptr_t)base & 15)) return false;
-    const cuuint64_t dims[2] = {cols, rows}, strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTcK, (cuuint32_t)kTcM}, elem[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (!fn || rows == 0 || cols == 0 || ((cols * elem_bytes) & 15) || ((uintptr_t)base & 15)) return false;
+    const cuuint64_t dims[2] = {cols, rows}, strides[1] = {cols * (uint64_t)elem_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows}, elem[2] = {1, 1};
+    return fn(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+              const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cfi_status_t launch_dense_tf32(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
+    const int grid_x = (l->d.out + kTfN - 1) / kTfN, grid_y = (batch + kTfM - 1) / kTfM;
+    if (grid_y > 65535) return CFI_ERR_SHAPE;
+    CUtensorMap map_x;
+    if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 4, kTfM)) return CFI_ERR_SHAPE;
+    if (cfi_status_t e = set_smem<cfi_dense_tf32_kernel>(kTfSmemBytes, l->device)) return e;
+    return launch_pdl(cfi_dense_tf32_kernel, dim3(grid_x, grid_y), kTfThreads, kTfSmemBytes, st, l->d, map_x, l->map_w,
+                      static_cast<float*>(y), batch);
 }
 
 cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
-    if (!l->tc_ok || l->dtype != CFI_BF16) return CFI_ERR_SHAPE;
+    if (!l->tc_ok) return CFI_ERR_SHAPE;
+    if (l->dtype != CFI_BF16) return launch_dense_tf32(l, x, y, batch, st);
     const int grid_x = (l->d.out + kTcN - 1) / kTcN, grid_y = (batch + kTcM - 1) / kTcM;
     if (grid_y > 65535) return CFI_ERR_SHAPE;
     CUtensorMap map_x;
-    if (!encode_bf16_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in)) return CFI_ERR_SHAPE;
+    if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 2, kTcM)) return CFI_ERR_SHAPE;
     if (l->d.act == CFI_ACT_GELU_ERF) {
         if (cfi_status_t e = set_smem<cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>>(kTcSmemBytes, l->device)) return e;
         return launch_pdl(cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d,
@@ -807,11 +819,22 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
                       l->map_w, static_cast<__nv_bfloat16*>(y), batch);
 }
 
+// Rates used to choose between the gather kernel and the split-TF32 dense kernel for fp32 layers (measured).
+constexpr double kDenseTf32Tflops = 500.0, kGatherTflops = 9.0;
+
 int choose_variant(const cfi_layer* l, int batch) {
     if (batch <= 8) return CFI_VARIANT_SPLITK;
     // bf16 at large batch: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
     // (10 TFLOP/s effective for the gather against several hundred dense); below a full 128-row tile it does not pay.
-    if (l->tc_ok && batch >= 96) return CFI_VARIANT_DENSE_TC;
+    if (l->tc_ok && batch >= 96) {
+        if (l->dtype == CFI_BF16) return CFI_VARIANT_DENSE_TC;
+        // fp32: three TF32 MMAs per product against the gather kernel's ~9 TFLOP/s effective.
+        const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + kTfN - 1) / kTfN);
+        const int64_t waves = (tiles + l->sm_count - 1) / l->sm_count;
+        const double t_dense = (double)waves * (6.0 * kTfM * kTfN * l->d.in) / (kDenseTf32Tflops * 1e12 / l->sm_count) + 5e-6;
+        const double t_gather = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12) + 6e-6;
+        if (t_dense < t_gather) return CFI_VARIANT_DENSE_TC;
+    }
     return batch_shape(l, batch).ok ? CFI_VARIANT_BATCH : CFI_VARIANT_SPLITK;
 }
 
@@ -1051,22 +1074,39 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                           seg_o.begin() + (size_t)o * (d.n_slabs + 1));
         if (st == CFI_OK) st = upload(l, seg_o, &d.seg);
 
-        // ---- dense bf16 copy for the tensor-core variant (zero rows for ablated and padding rows)
-        if (dtype == CFI_BF16 && in_features >= 8 && (in_features & 7) == 0 && (out_features & 7) == 0 && out_features > 0 &&
-            (size_t)out_features * in_features <= ((size_t)1 << 31)) {
-            l->out_pad = ((out_features + kTcN - 1) / kTcN) * kTcN;
-            std::vector<uint16_t> wd((size_t)l->out_pad * in_features, (uint16_t)0);
-            bool repeated = false;  // a column kept twice in one row cannot be one dense entry without re-rounding
-            for (int32_t r = 0; r < n_active; ++r)
-                for (int32_t j = 0; j < k; ++j) {
-                    const int32_t c = c_sorted[(size_t)r * k + j];
-                    repeated = repeated || (j > 0 && c == c_sorted[(size_t)r * k + j - 1]);
-                    wd[(size_t)active_rows[r] * in_features + c] = bf16_bits_rne(v_sorted[(size_t)r * k + j]);
+        // ---- dense copy for the tensor-core variant (zero rows for ablated and padding rows): bf16 for bf16 layers,
+        // fp32 for fp32 layers.  A column kept twice in one row cannot be one dense entry, so such layers go without.
+        {
+            const int eb = dtype == CFI_BF16 ? 2 : 4, tile_n = dtype == CFI_BF16 ? kTcN : kTfN;
+            bool usable = out_features > 0 && in_features * eb >= 16 && ((in_features * eb) & 15) == 0 &&
+                          ((out_features * eb) & 15) == 0 && (size_t)out_features * in_features * eb <= ((size_t)1 << 30);
+            for (int32_t r = 0; usable && r < n_active; ++r)
+                for (int32_t j = 1; j < k; ++j) usable = usable && c_sorted[(size_t)r * k + j] != c_sorted[(size_t)r * k + j - 1];
+            if (usable) {
+                l->out_pad = ((out_features + tile_n - 1) / tile_n) * tile_n;
+                const void* wd_dev = nullptr;
+                if (dtype == CFI_BF16) {
+                    std::vector<uint16_t> wd((size_t)l->out_pad * in_features, (uint16_t)0);
+                    for (int32_t r = 0; r < n_active; ++r)
+                        for (int32_t j = 0; j < k; ++j)
+                            wd[(size_t)active_rows[r] * in_features + c_sorted[(size_t)r * k + j]] =
+                                bf16_bits_rne(v_sorted[(size_t)r * k + j]);
+                    const uint16_t* p = nullptr;
+                    if (st == CFI_OK) st = upload(l, wd, &p);
+                    wd_dev = p;
+                } else {
+                    std::vector<float> wd((size_t)l->out_pad * in_features, 0.0f);
+                    for (int32_t r = 0; r < n_active; ++r)
+                        for (int32_t j = 0; j < k; ++j)
+                            wd[(size_t)active_rows[r] * in_features + c_sorted[(size_t)r * k + j]] = v_sorted[(size_t)r * k + j];
+                    const float* p = nullptr;
+                    if (st == CFI_OK) st = upload(l, wd, &p);
+                    wd_dev = p;
                 }
-            const uint16_t* wd_dev = nullptr;
-            if (st == CFI_OK) st = upload(l, wd, &wd_dev);
-            l->w_dense = wd_dev;
-            l->tc_ok = st == CFI_OK && !repeated && encode_bf16_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features);
+                l->w_dense = wd_dev;
+                l->tc_ok = st == CFI_OK && encode_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb,
+                                                      dtype == CFI_BF16 ? kTcN : kTfN);
+            }
         }
 
         std::vector<float> bias_h((size_t)out_features, 0.0f);

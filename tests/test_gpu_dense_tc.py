@@ -1,7 +1,9 @@
-"""The tensor-core variant (dense bf16 copy of the weight, tcgen05) against the oracle, element by element.
+"""The tensor-core variant (dense copy of the weight, tcgen05) against the oracle, element by element.
 
-It computes the same sums as the condensed forms (exact bf16 products, fp32 accumulation), so the bf16
-tolerance of the other parity tests applies and small-integer cases must agree bit for bit.
+bf16 layers: exact bf16 products, fp32 accumulation, so the bf16 tolerance of the other parity tests applies.
+fp32 layers: three TF32 products of operands split into two TF32-exact parts; what the split drops is below
+2^-19 of each term, so the fp32 tolerance (1e-5 of the sum's scale) applies unchanged.  Small-integer cases
+must agree bit for bit in both.
 """
 import numpy as np
 import pytest
@@ -15,25 +17,41 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("in_f,out_f,k,nabl", [(64, 8, 5, 1), (72, 136, 9, 10), (768, 384, 77, 19), (3072, 200, 307, 20)])
 @pytest.mark.parametrize("B", [1, 5, 128, 257])
 @pytest.mark.parametrize("act", ["none", "gelu"])
-def test_dense_tc_matches_oracle(in_f, out_f, k, nabl, B, act):
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_dense_tc_matches_oracle(in_f, out_f, k, nabl, B, act, dtype):
     L = inputs.make_layer(in_f, out_f, k, n_ablated=nabl, seed=in_f + B)
     x = inputs.make_x(B, in_f, seed=B)
-    y_ref, S = oracle_layer(L, x, "bf16", act)
-    dl = device_layer(L, "bf16", act)
-    y = run_device(dl, x, "bf16", "dense_tc")
+    y_ref, S = oracle_layer(L, x, dtype, act)
+    dl = device_layer(L, dtype, act)
+    y = run_device(dl, x, dtype, "dense_tc")
     dl.close()
     assert np.all(np.isfinite(y))
-    assert scaled_error(y, y_ref, S) <= TOL["bf16"]
+    assert scaled_error(y, y_ref, S) <= TOL[dtype]
 
 
-def test_dense_tc_exact_integers_and_agreement_with_gather():
+def test_dense_tf32_wide_dynamic_range():
+    """Inputs spread over many binades: the split must hold for every magnitude, not only for N(0,1)."""
+    L = inputs.make_layer(512, 128, 51, n_ablated=7, seed=9)
+    rng = np.random.default_rng(4)
+    x = (inputs.make_x(130, 512, seed=9) * np.exp2(rng.integers(-20, 20, size=(130, 512)))).astype(np.float32)
+    L.w_dense *= np.exp2(rng.integers(-12, 12, size=L.w_dense.shape)).astype(np.float32)
+    y_ref, S = oracle_layer(L, x, "f32")
+    dl = device_layer(L, "f32")
+    y = run_device(dl, x, "f32", "dense_tc")
+    dl.close()
+    assert scaled_error(y, y_ref, S) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_dense_tc_exact_integers_and_agreement_with_gather(dtype):
     L = inputs.make_layer(512, 152, 24, n_ablated=11, seed=7, integer_valued=True)
-    x = inputs.make_x(200, 512, seed=7, integer_valued=True, density=0.15)
-    y_ref, _ = oracle_layer(L, x, "bf16")
-    assert np.max(np.abs(y_ref)) <= 256
-    dl = device_layer(L, "bf16")
-    y_tc = run_device(dl, x, "bf16", "dense_tc")
-    y_gather = run_device(dl, x, "bf16", "batch")
+    x = inputs.make_x(200, 512, seed=7, integer_valued=True, density=0.15 if dtype == "bf16" else 1.0)
+    y_ref, _ = oracle_layer(L, x, dtype)
+    if dtype == "bf16":
+        assert np.max(np.abs(y_ref)) <= 256
+    dl = device_layer(L, dtype)
+    y_tc = run_device(dl, x, dtype, "dense_tc")
+    y_gather = run_device(dl, x, dtype, "batch")
     dl.close()
     assert np.array_equal(y_tc, y_ref) and np.array_equal(y_gather, y_ref)
 
@@ -46,9 +64,9 @@ def test_dense_tc_refuses_shapes_it_cannot_address():
         run_device(dl, inputs.make_x(4, 100), "bf16", "dense_tc")
     assert e.value.status == 2
     dl.close()
-    L = inputs.make_layer(64, 16, 4, seed=1)             # fp32 layers have no dense bf16 copy
+    L = inputs.make_layer(30, 16, 4, seed=1)             # fp32 rows of 120 bytes: not a multiple of 16
     dl = device_layer(L, "f32")
     with pytest.raises(cfi.CfiError):
-        run_device(dl, inputs.make_x(4, 64), "f32", "dense_tc")
+        run_device(dl, inputs.make_x(4, 30), "f32", "dense_tc")
     assert cfi.cfi_device_status(dl) == 0
     dl.close()
