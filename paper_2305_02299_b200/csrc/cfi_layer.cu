@@ -820,7 +820,7 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
 }
 
 // Rates used to choose between the gather kernel and the split-TF32 dense kernel for fp32 layers (measured).
-constexpr double kDenseTf32Tflops = 500.0, kGatherTflops = 9.0;
+constexpr double kDenseTf32SecondsPerBlock = 0.78e-6, kGatherTflops = 12.5;
 
 int choose_variant(const cfi_layer* l, int batch) {
     if (batch <= 8) return CFI_VARIANT_SPLITK;
@@ -828,11 +828,16 @@ int choose_variant(const cfi_layer* l, int batch) {
     // (10 TFLOP/s effective for the gather against several hundred dense); below a full 128-row tile it does not pay.
     if (l->tc_ok && batch >= 96) {
         if (l->dtype == CFI_BF16) return CFI_VARIANT_DENSE_TC;
-        // fp32: three TF32 MMAs per product against the gather kernel's ~9 TFLOP/s effective.
+        // fp32: the split-TF32 kernel takes a fixed time per 32-column block of K and tile (it is bound by the
+        // shared-memory traffic of splitting and re-reading the operands); the gather kernel's time is its FMAs
+        // at the rate it sustains plus the re-staging of x by every row tile.  Constants fitted to measurements.
+        const BatchShape bs = batch_shape(l, batch);
+        if (!bs.ok) return CFI_VARIANT_DENSE_TC;
         const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + kTfN - 1) / kTfN);
         const int64_t waves = (tiles + l->sm_count - 1) / l->sm_count;
-        const double t_dense = (double)waves * (6.0 * kTfM * kTfN * l->d.in) / (kDenseTf32Tflops * 1e12 / l->sm_count) + 5e-6;
-        const double t_gather = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12) + 6e-6;
+        const double t_dense = (double)waves * ((l->d.in + kTfK - 1) / kTfK) * kDenseTf32SecondsPerBlock + 3e-6;
+        const double staging = (double)bs.grid_y * kBatchTile * l->d.in * 4.0 * bs.grid_x;
+        const double t_gather = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12) + staging / 3e12 + 5e-6;
         if (t_dense < t_gather) return CFI_VARIANT_DENSE_TC;
     }
     return batch_shape(l, batch).ok ? CFI_VARIANT_BATCH : CFI_VARIANT_SPLITK;
