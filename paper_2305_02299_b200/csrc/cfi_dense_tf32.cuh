@@ -15,32 +15,49 @@
 //
 // The layer keeps one dense fp32 copy of its weight, Wd[out_pad][in].  Per 32-column block of K:
 //   warp 0, one lane   TMA: a 128 x 32 box of x and a 64 x 32 box of Wd (fp32, 128-byte swizzle) into a ring slot;
-//   warps 2..9         split both boxes in shared memory, hi in place and lo into the slot's second half (the
-//                      split is element-wise, so the swizzled layout is untouched), make the writes visible to
-//                      the tensor core (fence.proxy.async) and arrive on the slot's "ready" barrier;
-//   warp 1, one lane   4 K-steps x 3 tcgen05.mma (kind::tf32, M = 128, N = 64, K = 8), then tcgen05.commit
-//                      frees the slot;
+//   warps 2..5         split the x box: a thread reads its batch row from shared memory and writes hi and lo
+//                      straight into tensor memory (tcgen05.st), from where the MMA takes its A operand, so
+//                      x costs shared-memory bandwidth once instead of once per MMA;
+//   warps 6..9         split the Wd box in shared memory, hi in place and lo beside it (element-wise, so the
+//                      swizzled layout is untouched), and make the writes visible to the tensor core
+//                      (fence.proxy.async);
+//   warp 1, one lane   once all 256 splitting threads have arrived on the slot's "ready" barrier:
+//                      4 K-steps x 3 tcgen05.mma (kind::tf32, M = 128, N = 64, K = 8, A from tensor memory, B
+//                      from shared memory), then tcgen05.commit frees the slot;
 // and after the last block warps 2..9 run the epilogue: tcgen05.ld, bias, activation, y tile through shared
-// memory, 256-byte runs per batch row.  All mbarrier waits are bounded (status code 2), as in the bf16 kernel.
+// memory, 256-byte runs per batch row.  Tensor memory: columns 0..63 accumulator, then per slot 32 columns of
+// x_hi and 32 of x_lo.  All mbarrier waits are bounded (status code 2), as in the bf16 kernel.
 
-constexpr int kTfM = 128, kTfN = 64, kTfK = 32, kTfStages = 3;
+constexpr int kTfM = 128, kTfN = 64, kTfK = 32, kTfStages = 4;
 constexpr int kTfWorkerWarps = 8, kTfThreads = 64 + 32 * kTfWorkerWarps;
 constexpr uint32_t kTfABytes = kTfM * kTfK * 4, kTfBBytes = kTfN * kTfK * 4;   // 16 KB, 8 KB
-constexpr uint32_t kTfStageBytes = 2 * (kTfABytes + kTfBBytes);                // raw/hi then lo: 48 KB
+constexpr uint32_t kTfStageBytes = kTfABytes + 2 * kTfBBytes;                  // x raw | Wd hi | Wd lo: 32 KB
+constexpr uint32_t kTfTmemCols = 512;                                          // 64 + 4 * 64 = 320, next power of two
 constexpr size_t kTfSmemBytes = 1024 + kTfStages * kTfStageBytes + 1024;
 
 // fp32 accumulate, tf32 x tf32, both K-major, N = 64, M = 128.
 constexpr uint32_t kTfInstrDesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTfN >> 3) << 17) | ((uint32_t)(kTfM >> 4) << 24);
 
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
+// A operand from tensor memory (row m in lane m, 32-bit elements in consecutive columns), B from shared memory.
+__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
-        "l"(desc_a), "l"(desc_b), "r"(kTfInstrDesc), "r"(accumulate), "r"(0u)
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(desc_b), "r"(kTfInstrDesc), "r"(accumulate), "r"(0u)
         : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
 }
 
 // hi = v with the 13 low mantissa bits cleared; lo = the same of (v - hi).  Both are exact TF32 numbers.
@@ -49,8 +66,8 @@ __device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
     lo = __uint_as_float(__float_as_uint(v - hi) & 0xFFFFE000u);
 }
 
-// Shared memory from the first 1024-byte boundary: kTfStages slots of [A hi | B hi | A lo | B lo]; then
-//   +0 full[3], +32 ready[3], +64 empty[3], +96 accumulator barrier, +104 tensor-memory base, +128 bias[64].
+// Shared memory from the first 1024-byte boundary: kTfStages slots of [x raw | Wd hi | Wd lo]; then
+//   +0 full[4], +32 ready[4], +64 empty[4], +96 accumulator barrier, +104 tensor-memory base, +128 bias[64].
 __global__ void __launch_bounds__(kTfThreads, 1)
 cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                       float* __restrict__ y, int batch) {
@@ -74,7 +91,7 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(ctl + 104)), "r"(64u)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(ctl + 104)), "r"(kTfTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -107,16 +124,15 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             ok = mbar_wait(ready0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a_hi = smem_u32(ring + s * kTfStageBytes), b_hi = a_hi + kTfABytes;
-            const uint32_t a_lo = a_hi + kTfABytes + kTfBBytes, b_lo = a_lo + kTfABytes;
-            const uint64_t dah = umma_desc_k_sw128(a_hi), dbh = umma_desc_k_sw128(b_hi);
-            const uint64_t dal = umma_desc_k_sw128(a_lo), dbl = umma_desc_k_sw128(b_lo);
+            const uint32_t b_hi = smem_u32(ring + s * kTfStageBytes + kTfABytes), b_lo = b_hi + kTfBBytes;
+            const uint64_t dbh = umma_desc_k_sw128(b_hi), dbl = umma_desc_k_sw128(b_lo);
+            const uint32_t a_hi = tmem_base + (uint32_t)(kTfN + 64 * s), a_lo = a_hi + 32u;
 #pragma unroll
-            for (int k = 0; k < kTfK / 8; ++k) {  // 8 fp32 = 32 bytes further along K inside the swizzled row
+            for (int k = 0; k < kTfK / 8; ++k) {  // 8 fp32 further along K: 8 columns of tensor memory, 32 bytes of a row
                 const uint64_t off = (uint64_t)(2 * k);
-                umma_tf32(tmem_base, dal + off, dbh + off, (kb | k) != 0 ? 1u : 0u);  // small terms first
-                umma_tf32(tmem_base, dah + off, dbl + off, 1u);
-                umma_tf32(tmem_base, dah + off, dbh + off, 1u);
+                umma_tf32_ts(tmem_base, a_lo + 8u * k, dbh + off, (kb | k) != 0 ? 1u : 0u);  // small terms first
+                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbl + off, 1u);
+                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbh + off, 1u);
             }
             umma_commit(empty0 + 8 * s);
         }
@@ -128,16 +144,39 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             const int s = kb % kTfStages;
             ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
-            const uint32_t hi_off = ring + s * kTfStageBytes, lo_off = hi_off + kTfABytes + kTfBBytes;
+            if (warp < 6) {
+                // x: this thread's batch row (tensor-memory lane), 8 chunks of 16 bytes un-permuted from the swizzle.
+                const int m = 32 * (warp & 3) + lane;
+                const uint32_t row_off = ring + s * kTfStageBytes + (uint32_t)m * 128u;
+                uint32_t hi[32], lo[32];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float4 v = *reinterpret_cast<const float4*>(smem_at(row_off + (uint32_t)((c ^ (m & 7)) << 4)));
+                    float h, l;
+                    split_tf32(v.x, h, l), hi[4 * c + 0] = __float_as_uint(h), lo[4 * c + 0] = __float_as_uint(l);
+                    split_tf32(v.y, h, l), hi[4 * c + 1] = __float_as_uint(h), lo[4 * c + 1] = __float_as_uint(l);
+                    split_tf32(v.z, h, l), hi[4 * c + 2] = __float_as_uint(h), lo[4 * c + 2] = __float_as_uint(l);
+                    split_tf32(v.w, h, l), hi[4 * c + 3] = __float_as_uint(h), lo[4 * c + 3] = __float_as_uint(l);
+                }
+                const uint32_t t_hi = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(kTfN + 64 * s);
+                tmem_st32(t_hi, hi);
+                tmem_st32(t_hi + 32u, lo);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            } else {
+                // Wd: element-wise, hi in place, lo beside it.
+                const uint32_t hi_off = ring + s * kTfStageBytes + kTfABytes, lo_off = hi_off + kTfBBytes;
 #pragma unroll 2
-            for (uint32_t e = wt * 16u; e < kTfABytes + kTfBBytes; e += 32u * kTfWorkerWarps * 16u) {
-                float4 v = *reinterpret_cast<const float4*>(smem_at(hi_off + e)), h, l;
-                split_tf32(v.x, h.x, l.x);
-                split_tf32(v.y, h.y, l.y);
-                split_tf32(v.z, h.z, l.z);
-                split_tf32(v.w, h.w, l.w);
-                *reinterpret_cast<float4*>(smem_at(hi_off + e)) = h;
-                *reinterpret_cast<float4*>(smem_at(lo_off + e)) = l;
+                for (uint32_t e = (uint32_t)(tid - 192) * 16u; e < kTfBBytes; e += 128u * 16u) {
+                    const float4 v = *reinterpret_cast<const float4*>(smem_at(hi_off + e));
+                    float4 h, l;
+                    split_tf32(v.x, h.x, l.x);
+                    split_tf32(v.y, h.y, l.y);
+                    split_tf32(v.z, h.z, l.z);
+                    split_tf32(v.w, h.w, l.w);
+                    *reinterpret_cast<float4*>(smem_at(hi_off + e)) = h;
+                    *reinterpret_cast<float4*>(smem_at(lo_off + e)) = l;
+                }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
             mbar_arrive(ready0 + 8 * s);
@@ -183,6 +222,6 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     __syncthreads();
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(64u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTfTmemCols) : "memory");
     }
 }
