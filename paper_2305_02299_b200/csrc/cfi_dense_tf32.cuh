@@ -15,12 +15,11 @@
 //
 // The layer keeps one dense fp32 copy of its weight, Wd[out_pad][in].  Per 32-column block of K:
 //   warp 0, one lane   TMA: a 128 x 32 box of x and a 64 x 32 box of Wd (fp32, 128-byte swizzle) into a ring slot;
-//   warps 2..5         split the x box: a thread reads its batch row from shared memory and writes hi and lo
-//                      straight into tensor memory (tcgen05.st), from where the MMA takes its A operand, so
-//                      x costs shared-memory bandwidth once instead of once per MMA;
-//   warps 6..9         split the Wd box in shared memory, hi in place and lo beside it (element-wise, so the
-//                      swizzled layout is untouched), and make the writes visible to the tensor core
-//                      (fence.proxy.async);
+//   warps 2..9         split the x box: a thread reads half of its batch row from shared memory and writes hi and
+//                      lo straight into tensor memory (tcgen05.st), from where the MMA takes its A operand, so
+//                      x costs shared-memory bandwidth once instead of once per MMA; the same warps split the
+//                      Wd box in shared memory, hi in place and lo beside it (element-wise, so the swizzled
+//                      layout is untouched), and make those writes visible to the tensor core (fence.proxy.async);
 //   warp 1, one lane   once all 256 splitting threads have arrived on the slot's "ready" barrier:
 //                      4 K-steps x 3 tcgen05.mma (kind::tf32, M = 128, N = 64, K = 8, A from tensor memory, B
 //                      from shared memory), then tcgen05.commit frees the slot;
@@ -49,14 +48,12 @@ __device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, u
 __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
     asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(
+            taddr),
         "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
 
@@ -144,30 +141,30 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             const int s = kb % kTfStages;
             ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
-            if (warp < 6) {
-                // x: this thread's batch row (tensor-memory lane), 8 chunks of 16 bytes un-permuted from the swizzle.
-                const int m = 32 * (warp & 3) + lane;
+            {
+                // x: this thread's batch row (tensor-memory lane) and half of its 32 columns: 4 chunks of 16 bytes,
+                // un-permuted from the swizzle, split and written straight to tensor memory.
+                const int m = 32 * (warp & 3) + lane, chalf = (warp - 2) >> 2;
                 const uint32_t row_off = ring + s * kTfStageBytes + (uint32_t)m * 128u;
-                uint32_t hi[32], lo[32];
+                uint32_t hi[16], lo[16];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const float4 v = *reinterpret_cast<const float4*>(smem_at(row_off + (uint32_t)((c ^ (m & 7)) << 4)));
+                for (int c = 0; c < 4; ++c) {
+                    const float4 v =
+                        *reinterpret_cast<const float4*>(smem_at(row_off + (uint32_t)(((4 * chalf + c) ^ (m & 7)) << 4)));
                     float h, l;
                     split_tf32(v.x, h, l), hi[4 * c + 0] = __float_as_uint(h), lo[4 * c + 0] = __float_as_uint(l);
                     split_tf32(v.y, h, l), hi[4 * c + 1] = __float_as_uint(h), lo[4 * c + 1] = __float_as_uint(l);
                     split_tf32(v.z, h, l), hi[4 * c + 2] = __float_as_uint(h), lo[4 * c + 2] = __float_as_uint(l);
                     split_tf32(v.w, h, l), hi[4 * c + 3] = __float_as_uint(h), lo[4 * c + 3] = __float_as_uint(l);
                 }
-                const uint32_t t_hi = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(kTfN + 64 * s);
-                tmem_st32(t_hi, hi);
-                tmem_st32(t_hi + 32u, lo);
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            } else {
-                // Wd: element-wise, hi in place, lo beside it.
+                const uint32_t t_hi =
+                    tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(kTfN + 64 * s + 16 * chalf);
+                tmem_st16(t_hi, hi);
+                tmem_st16(t_hi + 32u, lo);
+                // Wd: element-wise, hi in place, lo beside it (2 of its 512 16-byte pieces per thread).
                 const uint32_t hi_off = ring + s * kTfStageBytes + kTfABytes, lo_off = hi_off + kTfBBytes;
-#pragma unroll 2
-                for (uint32_t e = (uint32_t)(tid - 192) * 16u; e < kTfBBytes; e += 128u * 16u) {
+#pragma unroll
+                for (uint32_t e = (uint32_t)wt * 16u; e < kTfBBytes; e += 32u * kTfWorkerWarps * 16u) {
                     const float4 v = *reinterpret_cast<const float4*>(smem_at(hi_off + e));
                     float4 h, l;
                     split_tf32(v.x, h.x, l.x);
@@ -177,6 +174,8 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                     *reinterpret_cast<float4*>(smem_at(hi_off + e)) = h;
                     *reinterpret_cast<float4*>(smem_at(lo_off + e)) = l;
                 }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
             mbar_arrive(ready0 + 8 * s);

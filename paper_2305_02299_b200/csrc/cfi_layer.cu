@@ -820,7 +820,7 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
 }
 
 // Rates used to choose between the gather kernel and the split-TF32 dense kernel for fp32 layers (measured).
-constexpr double kDenseTf32SecondsPerBlock = 0.78e-6, kGatherTflops = 12.5;
+constexpr double kDenseTf32SecondsPerBlock = 0.57e-6, kGatherTflops = 12.5;
 
 int choose_variant(const cfi_layer* l, int batch) {
     if (batch <= 8) return CFI_VARIANT_SPLITK;
