@@ -377,16 +377,35 @@ def main():
             "roofline": {"bound": "alu", "achieved": achieved_tflops, "peak": fma_peak_tflops, "unit": "TFLOP/s",
                          "frac": achieved_tflops / fma_peak_tflops, "traffic": None,
                          "peak_source": f"{sm_count} SMs x {FMA_LANES_PER_SM} fp32 FMA lanes x 2 x {sm_max_mhz:.0f} MHz",
-                         "kernel": "cfi_batch_kernel<float>" if chosen == "batch" else f"cfi_{chosen}_kernel",
+                         "kernel": {"batch": "cfi_batch_kernel<float>", "dense_tc": "cfi_dense_tf32_kernel"}.get(
+                             chosen, f"cfi_{chosen}_kernel"),
+                         "note": "bound/peak are the sparse problem's own roofline (2*B*n_active*k FMAs on the fp32 FMA "
+                                 "pipes, the bound of the gather formulation); when the chosen kernel is the tensor-core "
+                                 "variant the dense flops it executes are given under tensor_*",
                          "hbm_achieved_gbs": hbm_gbs, "hbm_peak_gbs": peaks["hbm_gbs"],
                          "hbm_frac": hbm_gbs / peaks["hbm_gbs"], "hbm_peak_source": f"{peak_kind} copy bandwidth",
                          "algorithmic_bytes": rep.bytes_per_step, "algorithmic_flops": flops,
                          "weight_bytes_streamed_per_batch_tile": int(info.weight_bytes_batch)},
+            "variants_us": {},
             "e2e": {"value": e2e_value, "unit": "GFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "us_per_call": e2e_sec / e2e_steps * 1e6, "steps": e2e_steps, "api": "cfi_forward_host"},
             "gpu_launches": launches,
             "clocks": sampler.summary(),
         }
+    if rank == 0:
+        if chosen == "dense_tc":
+            dense = 3 * 2.0 * w.batch * w.out_features * w.in_features   # three TF32 MMAs per product
+            tf32_peak = peaks["bf16_tflops"] * 0.5                      # nominal TF32 : bf16 ratio on the measured bf16 peak
+            line["roofline"].update({"tensor_executed_tflops": dense / per_call / 1e12, "tensor_peak_tflops": tf32_peak,
+                                     "tensor_frac": dense / per_call / 1e12 / tf32_peak,
+                                     "tensor_peak_source": f"{peak_kind} bf16 matmul peak x 0.5 (nominal TF32:bf16)"})
+        if world == 1 and not args.no_extras:
+            for v in ("batch", "dense_tc"):
+                try:
+                    sv, _ = time_steps(rep, torch, 5000, 10, v)
+                    line["variants_us"][v] = sv / 5000 * 1e6
+                except Exception as exc:  # a variant that cannot run this shape
+                    line["variants_us"][v] = str(exc)
     rep.close()
 
     if rank == 0 and world == 1 and not args.no_extras:
