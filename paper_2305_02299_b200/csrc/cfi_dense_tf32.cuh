@@ -15,20 +15,23 @@
 //
 // The layer keeps one dense fp32 copy of its weight, Wd[out_pad][in].  Per 32-column block of K:
 //   warp 0, one lane   TMA: a 128 x 32 box of x and a 64 x 32 box of Wd (fp32, 128-byte swizzle) into a ring slot;
-//   warps 2..9         split the x box: a thread reads half of its batch row from shared memory and writes hi and
-//                      lo straight into tensor memory (tcgen05.st), from where the MMA takes its A operand, so
-//                      x costs shared-memory bandwidth once instead of once per MMA; the same warps split the
-//                      Wd box in shared memory, hi in place and lo beside it (element-wise, so the swizzled
-//                      layout is untouched), and make those writes visible to the tensor core (fence.proxy.async);
-//   warp 1, one lane   once all 256 splitting threads have arrived on the slot's "ready" barrier:
+//   warps 2..17        four groups of four warps; group g takes the blocks kb = g (mod 4), so four blocks are being
+//                      split at once.  A thread reads its batch row of the x box from shared memory and writes
+//                      hi and lo straight into tensor memory (tcgen05.st), from where the MMA takes its A
+//                      operand, so x costs shared-memory bandwidth once instead of once per MMA; the group also
+//                      splits the Wd box in shared memory, hi in place and lo beside it (element-wise, so the
+//                      swizzled layout is untouched), and makes those writes visible to the tensor core
+//                      (fence.proxy.async);
+//   warp 1, one lane   once the group's 128 threads have arrived on the slot's "ready" barrier:
 //                      4 K-steps x 3 tcgen05.mma (kind::tf32, M = 128, N = 64, K = 8, A from tensor memory, B
 //                      from shared memory), then tcgen05.commit frees the slot;
-// and after the last block warps 2..9 run the epilogue: tcgen05.ld, bias, activation, y tile through shared
+// and after the last block warps 2..17 run the epilogue: tcgen05.ld, bias, activation, y tile through shared
 // memory, 256-byte runs per batch row.  Tensor memory: columns 0..63 accumulator, then per slot 32 columns of
 // x_hi and 32 of x_lo.  All mbarrier waits are bounded (status code 2), as in the bf16 kernel.
 
 constexpr int kTfM = 128, kTfN = 64, kTfK = 32, kTfStages = 4;
-constexpr int kTfWorkerWarps = 8, kTfThreads = 64 + 32 * kTfWorkerWarps;
+constexpr int kTfGroups = 4;  // groups of four worker warps; group g splits the K blocks kb with kb % kTfGroups == g
+constexpr int kTfWorkerWarps = 4 * kTfGroups, kTfThreads = 64 + 32 * kTfWorkerWarps;
 constexpr uint32_t kTfABytes = kTfM * kTfK * 4, kTfBBytes = kTfN * kTfK * 4;   // 16 KB, 8 KB
 constexpr uint32_t kTfStageBytes = kTfABytes + 2 * kTfBBytes;                  // x raw | Wd hi | Wd lo: 32 KB
 constexpr uint32_t kTfTmemCols = 512;                                          // 64 + 4 * 64 = 320, next power of two
@@ -81,7 +84,7 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     if (tid == 0) {
         for (int s = 0; s < kTfStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
-            mbar_init(ready0 + 8 * s, 32 * kTfWorkerWarps);
+            mbar_init(ready0 + 8 * s, 128);
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum, 1);
@@ -136,35 +139,39 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         if (ok) umma_commit(accum);
     } else if (warp >= 2) {
         // ---------------------------------------------------------------- split, then epilogue
-        const int wt = tid - 64;  // 0..255
-        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+        const int wt = tid - 64;            // 0 .. 32 * kTfWorkerWarps - 1
+        const int group = (warp - 2) >> 2;  // the group's four warps cover the four lane quarters of tensor memory
+        const int gt = wt & 127;            // thread within the group
+        for (int kb = group; kb < k_blocks && ok; kb += kTfGroups) {
             const int s = kb % kTfStages;
             ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
             {
-                // x: this thread's batch row (tensor-memory lane) and half of its 32 columns: 4 chunks of 16 bytes,
-                // un-permuted from the swizzle, split and written straight to tensor memory.
-                const int m = 32 * (warp & 3) + lane, chalf = (warp - 2) >> 2;
+                // x: this thread's batch row (tensor-memory lane): 8 chunks of 16 bytes, un-permuted from the
+                // swizzle, split and written straight to tensor memory.
+                const int m = 32 * (warp & 3) + lane;
                 const uint32_t row_off = ring + s * kTfStageBytes + (uint32_t)m * 128u;
-                uint32_t hi[16], lo[16];
+                const uint32_t t_hi = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(kTfN + 64 * s);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const float4 v =
-                        *reinterpret_cast<const float4*>(smem_at(row_off + (uint32_t)(((4 * chalf + c) ^ (m & 7)) << 4)));
-                    float h, l;
-                    split_tf32(v.x, h, l), hi[4 * c + 0] = __float_as_uint(h), lo[4 * c + 0] = __float_as_uint(l);
-                    split_tf32(v.y, h, l), hi[4 * c + 1] = __float_as_uint(h), lo[4 * c + 1] = __float_as_uint(l);
-                    split_tf32(v.z, h, l), hi[4 * c + 2] = __float_as_uint(h), lo[4 * c + 2] = __float_as_uint(l);
-                    split_tf32(v.w, h, l), hi[4 * c + 3] = __float_as_uint(h), lo[4 * c + 3] = __float_as_uint(l);
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t hi[16], lo[16];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const float4 v =
+                            *reinterpret_cast<const float4*>(smem_at(row_off + (uint32_t)(((4 * half + c) ^ (m & 7)) << 4)));
+                        float h, l;
+                        split_tf32(v.x, h, l), hi[4 * c + 0] = __float_as_uint(h), lo[4 * c + 0] = __float_as_uint(l);
+                        split_tf32(v.y, h, l), hi[4 * c + 1] = __float_as_uint(h), lo[4 * c + 1] = __float_as_uint(l);
+                        split_tf32(v.z, h, l), hi[4 * c + 2] = __float_as_uint(h), lo[4 * c + 2] = __float_as_uint(l);
+                        split_tf32(v.w, h, l), hi[4 * c + 3] = __float_as_uint(h), lo[4 * c + 3] = __float_as_uint(l);
+                    }
+                    tmem_st16(t_hi + 16u * half, hi);
+                    tmem_st16(t_hi + 32u + 16u * half, lo);
                 }
-                const uint32_t t_hi =
-                    tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(kTfN + 64 * s + 16 * chalf);
-                tmem_st16(t_hi, hi);
-                tmem_st16(t_hi + 32u, lo);
-                // Wd: element-wise, hi in place, lo beside it (2 of its 512 16-byte pieces per thread).
+                // Wd: element-wise, hi in place, lo beside it (4 of its 512 16-byte pieces per thread).
                 const uint32_t hi_off = ring + s * kTfStageBytes + kTfABytes, lo_off = hi_off + kTfBBytes;
 #pragma unroll
-                for (uint32_t e = (uint32_t)wt * 16u; e < kTfBBytes; e += 32u * kTfWorkerWarps * 16u) {
+                for (uint32_t e = (uint32_t)gt * 16u; e < kTfBBytes; e += 128u * 16u) {
                     const float4 v = *reinterpret_cast<const float4*>(smem_at(hi_off + e));
                     float4 h, l;
                     split_tf32(v.x, h.x, l.x);
@@ -180,34 +187,31 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the MMA's reads
             mbar_arrive(ready0 + 8 * s);
         }
+        ok = __all_sync(0xffffffffu, ok);
         if (ok) ok = mbar_wait(accum, 0u, kTcSpinLimit);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int q = warp & 3;            // tensor-memory lanes 32 q .. 32 q + 31
-        const int half = (warp - 2) >> 2;  // two warps share a lane quarter and split the 64 columns
+        const int q = warp & 3;  // tensor-memory lanes 32 q .. 32 q + 31; the group number picks 16 of the 64 columns
         const int row = 32 * q + lane;
         if (ok) {
             // y tile in shared memory: 128 rows x 256 bytes (64 fp32), 16-byte chunks permuted by chunk ^ (row & 15).
-            uint32_t v[2][16];
-            tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * half), v[0]);
-            tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * half + 16), v[1]);
+            uint32_t v[16];
+            tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(16 * group), v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int e4 = 0; e4 < 4; ++e4) {
-                    const int col = 32 * half + 16 * h + 4 * e4;
-                    const float4 bv = *reinterpret_cast<const float4*>(bias_s + col);
-                    float4 r;
-                    r.x = activate(__uint_as_float(v[h][4 * e4 + 0]) + bv.x, L.act);
-                    r.y = activate(__uint_as_float(v[h][4 * e4 + 1]) + bv.y, L.act);
-                    r.z = activate(__uint_as_float(v[h][4 * e4 + 2]) + bv.z, L.act);
-                    r.w = activate(__uint_as_float(v[h][4 * e4 + 3]) + bv.w, L.act);
-                    *reinterpret_cast<float4*>(smem_at(ring + row * 256 + (((col >> 2) ^ (row & 15)) << 4))) = r;
-                }
+            for (int e4 = 0; e4 < 4; ++e4) {
+                const int col = 16 * group + 4 * e4;
+                const float4 bv = *reinterpret_cast<const float4*>(bias_s + col);
+                float4 r;
+                r.x = activate(__uint_as_float(v[4 * e4 + 0]) + bv.x, L.act);
+                r.y = activate(__uint_as_float(v[4 * e4 + 1]) + bv.y, L.act);
+                r.z = activate(__uint_as_float(v[4 * e4 + 2]) + bv.z, L.act);
+                r.w = activate(__uint_as_float(v[4 * e4 + 3]) + bv.w, L.act);
+                *reinterpret_cast<float4*>(smem_at(ring + row * 256 + (((col >> 2) ^ (row & 15)) << 4))) = r;
+            }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(32 * kTfWorkerWarps) : "memory");
         if (ok) {
-            for (int r = wt >> 4; r < kTfM; r += 2 * kTfWorkerWarps) {  // 16 threads per row, 16 rows per pass
+            for (int r = wt >> 4; r < kTfM; r += 2 * kTfWorkerWarps) {  // 16 threads per row
                 const int ch = wt & 15, m = m0 + r, n = n0 + 4 * ch;
                 if (m < batch && n < L.out) {
                     const float4 val = *reinterpret_cast<const float4*>(smem_at(ring + r * 256 + ((ch ^ (r & 15)) << 4)));
