@@ -187,6 +187,12 @@ __device__ __forceinline__ void gather_fma(float (&acc)[BT], const float* xs, in
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Ask for `bytes` (a multiple of 16, from a 16-byte aligned address) to be brought into L2.  Costs one
+// instruction and no registers; later loads of the range then find it on chip.
+__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 // U = 16-byte vector pairs (weights + indices) in flight per lane: 4, or 8 for long rows so that a whole
 // row is requested at once.
 template <typename VT, int BT, int G, int U>
@@ -205,8 +211,13 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
     int o = blockIdx.x * (groups * rows_per_group) + g;
     int r = o < L.out ? (dense_rows ? o : L.slot[o]) : -1;
 
-    // The first vectors of the first row depend neither on x nor on the kernel before this one: they are
-    // requested first, so the weight stream is in flight while x is awaited and staged.
+    // The first row's weights and indices depend neither on x nor on the kernel before this one.  The whole row
+    // is asked into L2 by one lane, and its first vectors are requested into registers, before anything else,
+    // so the weight stream is in flight while x is awaited and staged.
+    if (lg == 0 && r >= 0) {
+        prefetch_l2(reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp, (uint32_t)(L.kp * sizeof(VT)));
+        prefetch_l2(L.indices + (size_t)r * L.kp, (uint32_t)(L.kp * 4));
+    }
     CK ck[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -261,6 +272,10 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
         if (more) {
             o += groups;
             r = o < L.out ? (dense_rows ? o : L.slot[o]) : -1;
+            if (lg == 0 && r >= 0) {
+                prefetch_l2(reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp, (uint32_t)(L.kp * sizeof(VT)));
+                prefetch_l2(L.indices + (size_t)r * L.kp, (uint32_t)(L.kp * 4));
+            }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int v = lg + u * G;
