@@ -608,11 +608,12 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     while (s.bt > 1 && (size_t)(l->d.in + 1) * s.bt * 4 > (size_t)l->smem_optin) s.bt >>= 1;
     const int nvec = l->d.kp / vec_of(l->dtype);
     s.g = splitk_lanes_per_row(nvec);
-    s.u = nvec > s.g * 4 ? 8 : 4;  // long rows: request the whole row (up to 8 vectors per lane) at once
-    // Enough CTAs to cover the SMs several times over (each CTA stages x for itself, and many small CTAs
-    // keep more independent requests in flight), but not more x staging than that needs.
+    s.u = 4;  // with the row already on its way into L2, four vector pairs per lane in registers are enough
+    // Every CTA stages x for itself (from L2), so larger CTAs spend less of the L2 bandwidth on x; a group takes
+    // more than one row only when the grid would otherwise exceed eight CTAs per SM (rows of a group run one
+    // after the other, which costs latency).
     const int64_t lanes = (int64_t)l->d.out * s.g;
-    s.threads = lanes >= (int64_t)l->sm_count * 8 * 256 ? 256 : 128;
+    s.threads = lanes >= (int64_t)l->sm_count * 256 ? 256 : 128;
     const int groups = s.threads / s.g;
     const int ctas_one_row_each = (l->d.out + groups - 1) / groups;
     const int target = l->sm_count * 8;
