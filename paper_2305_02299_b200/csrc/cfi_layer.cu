@@ -193,14 +193,15 @@ __device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
-// U = 16-byte vector pairs (weights + indices) in flight per lane: 4, or 8 for long rows so that a whole
-// row is requested at once.
-template <typename VT, int BT, int G, int U>
+// A lane keeps U = 4 16-byte vector pairs (weights + indices) in flight in registers; the rest of the row is
+// on its way into L2.  XS = loads of x in flight per thread while staging (8 where few threads stage a long x).
+template <typename VT, int BT, int G, int XS>
 __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch,
                                   int rows_per_group) {
     extern __shared__ __align__(16) float xs_f32[];  // [(in + 1)][BT]
     float* xs = xs_f32;
     using CK = Chunk<VT>;
+    constexpr int U = 4;
     pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int b0 = blockIdx.y * BT;
@@ -227,18 +228,32 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
     float bias = o < L.out ? L.bias[o] : 0.0f;
 
     pdl_wait();
-    // Stage the CTA's x rows, widened to fp32, transposed to [column][b].
+    // Stage the CTA's x rows, widened to fp32, transposed to [column][b].  Loads are issued kXStage at a time
+    // before their stores, so staging costs a few memory round trips, not one per element.
+    constexpr int kXStage = XS;
     if (BT == 1 && sizeof(VT) == 4 && (L.in & 3) == 0) {
         const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(x) + (size_t)b0 * L.in);
-        for (int c = tid; c < (L.in >> 2); c += nthr) reinterpret_cast<float4*>(xs)[c] = __ldg(src + c);
+        const int n4 = L.in >> 2;
+        for (int c0 = tid; c0 < n4; c0 += nthr * kXStage) {
+            float4 v[kXStage];
+#pragma unroll
+            for (int u = 0; u < kXStage; ++u)
+                if (c0 + u * nthr < n4) v[u] = __ldg(src + c0 + u * nthr);
+#pragma unroll
+            for (int u = 0; u < kXStage; ++u)
+                if (c0 + u * nthr < n4) reinterpret_cast<float4*>(xs)[c0 + u * nthr] = v[u];
+        }
     } else {
 #pragma unroll
         for (int b = 0; b < BT; ++b) {
-            if (b < nb) {
-                const VT* xr = x + (size_t)(b0 + b) * L.in;
-                for (int c = tid; c < L.in; c += nthr) xs[(size_t)c * BT + b] = to_f32(xr[c]);
-            } else {
-                for (int c = tid; c < L.in; c += nthr) xs[(size_t)c * BT + b] = 0.0f;
+            const VT* xr = x + (size_t)(b0 + b) * L.in;
+            for (int c0 = tid; c0 < L.in; c0 += nthr * kXStage) {
+                float v[kXStage];
+#pragma unroll
+                for (int u = 0; u < kXStage; ++u) v[u] = (b < nb && c0 + u * nthr < L.in) ? to_f32(xr[c0 + u * nthr]) : 0.0f;
+#pragma unroll
+                for (int u = 0; u < kXStage; ++u)
+                    if (c0 + u * nthr < L.in) xs[(size_t)(c0 + u * nthr) * BT + b] = v[u];
             }
         }
     }
@@ -589,7 +604,7 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 // ------------------------------------------------------------------------------------------------
 // host: launch shapes
 // ------------------------------------------------------------------------------------------------
-struct SplitkShape { int bt, g, u, threads, rows_per_group, grid_x, grid_y; size_t smem; };
+struct SplitkShape { int bt, g, xs, threads, rows_per_group, grid_x, grid_y; size_t smem; };
 struct BatchShape { int warps, rph, threads, rt, grid_x, grid_y; size_t smem; bool ok; };
 
 int vec_of(int dtype) { return dtype == CFI_BF16 ? 8 : 4; }
@@ -608,7 +623,6 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     while (s.bt > 1 && (size_t)(l->d.in + 1) * s.bt * 4 > (size_t)l->smem_optin) s.bt >>= 1;
     const int nvec = l->d.kp / vec_of(l->dtype);
     s.g = splitk_lanes_per_row(nvec);
-    s.u = 4;  // with the row already on its way into L2, four vector pairs per lane in registers are enough
     // Every CTA stages x for itself (from L2), so larger CTAs spend less of the L2 bandwidth on x; a group takes
     // more than one row only when the grid would otherwise exceed eight CTAs per SM (rows of a group run one
     // after the other, which costs latency).
@@ -618,6 +632,9 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     const int ctas_one_row_each = (l->d.out + groups - 1) / groups;
     const int target = l->sm_count * 8;
     s.rows_per_group = std::max(1, (ctas_one_row_each + target - 1) / target);
+    // x loads in flight per staging thread: 8 when 4 would need more than one round and the grid is small enough
+    // that the extra registers do not cost a wave.
+    s.xs = (l->d.in > 16 * s.threads && s.threads == 128) ? 8 : 4;
     s.grid_x = (l->d.out + groups * s.rows_per_group - 1) / (groups * s.rows_per_group);
     s.grid_y = (batch + s.bt - 1) / s.bt;
     s.smem = (size_t)(l->d.in + 1) * s.bt * 4;
@@ -703,7 +720,7 @@ cfi_status_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t
 template <typename VT, int BT, int G>
 cfi_status_t launch_splitk_g(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
                              cudaStream_t st) {
-    if (s.u == 8) {
+    if (s.xs == 8) {
         if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, BT, G, 8>>(s.smem, l->device)) return e;
         return launch_pdl(cfi_splitk_kernel<VT, BT, G, 8>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch,
                           s.rows_per_group);
