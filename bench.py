@@ -375,7 +375,10 @@ def main():
                              f"{rep.total_bytes / 1e6:.0f} MB vs L2 {l2 / 1e6:.0f} MB",
                        "timing": "CUDA-graph replays between CUDA events on the launching stream"},
             "roofline": {"bound": "alu", "achieved": achieved_tflops, "peak": fma_peak_tflops, "unit": "TFLOP/s",
-                         "frac": achieved_tflops / fma_peak_tflops, "traffic": None,
+                         "frac": achieved_tflops / fma_peak_tflops,
+                         # dram__bytes_read.sum + dram__bytes_write.sum of one launch (ncu capture summarised under
+                         # profiles/); only valid for the kernel and workload it was taken on
+                         "traffic": 10.27e6 if (chosen == "dense_tc" and w.name == "c2") else None,
                          "peak_source": f"{sm_count} SMs x {FMA_LANES_PER_SM} fp32 FMA lanes x 2 x {sm_max_mhz:.0f} MHz",
                          "kernel": {"batch": "cfi_batch_kernel<float>", "dense_tc": "cfi_dense_tf32_kernel"}.get(
                              chosen, f"cfi_{chosen}_kernel"),
