@@ -244,16 +244,31 @@ __global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
                 if (c0 + u * nthr < n4) reinterpret_cast<float4*>(xs)[c0 + u * nthr] = v[u];
         }
     } else {
+        // A thread takes kCols columns at a time: one load per column and batch row (each coalesced across the
+        // warp), all issued before the first store, then each column's BT values go to shared memory side by side.
+        constexpr int kCols = BT >= 8 ? 4 : BT >= 4 ? 4 : 8;
+        for (int c0 = tid; c0 < L.in; c0 += nthr * kCols) {
+            float v[kCols][BT];
 #pragma unroll
-        for (int b = 0; b < BT; ++b) {
-            const VT* xr = x + (size_t)(b0 + b) * L.in;
-            for (int c0 = tid; c0 < L.in; c0 += nthr * kXStage) {
-                float v[kXStage];
+            for (int u = 0; u < kCols; ++u)
 #pragma unroll
-                for (int u = 0; u < kXStage; ++u) v[u] = (b < nb && c0 + u * nthr < L.in) ? to_f32(xr[c0 + u * nthr]) : 0.0f;
+                for (int b = 0; b < BT; ++b)
+                    v[u][b] = (b < nb && c0 + u * nthr < L.in) ? to_f32(x[(size_t)(b0 + b) * L.in + c0 + u * nthr]) : 0.0f;
 #pragma unroll
-                for (int u = 0; u < kXStage; ++u)
-                    if (c0 + u * nthr < L.in) xs[(size_t)(c0 + u * nthr) * BT + b] = v[u];
+            for (int u = 0; u < kCols; ++u) {
+                const int c = c0 + u * nthr;
+                if (c < L.in) {
+                    if constexpr (BT == 1) {
+                        xs[c] = v[u][0];
+                    } else if constexpr (BT == 2) {
+                        *reinterpret_cast<float2*>(xs + (size_t)c * 2) = make_float2(v[u][0], v[u][1]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < BT / 4; ++q)
+                            *reinterpret_cast<float4*>(xs + (size_t)c * BT + 4 * q) =
+                                make_float4(v[u][4 * q], v[u][4 * q + 1], v[u][4 * q + 2], v[u][4 * q + 3]);
+                    }
+                }
             }
         }
     }
@@ -623,14 +638,17 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     while (s.bt > 1 && (size_t)(l->d.in + 1) * s.bt * 4 > (size_t)l->smem_optin) s.bt >>= 1;
     const int nvec = l->d.kp / vec_of(l->dtype);
     s.g = splitk_lanes_per_row(nvec);
-    // Every CTA stages x for itself (from L2), so larger CTAs spend less of the L2 bandwidth on x; a group takes
-    // more than one row only when the grid would otherwise exceed eight CTAs per SM (rows of a group run one
-    // after the other, which costs latency).
+    // Every CTA stages x for itself (from L2), so larger CTAs spend less of the L2 bandwidth on x.  The staged x
+    // also limits how many CTAs fit an SM; the grid is sized to one wave of what fits (at most eight CTAs per
+    // SM), with several rows per group when needed (rows of a group run one after the other).
+    s.smem = (size_t)(l->d.in + 1) * s.bt * 4;
+    const int fit = (int)std::max<size_t>(1, std::min<size_t>(8, ((size_t)227 * 1024) / (s.smem + 1024)));
     const int64_t lanes = (int64_t)l->d.out * s.g;
     s.threads = lanes >= (int64_t)l->sm_count * 256 ? 256 : 128;
+    if (fit <= 2 && lanes >= (int64_t)l->sm_count * 512) s.threads = 512;
     const int groups = s.threads / s.g;
     const int ctas_one_row_each = (l->d.out + groups - 1) / groups;
-    const int target = l->sm_count * 8;
+    const int target = l->sm_count * fit;
     s.rows_per_group = std::max(1, (ctas_one_row_each + target - 1) / target);
     // x loads in flight per staging thread: 8 when 4 would need more than one round and the grid is small enough
     // that the extra registers do not cost a wave.
@@ -856,7 +874,9 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
 constexpr double kDenseTf32SecondsPerBlock = 0.57e-6, kGatherTflops = 12.5;
 
 int choose_variant(const cfi_layer* l, int batch) {
-    if (batch <= 8) return CFI_VARIANT_SPLITK;
+    // Up to three batch tiles of 8 the split-k kernel (weights re-read from L2 per tile) beats the 64-wide tiles of
+    // the batch kernel, which would be mostly empty.
+    if (batch <= 24) return CFI_VARIANT_SPLITK;
     // bf16 at large batch: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
     // (10 TFLOP/s effective for the gather against several hundred dense); below a full 128-row tile it does not pay.
     if (l->tc_ok && batch >= 96) {
