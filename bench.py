@@ -340,22 +340,16 @@ def main():
     rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), rank=rank)
     sampler = ClockSampler(local)
     sec, launches = time_steps(rep, torch, args.steps, args.warmup, args.variant, barrier=barrier, sampler=sampler)
-    if dist:
-        t = torch.tensor([sec], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        sec = float(t.item())
+    sec = max_over_ranks(sec, dist, "cuda")
     flops = algorithmic_flops(w, rep.n_active)
     per_call = sec / args.steps
-    value = flops * world / per_call / 1e9
+    value = whole_job_value(flops, world, per_call)
 
     # End to end through the host-buffer entry point (each rank on its own GPU).
     e2e_steps = int(min(args.steps, 2000))
     e2e_sec, h2d, d2h = time_e2e(rep, torch, e2e_steps, 5)
-    if dist:
-        t = torch.tensor([e2e_sec], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_sec = float(t.item())
-    e2e_value = flops * world / (e2e_sec / e2e_steps) / 1e9
+    e2e_sec = max_over_ranks(e2e_sec, dist, "cuda")
+    e2e_value = whole_job_value(flops, world, e2e_sec / e2e_steps)
 
     line = None
     if rank == 0:
@@ -423,6 +417,21 @@ def main():
         print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
+
+
+def max_over_ranks(seconds: float, dist, device) -> float:
+    """Device time of a multi-rank run: the slowest rank's (all-reduce MAX over the process group)."""
+    if dist is None:
+        return seconds
+    import torch
+    t = torch.tensor([seconds], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_rank_step: float, world: int, seconds_per_step: float) -> float:
+    """GFLOP/s of all ranks together: every rank runs the same workload on its own batches (weak scaling)."""
+    return flops_per_rank_step * world / seconds_per_step / 1e9
 
 
 def _time_torch(fn, torch, iters=200):

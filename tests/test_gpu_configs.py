@@ -44,3 +44,43 @@ def test_vit_mlp_block_bf16_slice():
         assert scaled_error(y, y_ref, S) <= TOL["bf16"]
         dl.close()
         cur = oracle.round_bf16(y_ref.astype(np.float32))
+
+
+def test_vit_mlp_block_bf16_full_size_sampled():
+    """The bf16 MLP block at the full 50,432 rows, in the launch configuration the benchmark times (variant
+    auto, i.e. the tensor-core kernel): all outputs of 48 sampled batch rows per layer against the oracle."""
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    s = inputs.StackWorkload(blocks=1)
+    Ls, specs = s.layers(seed=0), s.layer_specs()
+    rng = np.random.default_rng(0)
+    rows = np.sort(rng.choice(s.batch, size=48, replace=False))
+    rows[0], rows[-1] = 0, s.batch - 1                      # first row, and the last row of the ragged last tile
+    cur = oracle.round_bf16(s.x(seed=0))
+    for L, sp in zip(Ls, specs):
+        dl = device_layer(L, "bf16", sp[4])
+        assert cfi.cfi_choose_variant(dl, s.batch) == 4
+        x_d = torch.from_numpy(cur).to("cuda", torch.bfloat16)
+        y_d = torch.empty((s.batch, sp[1]), device="cuda", dtype=torch.bfloat16)
+        cfi.cfi_forward(dl, x_d, y_d, s.batch)
+        torch.cuda.synchronize()
+        assert cfi.cfi_device_status(dl) == 0
+        y_ref, S = oracle_layer(L, cur[rows], "bf16", sp[4])
+        y = y_d[torch.from_numpy(rows).cuda()].double().cpu().numpy()
+        assert scaled_error(y, y_ref, S) <= TOL["bf16"]
+        dl.close()
+        cur = y_d.float().cpu().numpy()                      # the device's own output feeds the next layer
+
+
+def test_headline_workload_full_size_in_bench_configuration():
+    """c2 exactly as bench.py runs it (variant auto through cfi_forward), every output against the oracle, and
+    the gather and tensor-core variants against each other."""
+    w = W["c2"]
+    L, x = w.layer(), w.x()
+    y_ref, S = oracle_layer(L, x)
+    dl = device_layer(L)
+    ys = {v: run_device(dl, x, "f32", v) for v in ("auto", "batch", "dense_tc")}
+    dl.close()
+    for v, y in ys.items():
+        assert scaled_error(y, y_ref, S) <= 1e-5, v
+    assert np.max(np.abs(ys["batch"] - ys["dense_tc"]) / S) <= 2e-6
