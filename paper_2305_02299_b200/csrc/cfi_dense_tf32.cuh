@@ -32,20 +32,27 @@
 constexpr int kTfM = 128, kTfN = 64, kTfK = 32, kTfStages = 4;
 constexpr int kTfGroups = 4;  // groups of four worker warps; group g splits the K blocks kb with kb % kTfGroups == g
 constexpr int kTfWorkerWarps = 4 * kTfGroups, kTfThreads = 64 + 32 * kTfWorkerWarps;
+// A ring slot is always split by the same group, so that one phase bit per barrier is enough: a group that ran a
+// whole phase ahead on another group's slot would pass its wait early.
+static_assert(kTfStages == kTfGroups, "slot s belongs to group s");
 constexpr uint32_t kTfABytes = kTfM * kTfK * 4, kTfBBytes = kTfN * kTfK * 4;   // 16 KB, 8 KB
 constexpr uint32_t kTfStageBytes = kTfABytes + 2 * kTfBBytes;                  // x raw | Wd hi | Wd lo: 32 KB
-constexpr uint32_t kTfTmemCols = 512;                                          // 64 + 4 * 64 = 320, next power of two
+constexpr uint32_t kTfAccCols = 2 * kTfN;                                      // x_hi w_hi + x_lo w_hi | x_hi w_lo
+constexpr uint32_t kTfTmemCols = 512;                                          // 128 + 4 * 64 = 384, next power of two
 constexpr size_t kTfSmemBytes = 1024 + kTfStages * kTfStageBytes + 1024;
 
-// fp32 accumulate, tf32 x tf32, both K-major, N = 64, M = 128.
-constexpr uint32_t kTfInstrDesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTfN >> 3) << 17) | ((uint32_t)(kTfM >> 4) << 24);
+// fp32 accumulate, tf32 x tf32, both K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t tf_instr_desc(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTfM >> 4) << 24);
+}
 
 // A operand from tensor memory (row m in lane m, 32-bit elements in consecutive columns), B from shared memory.
-__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t accumulate) {
+__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
-        "r"(tmem_a), "l"(desc_b), "r"(kTfInstrDesc), "r"(accumulate), "r"(0u)
+        "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u)
         : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
@@ -124,15 +131,17 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             ok = mbar_wait(ready0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t b_hi = smem_u32(ring + s * kTfStageBytes + kTfABytes), b_lo = b_hi + kTfBBytes;
-            const uint64_t dbh = umma_desc_k_sw128(b_hi), dbl = umma_desc_k_sw128(b_lo);
-            const uint32_t a_hi = tmem_base + (uint32_t)(kTfN + 64 * s), a_lo = a_hi + 32u;
+            const uint32_t b_hi = smem_u32(ring + s * kTfStageBytes + kTfABytes);  // Wd lo follows at + kTfBBytes
+            const uint64_t dbh = umma_desc_k_sw128(b_hi);
+            const uint32_t a_hi = tmem_base + kTfAccCols + (uint32_t)(64 * s), a_lo = a_hi + 32u;
 #pragma unroll
             for (int k = 0; k < kTfK / 8; ++k) {  // 8 fp32 further along K: 8 columns of tensor memory, 32 bytes of a row
                 const uint64_t off = (uint64_t)(2 * k);
-                umma_tf32_ts(tmem_base, a_lo + 8u * k, dbh + off, (kb | k) != 0 ? 1u : 0u);  // small terms first
-                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbl + off, 1u);
-                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbh + off, 1u);
+                // Wd lo lies right behind Wd hi, so the two boxes read as one K-major operand of 128 rows: one MMA
+                // of N = 128 gives x_hi w_hi in columns 0..63 and x_hi w_lo in columns 64..127; a second of N = 64
+                // adds x_lo w_hi to the first half.  (An MMA of this size costs about the same whatever its N.)
+                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbh + off, tf_instr_desc(2 * kTfN), (kb | k) != 0 ? 1u : 0u);
+                umma_tf32_ts(tmem_base, a_lo + 8u * k, dbh + off, tf_instr_desc(kTfN), 1u);
             }
             umma_commit(empty0 + 8 * s);
         }
@@ -151,7 +160,7 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                 // swizzle, split and written straight to tensor memory.
                 const int m = 32 * (warp & 3) + lane;
                 const uint32_t row_off = ring + s * kTfStageBytes + (uint32_t)m * 128u;
-                const uint32_t t_hi = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(kTfN + 64 * s);
+                const uint32_t t_hi = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + kTfAccCols + (uint32_t)(64 * s);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     uint32_t hi[16], lo[16];
@@ -194,9 +203,13 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         const int row = 32 * q + lane;
         if (ok) {
             // y tile in shared memory: 128 rows x 256 bytes (64 fp32), 16-byte chunks permuted by chunk ^ (row & 15).
-            uint32_t v[16];
-            tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(16 * group), v);
+            uint32_t v[16], v1[16];
+            const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(16 * group);
+            tmem_ld16(t_acc, v);
+            tmem_ld16(t_acc + kTfN, v1);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(v1[e]));
 #pragma unroll
             for (int e4 = 0; e4 < 4; ++e4) {
                 const int col = 16 * group + 4 * e4;
