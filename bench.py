@@ -391,7 +391,7 @@ def main():
         }
     if rank == 0:
         if chosen == "dense_tc":
-            dense = 3 * 2.0 * w.batch * w.out_features * w.in_features   # three TF32 MMAs per product
+            dense = 3 * 2.0 * w.batch * w.out_features * w.in_features   # three TF32 products per fp32 product
             tf32_peak = peaks["bf16_tflops"] * 0.5                      # nominal TF32 : bf16 ratio on the measured bf16 peak
             line["roofline"].update({"tensor_executed_tflops": dense / per_call / 1e12, "tensor_peak_tflops": tf32_peak,
                                      "tensor_frac": dense / per_call / 1e12 / tf32_peak,
@@ -413,6 +413,8 @@ def main():
                                 "sample": f"whole workload ({cb['rows']} batch rows), median of {cb['calls']} calls"}
         line["context"] = context_leg(w, torch)
         line["stack_c5"] = stack_leg(cfi, torch, peaks, sm_count)
+        line["batch2048"] = batch2048_leg(W, cfi, torch, l2, peaks, sm_count)
+        line["stack_batch1"] = stack_batch1_leg(cfi, torch, l2, peaks)
     if rank == 0:
         print(json.dumps(line))
     if dist:
@@ -486,6 +488,75 @@ def stack_leg(cfi, torch, peaks, sm_count, rows=None, blocks=12):
             "effective_tflops": flops / sec / 1e12, "fma_frac": flops / sec / 1e12 / fma_peak,
             "algorithmic_bytes": bytes_, "hbm_frac": bytes_ / sec / 1e9 / peaks["hbm_gbs"],
             "l2": "activations of one layer (388 MB) exceed L2"}
+
+
+def batch2048_leg(W, cfi, torch, l2, peaks, sm_count):
+    """The headline layer at batch 2048, the largest batch of the paper's GPU figures (appendix, condensed
+    GPU benchmarks).  Cold: rotating replicas larger than L2."""
+    import dataclasses
+    w = dataclasses.replace(W["c2"], name="c2_b2048", batch=2048)
+    rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), max_replicas=16)
+    steps = 2000
+    out = {"batch": w.batch}
+    for v in ("auto", "batch"):
+        sec, _ = time_steps(rep, torch, steps, 10, v)
+        out[f"us_per_call_{v}"] = sec / steps * 1e6
+    flops = algorithmic_flops(w, rep.n_active)
+    fma_peak = sm_count * FMA_LANES_PER_SM * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+    out["effective_tflops"] = flops / (out["us_per_call_auto"] * 1e-6) / 1e12
+    out["fma_frac"] = out["effective_tflops"] / fma_peak
+    out["variant"] = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
+    rep.close()
+    return out
+
+
+def stack_batch1_leg(cfi, torch, l2, peaks, blocks=12, replicas=4):
+    """Online inference through a whole fp32 MLP stack at batch 1: 2 * blocks dependent launches per pass, each
+    released early by the one before it (programmatic dependent launch), replayed from a CUDA graph.  Rotating
+    replicas of the stack (together larger than L2) make every pass stream its weights from HBM."""
+    s = inputs.StackWorkload(blocks=blocks, batch=1, dtype="f32")
+    stacks, keep, flops, bytes_ = [], [], 0, 0
+    for r in range(replicas):
+        layers = []
+        for L, sp in zip(s.layers(seed=r), s.layer_specs()):
+            v, ix, rows = cfi.cfi_pack(L.w_dense, L.mask)
+            layers.append(cfi.cfi_create(v, ix, rows, L.bias, sp[0], sp[1], dtype="f32", act=sp[4]))
+            if r == 0:
+                flops += 2 * rows.shape[0] * sp[2]
+                bytes_ += rows.shape[0] * sp[2] * 8 + (sp[0] + 2 * sp[1]) * 4 + rows.shape[0] * 4
+        stacks.append(cfi.cfi_stack_create(layers, 1))
+        keep.append(layers)
+    x = torch.from_numpy(s.x(seed=0)).to("cuda", torch.float32)
+    y = torch.empty((1, s.d_model), device="cuda", dtype=torch.float32)
+    stream = torch.cuda.Stream()
+    passes = 50 * replicas
+    with torch.cuda.stream(stream):
+        for st in stacks:
+            cfi.cfi_stack_forward(st, x, y, 1)
+        stream.synchronize()
+        eager = _time_torch(lambda: cfi.cfi_stack_forward(stacks[0], x, y, 1), torch, iters=200)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(passes):
+                cfi.cfi_stack_forward(stacks[i % replicas], x, y, 1)
+        g.replay()
+        stream.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(20):
+            g.replay()
+        b.record(stream)
+        b.synchronize()
+    sec = a.elapsed_time(b) * 1e-3 / (20 * passes)
+    for st in stacks:
+        st.close()
+    for layers in keep:
+        for l in layers:
+            l.close()
+    return {"layers": 2 * blocks, "dtype": "f32", "us_per_pass_graph_cold": sec * 1e6, "us_per_layer": sec * 1e6 / (2 * blocks),
+            "us_per_pass_eager_warm": eager * 1e6, "algorithmic_bytes": bytes_,
+            "hbm_frac": bytes_ / sec / 1e9 / peaks["hbm_gbs"], "gflops": flops / sec / 1e9,
+            "l2": f"{replicas} rotating stacks, {replicas * bytes_ / 1e6:.0f} MB vs L2 {l2 / 1e6:.0f} MB"}
 
 
 def batch1_leg(W, cfi, torch, l2, peaks, peak_kind):
