@@ -871,7 +871,7 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
 }
 
 // Rates used to choose between the gather kernel and the split-TF32 dense kernel for fp32 layers (measured).
-constexpr double kDenseTf32SecondsPerBlock = 0.57e-6, kGatherTflops = 12.5;
+constexpr double kDenseTf32SecondsPerBlock = 0.45e-6, kGatherTflops = 12.5;
 
 int choose_variant(const cfi_layer* l, int batch) {
     // Up to three batch tiles of 8 the split-k kernel (weights re-read from L2 per tile) beats the 64-wide tiles of
@@ -888,9 +888,11 @@ int choose_variant(const cfi_layer* l, int batch) {
         if (!bs.ok) return CFI_VARIANT_DENSE_TC;
         const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + kTfN - 1) / kTfN);
         const int64_t waves = (tiles + l->sm_count - 1) / l->sm_count;
-        const double t_dense = (double)waves * ((l->d.in + kTfK - 1) / kTfK) * kDenseTf32SecondsPerBlock + 3e-6;
+        const double t_dense = (double)waves * ((l->d.in + kTfK - 1) / kTfK) * kDenseTf32SecondsPerBlock + 3.5e-6;
         const double staging = (double)bs.grid_y * kBatchTile * l->d.in * 4.0 * bs.grid_x;
-        const double t_gather = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12) + staging / 3e12 + 5e-6;
+        // Arithmetic and the re-staging of x overlap about half of the shorter of the two.
+        const double t_fma = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12), t_stage = staging / 3.7e12;
+        const double t_gather = t_fma + t_stage - 0.5 * std::min(t_fma, t_stage) + 5e-6;
         if (t_dense < t_gather) return CFI_VARIANT_DENSE_TC;
     }
     return batch_shape(l, batch).ok ? CFI_VARIANT_BATCH : CFI_VARIANT_SPLITK;
