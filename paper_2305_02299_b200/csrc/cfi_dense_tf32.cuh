@@ -28,6 +28,14 @@
 // and after the last block warps 2..17 run the epilogue: tcgen05.ld, bias, activation, y tile through shared
 // memory, 256-byte runs per batch row.  Tensor memory: columns 0..63 accumulator, then per slot 32 columns of
 // x_hi and 32 of x_lo.  All mbarrier waits are bounded (status code 2), as in the bf16 kernel.
+//
+// Split K over a thread-block cluster: a layer with few output tiles and a long K (3072 -> 768 at batch 256 has 24
+// tiles of 96 K blocks) would leave most SMs idle, so the launch may give each tile to a cluster of 2, 4 or 8 CTAs
+// (cluster dimension z).  CTA r of the cluster contracts the r-th share of the K blocks; the partial tiles are left
+// in each CTA's shared memory, and after a cluster barrier CTA r sums rows [128 r / S, 128 (r + 1) / S) of all S
+// partial tiles in rank order through distributed shared memory, adds the bias, applies the activation and stores
+// them.  The barrier is the hardware cluster barrier (no flags, no global workspace), the order of additions is
+// fixed, and the layer stays read-only, so concurrent calls on one layer remain safe.
 
 constexpr int kTfM = 128, kTfN = 64, kTfK = 32, kTfStages = 4;
 constexpr int kTfGroups = 4;  // groups of four worker warps; group g splits the K blocks kb with kb % kTfGroups == g
@@ -67,6 +75,34 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         : "memory");
 }
 
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+// Every thread of every CTA of the cluster; writes to shared memory before it are visible to reads through
+// distributed shared memory after it.
+__device__ __forceinline__ void cluster_sync_all() {
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// 16 bytes at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float4 v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(remote)
+                 : "memory");
+    return v;
+}
+
 // hi = v with the 13 low mantissa bits cleared; lo = the same of (v - hi).  Both are exact TF32 numbers.
 __device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
     hi = __uint_as_float(__float_as_uint(v) & 0xFFFFE000u);
@@ -87,6 +123,10 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     float* bias_s = reinterpret_cast<float*>(smem_at(ctl + 128));
     const int m0 = blockIdx.y * kTfM, n0 = blockIdx.x * kTfN;
     const int k_blocks = (L.in + kTfK - 1) / kTfK;
+    // This CTA's share of the K blocks: [kb0, kb0 + n_local).
+    const int split = (int)cluster_rank(), n_split = (int)cluster_size();
+    const int kb0 = (int)(((int64_t)k_blocks * split) / n_split);
+    const int n_local = (int)(((int64_t)k_blocks * (split + 1)) / n_split) - kb0;
 
     if (tid == 0) {
         for (int s = 0; s < kTfStages; ++s) {
@@ -115,20 +155,20 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
 
     if (warp == 0 && lane == 0) {
         // ---------------------------------------------------------------- TMA producer
-        for (int kb = 0; kb < k_blocks && ok; ++kb) {
-            const int s = kb % kTfStages;
-            if (kb >= kTfStages) ok = mbar_wait(empty0 + 8 * s, (uint32_t)(kb / kTfStages - 1) & 1u, kTcSpinLimit);
+        for (int i = 0; i < n_local && ok; ++i) {
+            const int s = i % kTfStages;
+            if (i >= kTfStages) ok = mbar_wait(empty0 + 8 * s, (uint32_t)(i / kTfStages - 1) & 1u, kTcSpinLimit);
             if (!ok) break;
             const uint32_t a_dst = smem_u32(ring + s * kTfStageBytes), b_dst = a_dst + kTfABytes;
             mbar_expect_tx(full0 + 8 * s, kTfABytes + kTfBBytes);
-            tma_load_2d(a_dst, &map_x, full0 + 8 * s, kb * kTfK, m0);
-            tma_load_2d(b_dst, &map_w, full0 + 8 * s, kb * kTfK, n0);
+            tma_load_2d(a_dst, &map_x, full0 + 8 * s, (kb0 + i) * kTfK, m0);
+            tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + i) * kTfK, n0);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
-        for (int kb = 0; kb < k_blocks && ok; ++kb) {
-            const int s = kb % kTfStages;
-            ok = mbar_wait(ready0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
+        for (int i = 0; i < n_local && ok; ++i) {
+            const int s = i % kTfStages;
+            ok = mbar_wait(ready0 + 8 * s, (uint32_t)(i / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t b_hi = smem_u32(ring + s * kTfStageBytes + kTfABytes);  // Wd lo follows at + kTfBBytes
@@ -140,7 +180,7 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                 // Wd lo lies right behind Wd hi, so the two boxes read as one K-major operand of 128 rows: one MMA
                 // of N = 128 gives x_hi w_hi in columns 0..63 and x_hi w_lo in columns 64..127; a second of N = 64
                 // adds x_lo w_hi to the first half.  (An MMA of this size costs about the same whatever its N.)
-                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbh + off, tf_instr_desc(2 * kTfN), (kb | k) != 0 ? 1u : 0u);
+                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbh + off, tf_instr_desc(2 * kTfN), (i | k) != 0 ? 1u : 0u);
                 umma_tf32_ts(tmem_base, a_lo + 8u * k, dbh + off, tf_instr_desc(kTfN), 1u);
             }
             umma_commit(empty0 + 8 * s);
@@ -151,9 +191,9 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         const int wt = tid - 64;            // 0 .. 32 * kTfWorkerWarps - 1
         const int group = (warp - 2) >> 2;  // the group's four warps cover the four lane quarters of tensor memory
         const int gt = wt & 127;            // thread within the group
-        for (int kb = group; kb < k_blocks && ok; kb += kTfGroups) {
-            const int s = kb % kTfStages;
-            ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / kTfStages) & 1u, kTcSpinLimit);
+        for (int i = group; i < n_local && ok; i += kTfGroups) {
+            const int s = i % kTfStages;
+            ok = mbar_wait(full0 + 8 * s, (uint32_t)(i / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
             {
                 // x: this thread's batch row (tensor-memory lane): 8 chunks of 16 bytes, un-permuted from the
@@ -202,37 +242,58 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         const int q = warp & 3;  // tensor-memory lanes 32 q .. 32 q + 31; the group number picks 16 of the 64 columns
         const int row = 32 * q + lane;
         if (ok) {
-            // y tile in shared memory: 128 rows x 256 bytes (64 fp32), 16-byte chunks permuted by chunk ^ (row & 15).
+            // This CTA's partial tile (no bias yet) in shared memory: 128 rows x 256 bytes (64 fp32), 16-byte chunks
+            // permuted by chunk ^ (row & 15).  The two accumulator halves are the two groups of products.
             uint32_t v[16], v1[16];
             const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(16 * group);
             tmem_ld16(t_acc, v);
             tmem_ld16(t_acc + kTfN, v1);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-            for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(v1[e]));
-#pragma unroll
             for (int e4 = 0; e4 < 4; ++e4) {
                 const int col = 16 * group + 4 * e4;
-                const float4 bv = *reinterpret_cast<const float4*>(bias_s + col);
-                float4 r;
-                r.x = activate(__uint_as_float(v[4 * e4 + 0]) + bv.x, L.act);
-                r.y = activate(__uint_as_float(v[4 * e4 + 1]) + bv.y, L.act);
-                r.z = activate(__uint_as_float(v[4 * e4 + 2]) + bv.z, L.act);
-                r.w = activate(__uint_as_float(v[4 * e4 + 3]) + bv.w, L.act);
+                float4 r = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                if (n_local > 0) {  // a CTA without K blocks has issued no MMA: its accumulator holds nothing
+                    r.x = __uint_as_float(v[4 * e4 + 0]) + __uint_as_float(v1[4 * e4 + 0]);
+                    r.y = __uint_as_float(v[4 * e4 + 1]) + __uint_as_float(v1[4 * e4 + 1]);
+                    r.z = __uint_as_float(v[4 * e4 + 2]) + __uint_as_float(v1[4 * e4 + 2]);
+                    r.w = __uint_as_float(v[4 * e4 + 3]) + __uint_as_float(v1[4 * e4 + 3]);
+                }
                 *reinterpret_cast<float4*>(smem_at(ring + row * 256 + (((col >> 2) ^ (row & 15)) << 4))) = r;
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * kTfWorkerWarps) : "memory");
-        if (ok) {
-            for (int r = wt >> 4; r < kTfM; r += 2 * kTfWorkerWarps) {  // 16 threads per row
-                const int ch = wt & 15, m = m0 + r, n = n0 + 4 * ch;
-                if (m < batch && n < L.out) {
-                    const float4 val = *reinterpret_cast<const float4*>(smem_at(ring + r * 256 + ((ch ^ (r & 15)) << 4)));
-                    *reinterpret_cast<float4*>(y + (size_t)m * L.out + n) = val;
+        if (n_split == 1) asm volatile("bar.sync 1, %0;" ::"n"(32 * kTfWorkerWarps) : "memory");
+    }
+    // The partial tiles of the whole cluster are complete: every thread of every CTA passes here, whatever `ok` says.
+    if (n_split > 1) cluster_sync_all();
+    if (warp >= 2 && ok) {
+        // Rows [split * rows_per, (split + 1) * rows_per) of the tile: sum over the cluster in rank order, bias,
+        // activation, store.  16 threads per row, 256-byte runs.
+        const int wt = tid - 64, ch = wt & 15, rows_per = kTfM / n_split;
+        const float4 bv = *reinterpret_cast<const float4*>(bias_s + 4 * ch);
+        for (int rr = wt >> 4; rr < rows_per; rr += 2 * kTfWorkerWarps) {
+            const int r = split * rows_per + rr, m = m0 + r, n = n0 + 4 * ch;
+            if (m < batch && n < L.out) {
+                const uint32_t off = ring + r * 256 + ((ch ^ (r & 15)) << 4);
+                float4 a;
+                if (n_split == 1) {
+                    a = *reinterpret_cast<const float4*>(smem_at(off));
+                } else {
+                    a = ld_cluster_f4(smem_u32(off), 0u);
+                    for (int p = 1; p < n_split; ++p) {
+                        const float4 t = ld_cluster_f4(smem_u32(off), (uint32_t)p);
+                        a.x += t.x, a.y += t.y, a.z += t.z, a.w += t.w;
+                    }
                 }
+                a.x = activate(a.x + bv.x, L.act);
+                a.y = activate(a.y + bv.y, L.act);
+                a.z = activate(a.z + bv.z, L.act);
+                a.w = activate(a.w + bv.w, L.act);
+                *reinterpret_cast<float4*>(y + (size_t)m * L.out + n) = a;
             }
         }
     }
+    if (n_split > 1) cluster_sync_all();  // no CTA leaves while another may still read its tile
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();

@@ -716,23 +716,34 @@ cfi_status_t set_smem(size_t bytes, int device) {
 
 // Launch with programmatic stream serialisation allowed: the kernel may start before its predecessor in the
 // stream has finished (see pdl_wait in the kernels).
+// cluster_z > 1 launches thread-block clusters of cluster_z CTAs along z (grid.z must be a multiple of it).
 template <typename... KArgs, typename... Args>
-cfi_status_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+cfi_status_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, int cluster_z,
+                                cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = dim3((unsigned)threads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr{};
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr.val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2]{};
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = (unsigned)cluster_z;
+    cfg.attrs = attr;
+    cfg.numAttrs = cluster_z > 1 ? 2 : 1;
     if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) {
         cudaGetLastError();
         return CFI_ERR_CUDA;
     }
     return CFI_OK;
+}
+
+template <typename... KArgs, typename... Args>
+cfi_status_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+    return launch_pdl_cluster(kernel, grid, threads, smem, 1, st, args...);
 }
 
 template <typename VT, int BT, int G>
@@ -843,14 +854,66 @@ bool encode_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Time model of the split-TF32 kernel (measured): seconds per 32-column block of K and tile, a fixed part per launch,
+// and the cluster reduction when K is split.
+constexpr double kDenseTf32SecondsPerBlock = 0.45e-6, kDenseTf32Fixed = 3.5e-6, kDenseTf32Reduce = 1.0e-6;
+
+// Clusters of `split` CTAs of the split-TF32 kernel that the device can hold at once (cached per device and size).
+int tf32_resident_clusters(const cfi_layer* l, int split) {
+    static std::atomic<int> cache[64][4];
+    const int slot = split == 1 ? 0 : split == 2 ? 1 : split == 4 ? 2 : 3;
+    if (l->device < 0 || l->device >= 64) return std::max(1, l->sm_count / split);
+    int v = cache[l->device][slot].load(std::memory_order_acquire);
+    if (v > 0) return v;
+    v = std::max(1, l->sm_count / split);
+    if (split > 1 && set_smem<cfi_dense_tf32_kernel>(kTfSmemBytes, l->device) == CFI_OK) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(1, 1, (unsigned)split);
+        cfg.blockDim = dim3(kTfThreads);
+        cfg.dynamicSmemBytes = kTfSmemBytes;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 1, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = (unsigned)split;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, cfi_dense_tf32_kernel, &cfg) == cudaSuccess && n > 0) v = n;
+        else cudaGetLastError();
+    }
+    cache[l->device][slot].store(v, std::memory_order_release);
+    return v;
+}
+
+struct Tf32Shape {
+    int split;       // CTAs per output tile (cluster size along z): 1, 2, 4 or 8
+    double seconds;  // modelled time of the launch
+};
+
+// Splitting K pays when the tiles alone leave SMs idle and every CTA still gets a few K blocks.
+Tf32Shape tf32_shape(const cfi_layer* l, int batch) {
+    const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + kTfN - 1) / kTfN);
+    const int k_blocks = (l->d.in + kTfK - 1) / kTfK;
+    Tf32Shape best{1, 0.0};
+    for (int split = 1; split <= 8; split *= 2) {
+        if (split > 1 && (k_blocks < 4 * split || tiles * split > 2 * (int64_t)l->sm_count)) break;
+        const int64_t resident = tf32_resident_clusters(l, split);
+        const int64_t waves = (tiles + resident - 1) / resident;
+        const double t = (double)waves * ((k_blocks + split - 1) / split) * kDenseTf32SecondsPerBlock + kDenseTf32Fixed +
+                         (split > 1 ? kDenseTf32Reduce : 0.0);
+        if (split == 1 || t < best.seconds) best = Tf32Shape{split, t};
+    }
+    return best;
+}
+
 cfi_status_t launch_dense_tf32(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
     const int grid_x = (l->d.out + kTfN - 1) / kTfN, grid_y = (batch + kTfM - 1) / kTfM;
     if (grid_y > 65535) return CFI_ERR_SHAPE;
     CUtensorMap map_x;
     if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 4, kTfM)) return CFI_ERR_SHAPE;
     if (cfi_status_t e = set_smem<cfi_dense_tf32_kernel>(kTfSmemBytes, l->device)) return e;
-    return launch_pdl(cfi_dense_tf32_kernel, dim3(grid_x, grid_y), kTfThreads, kTfSmemBytes, st, l->d, map_x, l->map_w,
-                      static_cast<float*>(y), batch);
+    const int split = tf32_shape(l, batch).split;
+    return launch_pdl_cluster(cfi_dense_tf32_kernel, dim3(grid_x, grid_y, split), kTfThreads, kTfSmemBytes, split, st, l->d,
+                              map_x, l->map_w, static_cast<float*>(y), batch);
 }
 
 cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
@@ -870,8 +933,8 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
                       l->map_w, static_cast<__nv_bfloat16*>(y), batch);
 }
 
-// Rates used to choose between the gather kernel and the split-TF32 dense kernel for fp32 layers (measured).
-constexpr double kDenseTf32SecondsPerBlock = 0.45e-6, kGatherTflops = 12.5;
+// Rate of the gather kernel's arithmetic, used to choose between it and the split-TF32 dense kernel (measured).
+constexpr double kGatherTflops = 12.5;
 
 int choose_variant(const cfi_layer* l, int batch) {
     // Up to three batch tiles of 8 the split-k kernel (weights re-read from L2 per tile) beats the 64-wide tiles of
@@ -879,16 +942,15 @@ int choose_variant(const cfi_layer* l, int batch) {
     if (batch <= 24) return CFI_VARIANT_SPLITK;
     // bf16 at large batch: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
     // (10 TFLOP/s effective for the gather against several hundred dense); below a full 128-row tile it does not pay.
-    if (l->tc_ok && batch >= 96) {
-        if (l->dtype == CFI_BF16) return CFI_VARIANT_DENSE_TC;
+    if (l->tc_ok && l->dtype == CFI_BF16 && batch >= 96) return CFI_VARIANT_DENSE_TC;
+    if (l->tc_ok && l->dtype == CFI_F32) {
         // fp32: the split-TF32 kernel takes a fixed time per 32-column block of K and tile (it is bound by the
-        // shared-memory traffic of splitting and re-reading the operands); the gather kernel's time is its FMAs
-        // at the rate it sustains plus the re-staging of x by every row tile.  Constants fitted to measurements.
+        // number of MMA instructions), whatever the fill of its 128-row batch tile, and can split K over a cluster
+        // when the tiles are few; the gather kernel's time is its FMAs at the rate it sustains plus the re-staging
+        // of x by every row tile.  Constants fitted to measurements.
         const BatchShape bs = batch_shape(l, batch);
         if (!bs.ok) return CFI_VARIANT_DENSE_TC;
-        const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + kTfN - 1) / kTfN);
-        const int64_t waves = (tiles + l->sm_count - 1) / l->sm_count;
-        const double t_dense = (double)waves * ((l->d.in + kTfK - 1) / kTfK) * kDenseTf32SecondsPerBlock + 3.5e-6;
+        const double t_dense = tf32_shape(l, batch).seconds;
         const double staging = (double)bs.grid_y * kBatchTile * l->d.in * 4.0 * bs.grid_x;
         // Arithmetic and the re-staging of x overlap about half of the shorter of the two.
         const double t_fma = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12), t_stage = staging / 3.7e12;

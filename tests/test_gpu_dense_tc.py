@@ -14,7 +14,9 @@ from parity import TOL, device_layer, oracle_layer, run_device, scaled_error
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("in_f,out_f,k,nabl", [(64, 8, 5, 1), (72, 136, 9, 10), (768, 384, 77, 19), (3072, 200, 307, 20)])
+@pytest.mark.parametrize("in_f,out_f,k,nabl", [(64, 8, 5, 1), (72, 136, 9, 10), (768, 384, 77, 19), (3072, 200, 307, 20),
+                                              # few tiles and a long K: K split over a cluster of 4 or 8 CTAs, uneven shares, ragged tail
+                                              (1000, 72, 100, 5), (520, 640, 52, 30)])
 @pytest.mark.parametrize("B", [1, 5, 128, 257])
 @pytest.mark.parametrize("act", ["none", "gelu"])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
