@@ -359,12 +359,17 @@ def main():
         hbm_gbs = rep.bytes_per_step / per_call / 1e9
         info = cfi.cfi_layer_info(rep.layers[0])
         chosen = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
+        tile_shape = None
+        if chosen == "dense_tc" and args.variant in ("auto", "dense_tc"):
+            tn, cl = cfi.cfi_dense_tile_shape(rep.layers[0], w.batch)
+            tile_shape = {"tile": [128, tn], "cluster_k_split": cl}
         line = {
             "metric": METRIC, "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": per_call * 1e3, "us_per_call": per_call * 1e6,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "in": w.in_features, "out": w.out_features, "k": w.k,
                        "n_active": rep.n_active, "batch": w.batch, "variant": chosen if args.variant == "auto" else args.variant,
+                       "dense_tile": tile_shape,
                        "l2": f"inputs larger than L2: {rep.R} rotating replicas of layer+x+y, "
                              f"{rep.total_bytes / 1e6:.0f} MB vs L2 {l2 / 1e6:.0f} MB",
                        "timing": "CUDA-graph replays between CUDA events on the launching stream"},

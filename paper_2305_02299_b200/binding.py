@@ -25,7 +25,7 @@ _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE,
 _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
-           "cfi_layer_info", "cfi_choose_variant", "cfi_device_status", "cfi_destroy",
+           "cfi_layer_info", "cfi_choose_variant", "cfi_dense_tile_shape", "cfi_device_status", "cfi_destroy",
            "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static",
            "cfi_probe_device")
 
@@ -75,6 +75,7 @@ def _load() -> ctypes.CDLL:
     lib.cfi_forward_host.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_layer_info.argtypes = [vp, ctypes.POINTER(LayerInfo)]
     lib.cfi_choose_variant.argtypes = [vp, ci, i32p]
+    lib.cfi_dense_tile_shape.argtypes = [vp, ci, i32p, i32p]
     lib.cfi_device_status.argtypes = [vp, vp, i32p]
     lib.cfi_destroy.argtypes = [vp]
     lib.cfi_stack_create.argtypes = [ctypes.POINTER(vp), ci, ci, ctypes.POINTER(vp)]
@@ -208,6 +209,13 @@ def cfi_choose_variant(layer: Layer, batch: int) -> int:
     v = ctypes.c_int32(0)
     _check(_lib.cfi_choose_variant(layer.handle, batch, ctypes.byref(v)), "cfi_choose_variant")
     return v.value
+
+
+def cfi_dense_tile_shape(layer: Layer, batch: int):
+    """(outputs per tile, CTAs sharing a tile through a cluster) of the tensor-core variant at this batch size."""
+    tn, cl = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_lib.cfi_dense_tile_shape(layer.handle, batch, ctypes.byref(tn), ctypes.byref(cl)), "cfi_dense_tile_shape")
+    return tn.value, cl.value
 
 
 def cfi_device_status(layer: Layer, stream=None) -> int:

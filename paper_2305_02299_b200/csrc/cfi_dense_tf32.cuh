@@ -37,17 +37,17 @@
 // them.  The barrier is the hardware cluster barrier (no flags, no global workspace), the order of additions is
 // fixed, and the layer stays read-only, so concurrent calls on one layer remain safe.
 
-constexpr int kTfM = 128, kTfN = 64, kTfK = 32, kTfStages = 4;
+constexpr int kTfM = 128, kTfK = 32, kTfStages = 4;  // the output tile is kTfM x TN with TN = 64 or 128 (template)
 constexpr int kTfGroups = 4;  // groups of four worker warps; group g splits the K blocks kb with kb % kTfGroups == g
 constexpr int kTfWorkerWarps = 4 * kTfGroups, kTfThreads = 64 + 32 * kTfWorkerWarps;
 // A ring slot is always split by the same group, so that one phase bit per barrier is enough: a group that ran a
 // whole phase ahead on another group's slot would pass its wait early.
 static_assert(kTfStages == kTfGroups, "slot s belongs to group s");
-constexpr uint32_t kTfABytes = kTfM * kTfK * 4, kTfBBytes = kTfN * kTfK * 4;   // 16 KB, 8 KB
-constexpr uint32_t kTfStageBytes = kTfABytes + 2 * kTfBBytes;                  // x raw | Wd hi | Wd lo: 32 KB
-constexpr uint32_t kTfAccCols = 2 * kTfN;                                      // x_hi w_hi + x_lo w_hi | x_hi w_lo
-constexpr uint32_t kTfTmemCols = 512;                                          // 128 + 4 * 64 = 384, next power of two
-constexpr size_t kTfSmemBytes = 1024 + kTfStages * kTfStageBytes + 1024;
+constexpr uint32_t kTfABytes = kTfM * kTfK * 4;                                 // x box: 16 KB
+constexpr uint32_t kTfTmemCols = 512;  // 2 TN accumulator columns (x_hi w_hi + x_lo w_hi | x_hi w_lo) + 4 slots of 64
+__host__ __device__ constexpr uint32_t tf_b_bytes(int tn) { return (uint32_t)tn * kTfK * 4; }  // Wd box: 8 or 16 KB
+__host__ __device__ constexpr uint32_t tf_stage_bytes(int tn) { return kTfABytes + 2 * tf_b_bytes(tn); }  // x | Wd hi | Wd lo
+__host__ __device__ constexpr size_t tf_smem_bytes(int tn) { return 1024 + (size_t)kTfStages * tf_stage_bytes(tn) + 1024; }
 
 // fp32 accumulate, tf32 x tf32, both K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t tf_instr_desc(int n) {
@@ -110,18 +110,22 @@ __device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
 }
 
 // Shared memory from the first 1024-byte boundary: kTfStages slots of [x raw | Wd hi | Wd lo]; then
-//   +0 full[4], +32 ready[4], +64 empty[4], +96 accumulator barrier, +104 tensor-memory base, +128 bias[64].
+//   +0 full[4], +32 ready[4], +64 empty[4], +96 accumulator barrier, +104 tensor-memory base, +128 bias[TN].
+template <int TN>
 __global__ void __launch_bounds__(kTfThreads, 1)
 cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                       float* __restrict__ y, int batch) {
     pdl_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t base = ((smem_u32(0) + 1023u) & ~1023u) - smem_u32(0);
-    const uint32_t ring = base, ctl = base + kTfStages * kTfStageBytes;
+    static_assert(TN == 64 || TN == 128, "tile width");
+    constexpr uint32_t kBBytes = tf_b_bytes(TN), kStageBytes = tf_stage_bytes(TN), kAccCols = 2 * TN;
+    static_assert(kAccCols + 64 * kTfStages <= kTfTmemCols, "tensor memory: accumulators + x slots");
+    const uint32_t ring = base, ctl = base + kTfStages * kStageBytes;
     const uint32_t full0 = smem_u32(ctl), ready0 = smem_u32(ctl + 32), empty0 = smem_u32(ctl + 64), accum = smem_u32(ctl + 96);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_at(ctl + 104));
     float* bias_s = reinterpret_cast<float*>(smem_at(ctl + 128));
-    const int m0 = blockIdx.y * kTfM, n0 = blockIdx.x * kTfN;
+    const int m0 = blockIdx.y * kTfM, n0 = blockIdx.x * TN;
     const int k_blocks = (L.in + kTfK - 1) / kTfK;
     // This CTA's share of the K blocks: [kb0, kb0 + n_local).
     const int split = (int)cluster_rank(), n_split = (int)cluster_size();
@@ -142,7 +146,7 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (tid >= 64 && tid < 64 + kTfN) {
+    if (tid >= 64 && tid < 64 + TN) {
         const int n = n0 + tid - 64;
         bias_s[tid - 64] = n < L.out ? L.bias[n] : 0.0f;
     }
@@ -159,8 +163,8 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             const int s = i % kTfStages;
             if (i >= kTfStages) ok = mbar_wait(empty0 + 8 * s, (uint32_t)(i / kTfStages - 1) & 1u, kTcSpinLimit);
             if (!ok) break;
-            const uint32_t a_dst = smem_u32(ring + s * kTfStageBytes), b_dst = a_dst + kTfABytes;
-            mbar_expect_tx(full0 + 8 * s, kTfABytes + kTfBBytes);
+            const uint32_t a_dst = smem_u32(ring + s * kStageBytes), b_dst = a_dst + kTfABytes;
+            mbar_expect_tx(full0 + 8 * s, kTfABytes + kBBytes);
             tma_load_2d(a_dst, &map_x, full0 + 8 * s, (kb0 + i) * kTfK, m0);
             tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + i) * kTfK, n0);
         }
@@ -171,17 +175,17 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             ok = mbar_wait(ready0 + 8 * s, (uint32_t)(i / kTfStages) & 1u, kTcSpinLimit);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t b_hi = smem_u32(ring + s * kTfStageBytes + kTfABytes);  // Wd lo follows at + kTfBBytes
+            const uint32_t b_hi = smem_u32(ring + s * kStageBytes + kTfABytes);  // Wd lo follows at + kBBytes
             const uint64_t dbh = umma_desc_k_sw128(b_hi);
-            const uint32_t a_hi = tmem_base + kTfAccCols + (uint32_t)(64 * s), a_lo = a_hi + 32u;
+            const uint32_t a_hi = tmem_base + kAccCols + (uint32_t)(64 * s), a_lo = a_hi + 32u;
 #pragma unroll
             for (int k = 0; k < kTfK / 8; ++k) {  // 8 fp32 further along K: 8 columns of tensor memory, 32 bytes of a row
                 const uint64_t off = (uint64_t)(2 * k);
-                // Wd lo lies right behind Wd hi, so the two boxes read as one K-major operand of 128 rows: one MMA
-                // of N = 128 gives x_hi w_hi in columns 0..63 and x_hi w_lo in columns 64..127; a second of N = 64
-                // adds x_lo w_hi to the first half.  (An MMA of this size costs about the same whatever its N.)
-                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbh + off, tf_instr_desc(2 * kTfN), (i | k) != 0 ? 1u : 0u);
-                umma_tf32_ts(tmem_base, a_lo + 8u * k, dbh + off, tf_instr_desc(kTfN), 1u);
+                // Wd lo lies right behind Wd hi, so the two boxes read as one K-major operand of 2 TN rows: one MMA
+                // of N = 2 TN gives x_hi w_hi in columns 0..TN-1 and x_hi w_lo in columns TN..2TN-1; a second of
+                // N = TN adds x_lo w_hi to the first half.  (An MMA costs about 50 cycles + 0.43 per column of N.)
+                umma_tf32_ts(tmem_base, a_hi + 8u * k, dbh + off, tf_instr_desc(2 * TN), (i | k) != 0 ? 1u : 0u);
+                umma_tf32_ts(tmem_base, a_lo + 8u * k, dbh + off, tf_instr_desc(TN), 1u);
             }
             umma_commit(empty0 + 8 * s);
         }
@@ -199,8 +203,8 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                 // x: this thread's batch row (tensor-memory lane): 8 chunks of 16 bytes, un-permuted from the
                 // swizzle, split and written straight to tensor memory.
                 const int m = 32 * (warp & 3) + lane;
-                const uint32_t row_off = ring + s * kTfStageBytes + (uint32_t)m * 128u;
-                const uint32_t t_hi = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + kTfAccCols + (uint32_t)(64 * s);
+                const uint32_t row_off = ring + s * kStageBytes + (uint32_t)m * 128u;
+                const uint32_t t_hi = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + kAccCols + (uint32_t)(64 * s);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     uint32_t hi[16], lo[16];
@@ -217,10 +221,10 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                     tmem_st16(t_hi + 16u * half, hi);
                     tmem_st16(t_hi + 32u + 16u * half, lo);
                 }
-                // Wd: element-wise, hi in place, lo beside it (4 of its 512 16-byte pieces per thread).
-                const uint32_t hi_off = ring + s * kTfStageBytes + kTfABytes, lo_off = hi_off + kTfBBytes;
+                // Wd: element-wise, hi in place, lo beside it (TN / 16 of its 8 TN 16-byte pieces per thread).
+                const uint32_t hi_off = ring + s * kStageBytes + kTfABytes, lo_off = hi_off + kBBytes;
 #pragma unroll
-                for (uint32_t e = (uint32_t)gt * 16u; e < kTfBBytes; e += 128u * 16u) {
+                for (uint32_t e = (uint32_t)gt * 16u; e < kBBytes; e += 128u * 16u) {
                     const float4 v = *reinterpret_cast<const float4*>(smem_at(hi_off + e));
                     float4 h, l;
                     split_tf32(v.x, h.x, l.x);
@@ -239,27 +243,31 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         ok = __all_sync(0xffffffffu, ok);
         if (ok) ok = mbar_wait(accum, 0u, kTcSpinLimit);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int q = warp & 3;  // tensor-memory lanes 32 q .. 32 q + 31; the group number picks 16 of the 64 columns
+        const int q = warp & 3;  // tensor-memory lanes 32 q .. 32 q + 31; the group number picks TN / 4 of the TN columns
         const int row = 32 * q + lane;
         if (ok) {
-            // This CTA's partial tile (no bias yet) in shared memory: 128 rows x 256 bytes (64 fp32), 16-byte chunks
-            // permuted by chunk ^ (row & 15).  The two accumulator halves are the two groups of products.
-            uint32_t v[16], v1[16];
-            const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(16 * group);
-            tmem_ld16(t_acc, v);
-            tmem_ld16(t_acc + kTfN, v1);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            // This CTA's partial tile (no bias yet) in shared memory: 128 rows of 4 TN bytes, 16-byte chunks permuted
+            // by chunk ^ (row & 15).  The two accumulator halves are the two groups of products.
 #pragma unroll
-            for (int e4 = 0; e4 < 4; ++e4) {
-                const int col = 16 * group + 4 * e4;
-                float4 r = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                if (n_local > 0) {  // a CTA without K blocks has issued no MMA: its accumulator holds nothing
-                    r.x = __uint_as_float(v[4 * e4 + 0]) + __uint_as_float(v1[4 * e4 + 0]);
-                    r.y = __uint_as_float(v[4 * e4 + 1]) + __uint_as_float(v1[4 * e4 + 1]);
-                    r.z = __uint_as_float(v[4 * e4 + 2]) + __uint_as_float(v1[4 * e4 + 2]);
-                    r.w = __uint_as_float(v[4 * e4 + 3]) + __uint_as_float(v1[4 * e4 + 3]);
+            for (int c16 = 0; c16 < TN / 64; ++c16) {
+                const int col0 = (TN / 4) * group + 16 * c16;
+                uint32_t v[16], v1[16];
+                const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col0;
+                tmem_ld16(t_acc, v);
+                tmem_ld16(t_acc + TN, v1);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int e4 = 0; e4 < 4; ++e4) {
+                    const int col = col0 + 4 * e4;
+                    float4 r = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    if (n_local > 0) {  // a CTA without K blocks has issued no MMA: its accumulator holds nothing
+                        r.x = __uint_as_float(v[4 * e4 + 0]) + __uint_as_float(v1[4 * e4 + 0]);
+                        r.y = __uint_as_float(v[4 * e4 + 1]) + __uint_as_float(v1[4 * e4 + 1]);
+                        r.z = __uint_as_float(v[4 * e4 + 2]) + __uint_as_float(v1[4 * e4 + 2]);
+                        r.w = __uint_as_float(v[4 * e4 + 3]) + __uint_as_float(v1[4 * e4 + 3]);
+                    }
+                    *reinterpret_cast<float4*>(smem_at(ring + row * (4 * TN) + (((col >> 2) ^ (row & 15)) << 4))) = r;
                 }
-                *reinterpret_cast<float4*>(smem_at(ring + row * 256 + (((col >> 2) ^ (row & 15)) << 4))) = r;
             }
         }
         if (n_split == 1) asm volatile("bar.sync 1, %0;" ::"n"(32 * kTfWorkerWarps) : "memory");
@@ -268,13 +276,14 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     if (n_split > 1) cluster_sync_all();
     if (warp >= 2 && ok) {
         // Rows [split * rows_per, (split + 1) * rows_per) of the tile: sum over the cluster in rank order, bias,
-        // activation, store.  16 threads per row, 256-byte runs.
-        const int wt = tid - 64, ch = wt & 15, rows_per = kTfM / n_split;
+        // activation, store.  TN / 4 threads per row, runs of 4 TN bytes.
+        constexpr int kPerRow = TN / 4, kRowsPerPass = 32 * kTfWorkerWarps / kPerRow;
+        const int wt = tid - 64, ch = wt % kPerRow, rows_per = (kTfM + n_split - 1) / n_split;
         const float4 bv = *reinterpret_cast<const float4*>(bias_s + 4 * ch);
-        for (int rr = wt >> 4; rr < rows_per; rr += 2 * kTfWorkerWarps) {
+        for (int rr = wt / kPerRow; rr < rows_per; rr += kRowsPerPass) {
             const int r = split * rows_per + rr, m = m0 + r, n = n0 + 4 * ch;
-            if (m < batch && n < L.out) {
-                const uint32_t off = ring + r * 256 + ((ch ^ (r & 15)) << 4);
+            if (r < kTfM && m < batch && n < L.out) {
+                const uint32_t off = ring + r * (4 * TN) + ((ch ^ (r & 15)) << 4);
                 float4 a;
                 if (n_split == 1) {
                     a = *reinterpret_cast<const float4*>(smem_at(off));

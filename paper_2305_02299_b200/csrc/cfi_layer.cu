@@ -60,7 +60,8 @@ struct cfi_layer {
     const void* w_dense = nullptr;
     int out_pad = 0;
     bool tc_ok = false;
-    CUtensorMap map_w{};
+    CUtensorMap map_w{};       // dense copy in boxes of 128 rows (bf16) or 64 rows (fp32)
+    CUtensorMap map_w_wide{};  // fp32 only: boxes of 128 rows
 };
 
 struct cfi_stack {
@@ -854,66 +855,94 @@ bool encode_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Time model of the split-TF32 kernel (measured): seconds per 32-column block of K and tile, a fixed part per launch,
-// and the cluster reduction when K is split.
-constexpr double kDenseTf32SecondsPerBlock = 0.45e-6, kDenseTf32Fixed = 3.5e-6, kDenseTf32Reduce = 1.0e-6;
+// Time model of the split-TF32 kernel (measured): seconds per 32-column block of K and tile of 64 or 128 outputs; a
+// fixed part per wave of CTAs (prologue, pipeline fill, epilogue: CTAs are not persistent, so a second wave pays it
+// again), larger for the wide tile; the cluster reduction when K is split; and the launch itself.
+constexpr double kDenseTf32SecondsPerBlock64 = 0.45e-6, kDenseTf32SecondsPerBlock128 = 0.61e-6, kDenseTf32Wave64 = 3.0e-6,
+                 kDenseTf32Wave128 = 4.5e-6, kDenseTf32Reduce = 1.0e-6, kDenseTf32Launch = 0.7e-6;
+constexpr int kTfMaxSplit = 8;
 
-// Clusters of `split` CTAs of the split-TF32 kernel that the device can hold at once (cached per device and size).
-int tf32_resident_clusters(const cfi_layer* l, int split) {
-    static std::atomic<int> cache[64][4];
-    const int slot = split == 1 ? 0 : split == 2 ? 1 : split == 4 ? 2 : 3;
-    if (l->device < 0 || l->device >= 64) return std::max(1, l->sm_count / split);
-    int v = cache[l->device][slot].load(std::memory_order_acquire);
-    if (v > 0) return v;
-    v = std::max(1, l->sm_count / split);
-    if (split > 1 && set_smem<cfi_dense_tf32_kernel>(kTfSmemBytes, l->device) == CFI_OK) {
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3(1, 1, (unsigned)split);
-        cfg.blockDim = dim3(kTfThreads);
-        cfg.dynamicSmemBytes = kTfSmemBytes;
-        cudaLaunchAttribute attr{};
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = 1, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = (unsigned)split;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, cfi_dense_tf32_kernel, &cfg) == cudaSuccess && n > 0) v = n;
-        else cudaGetLastError();
+template <int TN>
+int tf32_query_clusters(const cfi_layer* l, int split) {
+    if (set_smem<cfi_dense_tf32_kernel<TN>>(tf_smem_bytes(TN), l->device) != CFI_OK) return 0;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(1, 1, (unsigned)split);
+    cfg.blockDim = dim3(kTfThreads);
+    cfg.dynamicSmemBytes = tf_smem_bytes(TN);
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 1, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = (unsigned)split;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, cfi_dense_tf32_kernel<TN>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
     }
-    cache[l->device][slot].store(v, std::memory_order_release);
-    return v;
+    return n;
+}
+
+// Clusters of `split` CTAs of the split-TF32 kernel that the device can hold at once; 0 if it cannot launch that
+// cluster size (cached per device; -1 in the cache stands for 0).
+int tf32_resident_clusters(const cfi_layer* l, int tile_n, int split) {
+    static std::atomic<int> cache[64][2][kTfMaxSplit + 1];
+    if (split == 1) return std::max(1, l->sm_count);
+    if (l->device < 0 || l->device >= 64) return 0;
+    std::atomic<int>& c = cache[l->device][tile_n == 128 ? 1 : 0][split];
+    int v = c.load(std::memory_order_acquire);
+    if (v == 0) {
+        v = tile_n == 128 ? tf32_query_clusters<128>(l, split) : tf32_query_clusters<64>(l, split);
+        if (v <= 0) v = -1;
+        c.store(v, std::memory_order_release);
+    }
+    return v > 0 ? v : 0;
 }
 
 struct Tf32Shape {
-    int split;       // CTAs per output tile (cluster size along z): 1, 2, 4 or 8
+    int tile_n;      // outputs per tile: 64 or 128
+    int split;       // CTAs per output tile (cluster size along z): 1 .. 8
     double seconds;  // modelled time of the launch
 };
 
-// Splitting K pays when the tiles alone leave SMs idle and every CTA still gets a few K blocks.
+// Wide tiles need fewer MMA instructions per output; splitting K over a cluster fills the SMs that the tiles alone
+// would leave idle, as long as every CTA still gets a few K blocks.
 Tf32Shape tf32_shape(const cfi_layer* l, int batch) {
-    const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + kTfN - 1) / kTfN);
     const int k_blocks = (l->d.in + kTfK - 1) / kTfK;
-    Tf32Shape best{1, 0.0};
-    for (int split = 1; split <= 8; split *= 2) {
-        if (split > 1 && (k_blocks < 4 * split || tiles * split > 2 * (int64_t)l->sm_count)) break;
-        const int64_t resident = tf32_resident_clusters(l, split);
-        const int64_t waves = (tiles + resident - 1) / resident;
-        const double t = (double)waves * ((k_blocks + split - 1) / split) * kDenseTf32SecondsPerBlock + kDenseTf32Fixed +
-                         (split > 1 ? kDenseTf32Reduce : 0.0);
-        if (split == 1 || t < best.seconds) best = Tf32Shape{split, t};
+    Tf32Shape best{64, 1, 0.0};
+    bool have = false;
+    for (int tile_n = 64; tile_n <= 128; tile_n *= 2) {
+        const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + tile_n - 1) / tile_n);
+        const double per_block = tile_n == 128 ? kDenseTf32SecondsPerBlock128 : kDenseTf32SecondsPerBlock64;
+        const double per_wave = tile_n == 128 ? kDenseTf32Wave128 : kDenseTf32Wave64;
+        for (int split = 1; split <= kTfMaxSplit; ++split) {
+            if (split > 1 && (k_blocks < 4 * split || tiles * split > 2 * (int64_t)l->sm_count)) break;
+            const int64_t resident = tf32_resident_clusters(l, tile_n, split);
+            if (resident == 0) continue;
+            const int64_t waves = (tiles + resident - 1) / resident;
+            const double t = (double)waves * (((k_blocks + split - 1) / split) * per_block + per_wave +
+                                              (split > 1 ? kDenseTf32Reduce : 0.0)) + kDenseTf32Launch;
+            if (!have || t < best.seconds) best = Tf32Shape{tile_n, split, t}, have = true;
+        }
     }
     return best;
 }
 
+template <int TN>
+cfi_status_t launch_dense_tf32_n(const cfi_layer* l, const CUtensorMap& map_x, const CUtensorMap& map_w, int split, void* y,
+                                 int batch, cudaStream_t st) {
+    const int grid_x = (l->d.out + TN - 1) / TN, grid_y = (batch + kTfM - 1) / kTfM;
+    if (cfi_status_t e = set_smem<cfi_dense_tf32_kernel<TN>>(tf_smem_bytes(TN), l->device)) return e;
+    return launch_pdl_cluster(cfi_dense_tf32_kernel<TN>, dim3(grid_x, grid_y, split), kTfThreads, tf_smem_bytes(TN), split, st,
+                              l->d, map_x, map_w, static_cast<float*>(y), batch);
+}
+
 cfi_status_t launch_dense_tf32(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
-    const int grid_x = (l->d.out + kTfN - 1) / kTfN, grid_y = (batch + kTfM - 1) / kTfM;
-    if (grid_y > 65535) return CFI_ERR_SHAPE;
+    if ((batch + kTfM - 1) / kTfM > 65535) return CFI_ERR_SHAPE;
     CUtensorMap map_x;
     if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 4, kTfM)) return CFI_ERR_SHAPE;
-    if (cfi_status_t e = set_smem<cfi_dense_tf32_kernel>(kTfSmemBytes, l->device)) return e;
-    const int split = tf32_shape(l, batch).split;
-    return launch_pdl_cluster(cfi_dense_tf32_kernel, dim3(grid_x, grid_y, split), kTfThreads, kTfSmemBytes, split, st, l->d,
-                              map_x, l->map_w, static_cast<float*>(y), batch);
+    const Tf32Shape sh = tf32_shape(l, batch);
+    if (sh.tile_n == 128) return launch_dense_tf32_n<128>(l, map_x, l->map_w_wide, sh.split, y, batch, st);
+    return launch_dense_tf32_n<64>(l, map_x, l->map_w, sh.split, y, batch, st);
 }
 
 cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
@@ -1199,7 +1228,7 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
         // ---- dense copy for the tensor-core variant (zero rows for ablated and padding rows): bf16 for bf16 layers,
         // fp32 for fp32 layers.  A column kept twice in one row cannot be one dense entry, so such layers go without.
         {
-            const int eb = dtype == CFI_BF16 ? 2 : 4, tile_n = dtype == CFI_BF16 ? kTcN : kTfN;
+            const int eb = dtype == CFI_BF16 ? 2 : 4, tile_n = 128;
             bool usable = out_features > 0 && in_features * eb >= 16 && ((in_features * eb) & 15) == 0 &&
                           ((out_features * eb) & 15) == 0 && (size_t)out_features * in_features * eb <= ((size_t)1 << 30);
             for (int32_t r = 0; usable && r < n_active; ++r)
@@ -1227,7 +1256,9 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                 }
                 l->w_dense = wd_dev;
                 l->tc_ok = st == CFI_OK && encode_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb,
-                                                      dtype == CFI_BF16 ? kTcN : kTfN);
+                                                      dtype == CFI_BF16 ? kTcN : 64);
+                if (l->tc_ok && dtype == CFI_F32)  // the same copy in boxes of 128 rows for the wide tile
+                    l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb, 128);
             }
         }
 
@@ -1261,6 +1292,19 @@ extern "C" cfi_status_t cfi_destroy(cfi_layer_t* layer) {
 extern "C" cfi_status_t cfi_choose_variant(const cfi_layer_t* layer, int32_t batch, int32_t* variant) {
     if (!layer || !variant) return CFI_ERR_NULL;
     *variant = choose_variant(layer, batch);
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_dense_tile_shape(const cfi_layer_t* layer, int32_t batch, int32_t* tile_n, int32_t* cluster) {
+    if (!layer || !tile_n || !cluster) return CFI_ERR_NULL;
+    if (!layer->tc_ok || batch < 1) return CFI_ERR_SHAPE;
+    DeviceGuard g(layer->device);
+    if (layer->dtype == CFI_BF16) {
+        *tile_n = kTcN, *cluster = 1;
+    } else {
+        const Tf32Shape sh = tf32_shape(layer, batch);
+        *tile_n = sh.tile_n, *cluster = sh.split;
+    }
     return CFI_OK;
 }
 

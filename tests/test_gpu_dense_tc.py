@@ -31,6 +31,32 @@ def test_dense_tc_matches_oracle(in_f, out_f, k, nabl, B, act, dtype):
     assert scaled_error(y, y_ref, S) <= TOL[dtype]
 
 
+# (in, out, k, ablated, batch) chosen so that together they run both tile widths and clusters of several sizes.
+TF32_SHAPES = [(3072, 768, 307, 77, 256), (3072, 768, 307, 77, 64), (768, 3072, 77, 0, 256), (768, 3072, 77, 0, 100),
+               (4096, 512, 205, 10, 130), (1000, 72, 100, 5, 257), (520, 640, 52, 30, 128), (768, 3072, 77, 150, 700)]
+
+
+def test_dense_tf32_launch_shapes_cover_wide_tiles_and_clusters():
+    """Every tile width and several cluster sizes occur among TF32_SHAPES (else the cases below prove less than
+    they seem to), and each case matches the oracle."""
+    from paper_2305_02299_b200 import binding as cfi
+    seen = set()
+    for in_f, out_f, k, nabl, B in TF32_SHAPES:
+        L = inputs.make_layer(in_f, out_f, k, n_ablated=nabl, seed=in_f + out_f)
+        x = inputs.make_x(B, in_f, seed=B)
+        y_ref, S = oracle_layer(L, x, "f32", "gelu")
+        dl = device_layer(L, "f32", "gelu")
+        shape = cfi.cfi_dense_tile_shape(dl, B)
+        seen.add(shape)
+        y = run_device(dl, x, "f32", "dense_tc")
+        dl.close()
+        assert scaled_error(y, y_ref, S) <= TOL["f32"], (in_f, out_f, B, shape)
+    tiles = {t for t, _ in seen}
+    clusters = {c for _, c in seen}
+    assert tiles == {64, 128}, seen
+    assert 1 in clusters and len([c for c in clusters if c > 1]) >= 2, seen
+
+
 def test_dense_tf32_wide_dynamic_range():
     """Inputs spread over many binades: the split must hold for every magnitude, not only for N(0,1)."""
     L = inputs.make_layer(512, 128, 51, n_ablated=7, seed=9)
