@@ -146,15 +146,16 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (tid >= 64 && tid < 64 + TN) {
-        const int n = n0 + tid - 64;
-        bias_s[tid - 64] = n < L.out ? L.bias[n] : 0.0f;
-    }
+    // The bias is read only after the main loop (and after a barrier), so its load from global memory is issued
+    // here and lands in shared memory after the prologue's barrier instead of holding it up.
+    float bias_v = 0.0f;
+    if (tid >= 64 && tid < 64 + TN && n0 + tid - 64 < L.out) bias_v = L.bias[n0 + tid - 64];
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();  // x and y may belong to the kernel before this one
+    if (tid >= 64 && tid < 64 + TN) bias_s[tid - 64] = bias_v;
     bool ok = true;
 
     if (warp == 0 && lane == 0) {
