@@ -61,7 +61,7 @@ struct cfi_layer {
     int out_pad = 0;
     bool tc_ok = false;
     CUtensorMap map_w{};       // dense copy in boxes of 128 rows (bf16) or 64 rows (fp32)
-    CUtensorMap map_w_wide{};  // fp32 only: boxes of 128 rows
+    CUtensorMap map_w_wide{};  // boxes of 128 rows (fp32) or 256 rows (bf16) for the wide tiles
 };
 
 struct cfi_stack {
@@ -616,6 +616,7 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 
 #include "cfi_dense_tc.cuh"
 #include "cfi_dense_tf32.cuh"
+#include "cfi_dense_tc_persistent.cuh"
 
 // ------------------------------------------------------------------------------------------------
 // host: launch shapes
@@ -945,6 +946,12 @@ cfi_status_t launch_dense_tf32(const cfi_layer* l, const void* x, void* y, int b
     return launch_dense_tf32_n<64>(l, map_x, l->map_w, sh.split, y, batch, st);
 }
 
+// bf16: with at least two 128 x 256 tiles per SM the persistent kernel runs, else one 128 x 128 tile per CTA.
+bool tc_bf16_persistent(const cfi_layer* l, int batch) {
+    const int64_t n_tiles = (int64_t)((l->d.out + kTpN - 1) / kTpN) * ((batch + kTcM - 1) / kTcM);
+    return n_tiles >= 2 * (int64_t)l->sm_count && n_tiles < (1ll << 31);
+}
+
 cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
     if (!l->tc_ok) return CFI_ERR_SHAPE;
     if (l->dtype != CFI_BF16) return launch_dense_tf32(l, x, y, batch, st);
@@ -952,6 +959,21 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
     if (grid_y > 65535) return CFI_ERR_SHAPE;
     CUtensorMap map_x;
     if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 2, kTcM)) return CFI_ERR_SHAPE;
+    // Many tiles per SM: one persistent CTA per SM with 128 x 256 tiles that overlaps each tile's epilogue with the
+    // next tile's MMAs.
+    const int wide_x = (l->d.out + kTpN - 1) / kTpN;
+    const int64_t n_tiles = (int64_t)wide_x * grid_y;
+    if (tc_bf16_persistent(l, batch)) {
+        const int ctas = l->sm_count;
+        if (l->d.act == CFI_ACT_GELU_ERF) {
+            if (cfi_status_t e = set_smem<cfi_dense_tc_persistent_kernel<CFI_ACT_GELU_ERF>>(kTpSmemBytes, l->device)) return e;
+            return launch_pdl(cfi_dense_tc_persistent_kernel<CFI_ACT_GELU_ERF>, dim3(ctas), kTpThreads, kTpSmemBytes, st, l->d,
+                              map_x, l->map_w_wide, static_cast<__nv_bfloat16*>(y), batch, wide_x, (int)n_tiles);
+        }
+        if (cfi_status_t e = set_smem<cfi_dense_tc_persistent_kernel<CFI_ACT_NONE>>(kTpSmemBytes, l->device)) return e;
+        return launch_pdl(cfi_dense_tc_persistent_kernel<CFI_ACT_NONE>, dim3(ctas), kTpThreads, kTpSmemBytes, st, l->d, map_x,
+                          l->map_w_wide, static_cast<__nv_bfloat16*>(y), batch, wide_x, (int)n_tiles);
+    }
     if (l->d.act == CFI_ACT_GELU_ERF) {
         if (cfi_status_t e = set_smem<cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>>(kTcSmemBytes, l->device)) return e;
         return launch_pdl(cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d,
@@ -1257,8 +1279,9 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                 l->w_dense = wd_dev;
                 l->tc_ok = st == CFI_OK && encode_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb,
                                                       dtype == CFI_BF16 ? kTcN : 64);
-                if (l->tc_ok && dtype == CFI_F32)  // the same copy in boxes of 128 rows for the wide tile
-                    l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb, 128);
+                if (l->tc_ok)  // the same copy in the boxes of the wide tiles: 128 rows (fp32), 256 rows (bf16)
+                    l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb,
+                                          dtype == CFI_BF16 ? kTpN : 128);
             }
         }
 
@@ -1300,7 +1323,7 @@ extern "C" cfi_status_t cfi_dense_tile_shape(const cfi_layer_t* layer, int32_t b
     if (!layer->tc_ok || batch < 1) return CFI_ERR_SHAPE;
     DeviceGuard g(layer->device);
     if (layer->dtype == CFI_BF16) {
-        *tile_n = kTcN, *cluster = 1;
+        *tile_n = tc_bf16_persistent(layer, batch) ? kTpN : kTcN, *cluster = 1;
     } else {
         const Tf32Shape sh = tf32_shape(layer, batch);
         *tile_n = sh.tile_n, *cluster = sh.split;

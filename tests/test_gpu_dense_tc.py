@@ -57,6 +57,27 @@ def test_dense_tf32_launch_shapes_cover_wide_tiles_and_clusters():
     assert 1 in clusters and len([c for c in clusters if c > 1]) >= 2, seen
 
 
+@pytest.mark.parametrize("in_f,out_f,k,nabl,B,act", [(768, 1000, 77, 50, 9601, "gelu"), (1024, 512, 102, 0, 19001, "none"),
+                                                     (200, 2048, 20, 100, 4801, "gelu"), (768, 3072, 77, 154, 7000, "gelu")])
+def test_dense_tc_bf16_many_tiles_per_sm(in_f, out_f, k, nabl, B, act):
+    """Enough 128 x 256 tiles for the persistent bf16 kernel (at least two per SM): ragged last batch tile and last
+    output tile (also one that ends in the first half of a tile), ablated rows, more tiles than CTAs so that both
+    accumulator buffers and the bias buffer are reused."""
+    from paper_2305_02299_b200 import binding as cfi
+    L = inputs.make_layer(in_f, out_f, k, n_ablated=nabl, seed=B)
+    x = inputs.make_x(B, in_f, seed=B + 1)
+    y_ref, S = oracle_layer(L, x, "bf16", act)
+    dl = device_layer(L, "bf16", act)
+    assert cfi.cfi_dense_tile_shape(dl, B) == (256, 1)
+    assert cfi.cfi_dense_tile_shape(dl, 256) == (128, 1)
+    y = run_device(dl, x, "bf16", "dense_tc")
+    y2 = run_device(dl, x, "bf16", "dense_tc")
+    dl.close()
+    assert np.all(np.isfinite(y))
+    assert scaled_error(y, y_ref, S) <= TOL["bf16"]
+    assert np.array_equal(y, y2)
+
+
 def test_dense_tf32_wide_dynamic_range():
     """Inputs spread over many binades: the split must hold for every magnitude, not only for N(0,1)."""
     L = inputs.make_layer(512, 128, 51, n_ablated=7, seed=9)
