@@ -91,6 +91,46 @@ cfi_status_t cfi_pack(const float* w_dense, const uint8_t* mask, int32_t out_fea
                       int32_t* k, int32_t* n_active, float* values, int32_t* indices, int32_t* active_rows);
 
 /*
+ * cfi_compact_producer / cfi_compact_consumer — the paper's own output form, host only.
+ * (Algorithm 1 returns (batch, active_neurons): Sec. 4.4 removes ablated neurons from the layer altogether, where
+ *  cfi_forward writes all out_features columns with act(bias) in the ablated ones.)
+ *
+ * A layer in compact form is an ordinary layer for cfi_create with out_features = n_active and
+ * active_rows = 0 .. n_active-1; its output is the full-width output with the ablated columns deleted.
+ * cfi_compact_producer writes that layer's bias and row list:
+ *
+ *   bias          host, float [out_features] or NULL (= zeros)
+ *   active_rows   host, int32 [n_active], each in [0, out_features), no repeats
+ *   bias_compact  host, float [n_active], written:  bias_compact[r] = bias[active_rows[r]]
+ *   rows_compact  host, int32 [n_active], written:  0, 1, ..., n_active-1
+ *
+ * cfi_compact_consumer rewrites, in place, the layer that reads such an output (its in_features become the
+ * producer's n_active):
+ *
+ *   prod_active_rows, prod_n_active, prod_out   the producer's row list (as above) and full width
+ *   prod_const    host, float [prod_out] or NULL (= zeros): what the producer emits in each of its columns when
+ *                 that column is ablated, i.e. act(bias) in the producer's storage precision; only ablated entries
+ *                 are read
+ *   values        host, float [n_active, k], in/out
+ *   indices       host, int32 [n_active, k], in/out: full-width columns in, compact columns out
+ *   active_rows   host, int32 [n_active]: the consumer's own row list (selects the bias entry of a row)
+ *   bias          host, float [out_features], in/out
+ *
+ * An entry that reads an active column c of the producer gets the compact column (the rank of c in
+ * prod_active_rows).  An entry that reads an ablated column multiplied a constant: values * prod_const[c] is added
+ * (in fp32) to the bias of the entry's row, the value becomes 0 and the index the smallest compact column the row
+ * does not use yet, so that fan-in stays constant and no column repeats.  The result equals the full-width pair of
+ * layers up to the rounding of those bias updates.
+ * CFI_ERR_NULL, CFI_ERR_SHAPE (negative sizes, k > prod_n_active), CFI_ERR_INDEX_RANGE (an index or row number out
+ * of range, a repeated producer row).
+ */
+cfi_status_t cfi_compact_producer(const float* bias, const int32_t* active_rows, int32_t n_active, int32_t out_features,
+                                  float* bias_compact, int32_t* rows_compact);
+cfi_status_t cfi_compact_consumer(const int32_t* prod_active_rows, int32_t prod_n_active, int32_t prod_out,
+                                  const float* prod_const, float* values, int32_t* indices, const int32_t* active_rows,
+                                  int32_t n_active, int32_t k, float* bias, int32_t out_features);
+
+/*
  * cfi_create — build a device-resident layer from condensed arrays (the inputs w and indx of
  * Algorithm 1, plus the bias that Sec. 4.4 extracts with the weights).
  *

@@ -24,7 +24,7 @@ _DTYPES = {"f32": F32, "fp32": F32, "float32": F32, "bf16": BF16, "bfloat16": BF
 _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE, ACT_GELU: ACT_GELU}
 _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
 
-EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
+EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_dense_tile_shape", "cfi_device_status", "cfi_destroy",
            "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static",
            "cfi_probe_device")
@@ -69,6 +69,8 @@ def _load() -> ctypes.CDLL:
     lib.cfi_status_string.restype = ctypes.c_char_p
     lib.cfi_status_string.argtypes = [ctypes.c_int]
     lib.cfi_pack.argtypes = [f32p, u8p, ci, ci, i32p, i32p, f32p, i32p, i32p]
+    lib.cfi_compact_producer.argtypes = [f32p, i32p, ci, ci, f32p, i32p]
+    lib.cfi_compact_consumer.argtypes = [i32p, ci, ci, f32p, f32p, i32p, i32p, ci, ci, f32p, ci]
     lib.cfi_create.argtypes = [f32p, i32p, i32p, f32p, ci, ci, ci, ci, ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
     lib.cfi_forward.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_forward_variant.argtypes = [vp, vp, vp, ci, vp, ctypes.c_int]
@@ -181,6 +183,31 @@ def cfi_create(values, indices, active_rows, bias, in_features: int, out_feature
                            _hp(b, ctypes.c_float), n_active, k, in_features, out_features, _DTYPES[dtype],
                            _ACTS[act], ctypes.byref(h)), "cfi_create")
     return Layer(h.value, in_features, out_features, _DTYPES[dtype])
+
+
+def cfi_compact_producer(bias, active_rows, out_features: int):
+    """(bias_compact, rows_compact) of the layer in the paper's compact output form (ablated columns removed)."""
+    rows = np.ascontiguousarray(active_rows, dtype=np.int32)
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    bc, rc = np.empty(rows.shape[0], np.float32), np.empty(rows.shape[0], np.int32)
+    _check(_lib.cfi_compact_producer(_hp(b, ctypes.c_float), _hp(rows, ctypes.c_int32), rows.shape[0], out_features,
+                                     _hp(bc, ctypes.c_float), _hp(rc, ctypes.c_int32)), "cfi_compact_producer")
+    return bc, rc
+
+
+def cfi_compact_consumer(prod_active_rows, prod_out: int, prod_const, values, indices, active_rows, bias):
+    """Returns (values, indices, bias) of the layer that reads a compact output; inputs are not modified."""
+    pr = np.ascontiguousarray(prod_active_rows, dtype=np.int32)
+    pc = None if prod_const is None else np.ascontiguousarray(prod_const, dtype=np.float32)
+    v = np.array(values, dtype=np.float32, order="C", copy=True)
+    ix = np.array(indices, dtype=np.int32, order="C", copy=True)
+    rows = np.ascontiguousarray(active_rows, dtype=np.int32)
+    b = np.array(bias, dtype=np.float32, order="C", copy=True)
+    n_active, k = v.shape
+    _check(_lib.cfi_compact_consumer(_hp(pr, ctypes.c_int32), pr.shape[0], prod_out, _hp(pc, ctypes.c_float),
+                                     _hp(v, ctypes.c_float), _hp(ix, ctypes.c_int32), _hp(rows, ctypes.c_int32), n_active, k,
+                                     _hp(b, ctypes.c_float), b.shape[0]), "cfi_compact_consumer")
+    return v, ix, b
 
 
 def cfi_forward(layer: Layer, x, y, batch: int, stream=None) -> None:
