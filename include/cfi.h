@@ -62,7 +62,8 @@ typedef enum {
     CFI_VARIANT_SPLITK = 2,   /* small batch: lanes split a row's k terms, x staged in shared memory     */
     CFI_VARIANT_BATCH = 3,    /* large batch: lanes own batch columns, x tile transposed in shared memory */
     CFI_VARIANT_DENSE_TC = 4  /* large batch: dense copy of the weight on the tensor cores (tcgen05): bf16 layers
-                                 directly, fp32 layers as three TF32 products of split operands; needs row pitches
+                                 directly, fp32 layers as three TF32 products of split operands (K may be split over a
+                                 thread-block cluster); needs row pitches
                                  of x, y and the weight that are multiples of 16 bytes and no repeated column in a
                                  row, otherwise CFI_ERR_SHAPE */
 } cfi_variant_t;

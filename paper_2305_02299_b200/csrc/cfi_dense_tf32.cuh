@@ -8,13 +8,13 @@
 //
 //     a = a_hi + a_lo + r,   a_hi = a with the low 13 mantissa bits cleared,   a_lo = (a - a_hi) likewise cleared,
 //
-// so that |r| < 2^-21 |a|, and the product is taken as  x_hi w_hi + x_hi w_lo + x_lo w_hi  (three MMAs, fp32
-// accumulation in tensor memory).  What is dropped (x_lo w_lo and the two remainders) is below 2^-19 of the
+// so that |r| < 2^-21 |a|, and the product is taken as  x_hi w_hi + x_hi w_lo + x_lo w_hi  (three products in
+// two MMAs, fp32 accumulation in tensor memory).  What is dropped (x_lo w_lo and the two remainders) is below 2^-19 of the
 // term, fifty times inside the tolerance.  Because both parts are exactly representable in TF32, the result
 // does not depend on how the tensor core would convert a general fp32 operand.
 //
 // The layer keeps one dense fp32 copy of its weight, Wd[out_pad][in].  Per 32-column block of K:
-//   warp 0, one lane   TMA: a 128 x 32 box of x and a 64 x 32 box of Wd (fp32, 128-byte swizzle) into a ring slot;
+//   warp 0, one lane   TMA: a 128 x 32 box of x and a TN x 32 box of Wd (fp32, 128-byte swizzle) into a ring slot;
 //   warps 2..17        four groups of four warps; group g takes the blocks kb = g (mod 4), so four blocks are being
 //                      split at once.  A thread reads its batch row of the x box from shared memory and writes
 //                      hi and lo straight into tensor memory (tcgen05.st), from where the MMA takes its A
@@ -22,15 +22,20 @@
 //                      splits the Wd box in shared memory, hi in place and lo beside it (element-wise, so the
 //                      swizzled layout is untouched), and makes those writes visible to the tensor core
 //                      (fence.proxy.async);
-//   warp 1, one lane   once the group's 128 threads have arrived on the slot's "ready" barrier:
-//                      4 K-steps x 3 tcgen05.mma (kind::tf32, M = 128, N = 64, K = 8, A from tensor memory, B
-//                      from shared memory), then tcgen05.commit frees the slot;
-// and after the last block warps 2..17 run the epilogue: tcgen05.ld, bias, activation, y tile through shared
-// memory, 256-byte runs per batch row.  Tensor memory: columns 0..63 accumulator, then per slot 32 columns of
-// x_hi and 32 of x_lo.  All mbarrier waits are bounded (status code 2), as in the bf16 kernel.
+//   warp 1, one lane   once the group's 128 threads have arrived on the slot's "ready" barrier: 4 K-steps x 2
+//                      tcgen05.mma (kind::tf32, M = 128, K = 8, A from tensor memory, B from shared memory): Wd lo
+//                      lies right behind Wd hi, so x_hi x [Wd hi; Wd lo] is one MMA of N = 2 TN (the two products
+//                      land in accumulator columns 0..TN-1 and TN..2TN-1) and x_lo x Wd hi a second of N = TN onto
+//                      the first half; then tcgen05.commit frees the slot.  (An MMA costs about 50 cycles + 0.43 per
+//                      column of N here, so fewer and wider MMAs win; hence also the tile width TN = 128 where the
+//                      shape gives enough tiles.)
+// and after the last block warps 2..17 run the epilogue: tcgen05.ld of both accumulator halves, their sum, bias,
+// activation, y tile through shared memory, runs of 4 TN bytes per batch row.  Tensor memory: 2 TN accumulator
+// columns, then per slot 32 columns of x_hi and 32 of x_lo.  All mbarrier waits are bounded (status code 2), as in
+// the bf16 kernel.
 //
 // Split K over a thread-block cluster: a layer with few output tiles and a long K (3072 -> 768 at batch 256 has 24
-// tiles of 96 K blocks) would leave most SMs idle, so the launch may give each tile to a cluster of 2, 4 or 8 CTAs
+// tiles of 96 K blocks) would leave most SMs idle, so the launch may give each tile to a cluster of up to 8 CTAs
 // (cluster dimension z).  CTA r of the cluster contracts the r-th share of the K blocks; the partial tiles are left
 // in each CTA's shared memory, and after a cluster barrier CTA r sums rows [128 r / S, 128 (r + 1) / S) of all S
 // partial tiles in rank order through distributed shared memory, adds the bias, applies the activation and stores
