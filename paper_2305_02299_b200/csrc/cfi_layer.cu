@@ -946,10 +946,11 @@ cfi_status_t launch_dense_tf32(const cfi_layer* l, const void* x, void* y, int b
     return launch_dense_tf32_n<64>(l, map_x, l->map_w, sh.split, y, batch, st);
 }
 
-// bf16: with at least two 128 x 256 tiles per SM the persistent kernel runs, else one 128 x 128 tile per CTA.
+// bf16: with at least one 128 x 256 tile per SM the persistent kernel runs (measured: faster from about there
+// on), else one 128 x 128 tile per CTA.
 bool tc_bf16_persistent(const cfi_layer* l, int batch) {
     const int64_t n_tiles = (int64_t)((l->d.out + kTpN - 1) / kTpN) * ((batch + kTcM - 1) / kTcM);
-    return n_tiles >= 2 * (int64_t)l->sm_count && n_tiles < (1ll << 31);
+    return n_tiles >= (int64_t)l->sm_count && n_tiles < (1ll << 31);
 }
 
 cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
@@ -959,8 +960,8 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
     if (grid_y > 65535) return CFI_ERR_SHAPE;
     CUtensorMap map_x;
     if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 2, kTcM)) return CFI_ERR_SHAPE;
-    // Many tiles per SM: one persistent CTA per SM with 128 x 256 tiles that overlaps each tile's epilogue with the
-    // next tile's MMAs.
+    // A tile or more per SM: one persistent CTA per SM with 128 x 256 tiles that overlaps each tile's epilogue with
+    // the next tile's MMAs.
     const int wide_x = (l->d.out + kTpN - 1) / kTpN;
     const int64_t n_tiles = (int64_t)wide_x * grid_y;
     if (tc_bf16_persistent(l, batch)) {
