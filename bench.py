@@ -421,6 +421,11 @@ def main():
         line["context"] = context_leg(w, torch)
         line["stack_c5"] = stack_leg(cfi, torch, peaks, sm_count)
         line["batch2048"] = batch2048_leg(W, cfi, torch, l2, peaks, sm_count)
+        # Ceilings measured in this run by the library's own micro-probes (fp32 FMA, L2 read, empty launch).
+        try:
+            line["device_probe"] = cfi.cfi_probe_device().as_dict()
+        except Exception as exc:
+            line["device_probe"] = str(exc)
         line["stack_batch1"] = stack_batch1_leg(cfi, torch, l2, peaks)
     if rank == 0:
         print(json.dumps(line))
