@@ -24,7 +24,7 @@ from typing import Dict, List, Optional, Tuple
 
 import numpy as np
 
-_T_MASK, _T_WEIGHT, _T_BIAS, _T_ABLATE, _T_X = 1, 2, 3, 4, 5
+_T_MASK, _T_WEIGHT, _T_BIAS, _T_ABLATE, _T_X, _T_XI = 1, 2, 3, 4, 5, 6
 
 
 def _rng(seed: int, stream: int, tensor: int) -> np.random.Generator:
@@ -202,3 +202,25 @@ class StackWorkload:
 
     def x(self, seed: int = 0, batch: Optional[int] = None) -> np.ndarray:
         return make_x(self.batch if batch is None else batch, self.d_model, seed=seed, stream=self.stream)
+
+
+# ----------------------------------------------------------------------------
+# Draws for the output-norm-variance simulation (Sec. 3, "Constant Fan-In
+# sparsity"; appendix "Computing the output norm variance", Definition 1):
+# many independent square layers with W ~ N(0,1) iid, exactly k ones per row of
+# I (rows independent, uniform over the k-subsets), xi ~ Ber(1/2)^n and u
+# uniform on the unit sphere.  Only the draws; the scaling sqrt(2/k), the
+# products and the norms are the caller's.
+# ----------------------------------------------------------------------------
+def make_norm_variance_draws(n: int, k: int, layers: int, batch: int, *, seed: int = 0, stream: int = 900):
+    """Returns (w [layers,n,k] f32 ~ N(0,1), cols [layers,n,k] int32 distinct per row and ascending,
+    xi [layers,batch,n] f32 in {0,1}, u [layers,batch,n] f32 with unit rows)."""
+    if not (1 <= k <= n):
+        raise ValueError("need 1 <= k <= n")
+    cols = _choose_columns(_rng(seed, stream, _T_MASK), layers * n, n, k).reshape(layers, n, k)
+    cols = np.sort(cols, axis=2).astype(np.int32)
+    w = _rng(seed, stream, _T_WEIGHT).standard_normal((layers, n, k), dtype=np.float32)
+    xi = (_rng(seed, stream, _T_XI).random((layers, batch, n), dtype=np.float32) < 0.5).astype(np.float32)
+    g = _rng(seed, stream, _T_X).standard_normal((layers, batch, n))
+    u = (g / np.linalg.norm(g, axis=2, keepdims=True)).astype(np.float32)
+    return w, cols, xi, u
