@@ -991,7 +991,18 @@ constexpr double kGatherTflops = 12.5;
 int choose_variant(const cfi_layer* l, int batch) {
     // Up to three batch tiles of 8 the split-k kernel (weights re-read from L2 per tile) beats the 64-wide tiles of
     // the batch kernel, which would be mostly empty.
-    if (batch <= 24) return CFI_VARIANT_SPLITK;
+    if (batch <= 24) {
+        // Two or three passes of the split-k kernel over a large fp32 layer can take longer than the tensor-core
+        // variant does for any batch up to 128 (measured 4096 x 4096 at 80 %, batch 16: 31 against 25 us; 3072 -> 768:
+        // 22 against 11 us).  A pass of eight batch rows costs about 2.3 us plus the larger of staging x (90 ns per KB
+        // of the 8-row tile, every CTA stages all of it) and the weights (176 G entries per second).
+        if (batch > 8 && l->tc_ok && l->dtype == CFI_F32) {
+            const double t_stage = (double)l->d.in * 8 * 4 / 1024.0 * 90e-9, t_fma = (double)l->d.n_active * l->d.k / 176e9;
+            const double t_splitk = ((batch + 7) / 8) * (2.3e-6 + std::max(t_stage, t_fma));
+            if (tf32_shape(l, batch).seconds < t_splitk) return CFI_VARIANT_DENSE_TC;
+        }
+        return CFI_VARIANT_SPLITK;
+    }
     // bf16 at large batch: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
     // (10 TFLOP/s effective for the gather against several hundred dense); below a full 128-row tile it does not pay.
     if (l->tc_ok && l->dtype == CFI_BF16 && batch >= 96) return CFI_VARIANT_DENSE_TC;
