@@ -203,7 +203,7 @@ cfi_status_t cfi_choose_variant(const cfi_layer_t* layer, int32_t batch, int32_t
 /*
  * Launch shape CFI_VARIANT_DENSE_TC would use for this batch size: outputs per tile (*tile_n: 64 or 128 for fp32
  * layers; 128, or 256 for the persistent kernel, for bf16 layers) and the number of CTAs that share one output tile
- * by splitting K over a thread-block cluster (*cluster: 1 .. 8; always 1 for bf16 layers).  An introspection call for tests and benchmarks; the paper has no counterpart.
+ * by splitting K over a thread-block cluster (*cluster: 1 .. 8).  An introspection call for tests and benchmarks; the paper has no counterpart.
  * CFI_ERR_SHAPE if the layer has no dense copy (see CFI_VARIANT_DENSE_TC), CFI_ERR_NULL on a NULL argument.
  */
 cfi_status_t cfi_dense_tile_shape(const cfi_layer_t* layer, int32_t batch, int32_t* tile_n, int32_t* cluster);

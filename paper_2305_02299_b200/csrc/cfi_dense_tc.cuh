@@ -30,6 +30,12 @@
 // Every mbarrier wait is bounded.  If one expires the thread records code 2 in the layer's status word and
 // leaves its role's loop; all roles still meet at the final barrier, tensor memory is freed and the kernel
 // returns.
+//
+// With few tiles and a long K the launch may give each tile to a thread-block cluster of up to 8 CTAs (cluster
+// dimension z): CTA r contracts the r-th share of the K blocks and leaves its fp32 partial tile (no bias) in its
+// shared memory; after the hardware cluster barrier CTA r sums rows [128 r / S, 128 (r + 1) / S) of all S partial
+// tiles in rank order through distributed shared memory, adds the bias, applies the activation, rounds to bf16
+// and stores; a second cluster barrier keeps every CTA's shared memory alive until its peers have read it.
 
 #include <cuda.h>  // CUtensorMap and the enums of cuTensorMapEncodeTiled (types only; the entry point is looked up at run time)
 
@@ -102,6 +108,35 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "memory");
 }
 
+// Thread-block cluster helpers (K split over a cluster, see below and cfi_dense_tf32.cuh).
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+// Every thread of every CTA of the cluster; writes to shared memory before it are visible to reads through
+// distributed shared memory after it.
+__device__ __forceinline__ void cluster_sync_all() {
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// 16 bytes at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float4 v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(remote)
+                 : "memory");
+    return v;
+}
+
 // Activation for the epilogue, chosen at compile time.  GELU is v * Phi(v) with Phi = (1 + erf(v / sqrt 2)) / 2;
 // erf is evaluated with the rational-times-Gaussian formula of Abramowitz & Stegun 7.1.26 (absolute error
 // below 1.5e-7, far inside a bf16 result), with the factors 1/sqrt 2 and 1/2 folded into its constants, and
@@ -140,7 +175,11 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_at(ctl + 72));
     float* bias_s = reinterpret_cast<float*>(smem_at(ctl + 128));
     const int m0 = blockIdx.y * kTcM, n0 = blockIdx.x * kTcN;
-    const int k_blocks = (L.in + kTcK - 1) / kTcK;
+    const int k_blocks_all = (L.in + kTcK - 1) / kTcK;
+    // This CTA's share of the K blocks: [kb0, kb0 + k_blocks).
+    const int split = (int)cluster_rank(), n_split = (int)cluster_size();
+    const int kb0 = (int)(((int64_t)k_blocks_all * split) / n_split);
+    const int k_blocks = (int)(((int64_t)k_blocks_all * (split + 1)) / n_split) - kb0;
 
     if (tid == 0) {
         for (int s = 0; s < kTcStages; ++s) {
@@ -174,8 +213,8 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
             if (!ok) break;
             const uint32_t a_dst = smem_u32(ring + s * kTcStageBytes), b_dst = a_dst + kTcM * kTcK * 2;
             mbar_expect_tx(full0 + 8 * s, kTcStageBytes);
-            tma_load_2d(a_dst, &map_x, full0 + 8 * s, kb * kTcK, m0);
-            tma_load_2d(b_dst, &map_w, full0 + 8 * s, kb * kTcK, n0);
+            tma_load_2d(a_dst, &map_x, full0 + 8 * s, (kb0 + kb) * kTcK, m0);
+            tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + kb) * kTcK, n0);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
@@ -199,7 +238,24 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
         const int q = warp & 3;            // a warp may read the tensor-memory lanes 32 q .. 32 q + 31
         const int half = (warp - 2) >> 2;  // two warps share a lane quarter and split the 128 columns
         const int row = 32 * q + lane;     // batch row of the tile held by this thread
-        if (ok) {
+        if (ok && n_split > 1) {
+            // Partial tile, fp32, no bias: 128 rows x 512 bytes, 16-byte chunks permuted by chunk ^ (row & 15).
+#pragma unroll 1
+            for (int c = 64 * half; c < 64 * half + 64; c += 16) {
+                uint32_t v[16];
+                tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int e4 = 0; e4 < 4; ++e4) {
+                    float4 r = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    if (k_blocks > 0)  // a CTA without K blocks has issued no MMA: its accumulator holds nothing
+                        r = make_float4(__uint_as_float(v[4 * e4]), __uint_as_float(v[4 * e4 + 1]), __uint_as_float(v[4 * e4 + 2]),
+                                        __uint_as_float(v[4 * e4 + 3]));
+                    const int ch = (c >> 2) + e4;
+                    *reinterpret_cast<float4*>(smem_at(ring + row * 512 + ((ch ^ (row & 15)) << 4))) = r;
+                }
+            }
+        } else if (ok) {
             // y tile in shared memory: 128 rows x 256 bytes, 16-byte chunks permuted by chunk ^ (row & 15).
 #pragma unroll 1
             for (int c = 64 * half; c < 64 * half + 64; c += 32) {
@@ -229,8 +285,8 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
                 }
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * kTcEpilogueWarps) : "memory");  // the epilogue warps only
-        if (ok) {
+        if (n_split == 1) asm volatile("bar.sync 1, %0;" ::"n"(32 * kTcEpilogueWarps) : "memory");  // the epilogue warps only
+        if (ok && n_split == 1) {
             const int et = tid - 64;  // 16 threads per row, 16 rows per pass
             for (int r = et >> 4; r < kTcM; r += 2 * kTcEpilogueWarps) {
                 const int ch = et & 15, m = m0 + r, n = n0 + 8 * ch;
@@ -240,6 +296,32 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
                 }
             }
         }
+    }
+    if (n_split > 1) {
+        // Every thread of every CTA of the cluster passes both barriers, whatever `ok` says.
+        cluster_sync_all();  // the partial tiles are complete
+        if (warp >= 2 && ok) {
+            // Rows [split * rows_per, (split + 1) * rows_per): sum over the cluster in rank order, bias, activation,
+            // bf16, store.  32 threads per row (4 columns each), 8 rows per pass, 256-byte runs.
+            const int et = tid - 64, ch = et & 31, rows_per = (kTcM + n_split - 1) / n_split, n = n0 + 4 * ch;
+            const float4 bv = *reinterpret_cast<const float4*>(bias_s + 4 * ch);
+            for (int rr = et >> 5; rr < rows_per; rr += kTcEpilogueWarps) {
+                const int r = split * rows_per + rr, m = m0 + r;
+                if (r < kTcM && m < batch && n < L.out) {
+                    const uint32_t off = smem_u32(ring + r * 512 + ((ch ^ (r & 15)) << 4));
+                    float4 a = ld_cluster_f4(off, 0u);
+                    for (int p = 1; p < n_split; ++p) {
+                        const float4 t = ld_cluster_f4(off, (uint32_t)p);
+                        a.x += t.x, a.y += t.y, a.z += t.z, a.w += t.w;
+                    }
+                    const __nv_bfloat162 p01 = __floats2bfloat162_rn(activate_tc<ACT>(a.x + bv.x), activate_tc<ACT>(a.y + bv.y));
+                    const __nv_bfloat162 p23 = __floats2bfloat162_rn(activate_tc<ACT>(a.z + bv.z), activate_tc<ACT>(a.w + bv.w));
+                    *reinterpret_cast<uint2*>(y + (size_t)m * L.out + n) =
+                        make_uint2(*reinterpret_cast<const uint32_t*>(&p01), *reinterpret_cast<const uint32_t*>(&p23));
+                }
+            }
+        }
+        cluster_sync_all();  // no CTA leaves while another may still read its tile
     }
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

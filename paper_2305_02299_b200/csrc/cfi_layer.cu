@@ -197,7 +197,7 @@ __device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
 // A lane keeps U = 4 16-byte vector pairs (weights + indices) in flight in registers; the rest of the row is
 // on its way into L2.  XS = loads of x in flight per thread while staging (8 where few threads stage a long x).
 template <typename VT, int BT, int G, int XS>
-__global__ void cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch,
+__global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch,
                                   int rows_per_group) {
     extern __shared__ __align__(16) float xs_f32[];  // [(in + 1)][BT]
     float* xs = xs_f32;
@@ -953,6 +953,54 @@ bool tc_bf16_persistent(const cfi_layer* l, int batch) {
     return n_tiles >= (int64_t)l->sm_count && n_tiles < (1ll << 31);
 }
 
+// Clusters of `split` CTAs of the one-tile bf16 kernel that the device can hold at once; 0 if it cannot launch that
+// cluster size (cached per device; -1 in the cache stands for 0).  Both activations have the same footprint.
+int tc_bf16_resident_clusters(const cfi_layer* l, int split) {
+    static std::atomic<int> cache[64][kTfMaxSplit + 1];
+    if (split == 1) return std::max(1, 2 * l->sm_count);
+    if (l->device < 0 || l->device >= 64) return 0;
+    std::atomic<int>& c = cache[l->device][split];
+    int v = c.load(std::memory_order_acquire);
+    if (v == 0) {
+        v = -1;
+        if (set_smem<cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>>(kTcSmemBytes, l->device) == CFI_OK) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3(1, 1, (unsigned)split);
+            cfg.blockDim = dim3(kTcThreads);
+            cfg.dynamicSmemBytes = kTcSmemBytes;
+            cudaLaunchAttribute attr{};
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 1, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = (unsigned)split;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>, &cfg) == cudaSuccess && n > 0) v = n;
+            else cudaGetLastError();
+        }
+        c.store(v, std::memory_order_release);
+    }
+    return v > 0 ? v : 0;
+}
+
+// K split of the one-tile bf16 kernel: as for the split-TF32 kernel, a time model over the cluster sizes (seconds
+// per 64-column block of K, a fixed part per wave of CTAs, the cluster reduction, the launch; measured).
+int tc_bf16_split(const cfi_layer* l, int batch, double* seconds = nullptr) {
+    const int64_t tiles = (int64_t)((batch + kTcM - 1) / kTcM) * ((l->d.out + kTcN - 1) / kTcN);
+    const int k_blocks = (l->d.in + kTcK - 1) / kTcK;
+    int best = 1;
+    double best_t = 0.0;
+    for (int split = 1; split <= kTfMaxSplit; ++split) {
+        if (split > 1 && (k_blocks < 4 * split || tiles * split > 4 * (int64_t)l->sm_count)) break;
+        const int64_t resident = tc_bf16_resident_clusters(l, split);
+        if (resident == 0) continue;
+        const int64_t waves = (tiles + resident - 1) / resident;
+        const double t = (double)waves * (((k_blocks + split - 1) / split) * 0.27e-6 + 3.0e-6 + (split > 1 ? 1.0e-6 : 0.0)) + 0.7e-6;
+        if (split == 1 || t < best_t) best = split, best_t = t;
+    }
+    if (seconds) *seconds = best_t;
+    return best;
+}
+
 cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
     if (!l->tc_ok) return CFI_ERR_SHAPE;
     if (l->dtype != CFI_BF16) return launch_dense_tf32(l, x, y, batch, st);
@@ -975,14 +1023,15 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
         return launch_pdl(cfi_dense_tc_persistent_kernel<CFI_ACT_NONE>, dim3(ctas), kTpThreads, kTpSmemBytes, st, l->d, map_x,
                           l->map_w_wide, static_cast<__nv_bfloat16*>(y), batch, wide_x, (int)n_tiles);
     }
+    const int split = tc_bf16_split(l, batch);
     if (l->d.act == CFI_ACT_GELU_ERF) {
         if (cfi_status_t e = set_smem<cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>>(kTcSmemBytes, l->device)) return e;
-        return launch_pdl(cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d,
-                          map_x, l->map_w, static_cast<__nv_bfloat16*>(y), batch);
+        return launch_pdl_cluster(cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>, dim3(grid_x, grid_y, split), kTcThreads, kTcSmemBytes,
+                                  split, st, l->d, map_x, l->map_w, static_cast<__nv_bfloat16*>(y), batch);
     }
     if (cfi_status_t e = set_smem<cfi_dense_tc_kernel<CFI_ACT_NONE>>(kTcSmemBytes, l->device)) return e;
-    return launch_pdl(cfi_dense_tc_kernel<CFI_ACT_NONE>, dim3(grid_x, grid_y), kTcThreads, kTcSmemBytes, st, l->d, map_x,
-                      l->map_w, static_cast<__nv_bfloat16*>(y), batch);
+    return launch_pdl_cluster(cfi_dense_tc_kernel<CFI_ACT_NONE>, dim3(grid_x, grid_y, split), kTcThreads, kTcSmemBytes, split, st,
+                              l->d, map_x, l->map_w, static_cast<__nv_bfloat16*>(y), batch);
 }
 
 // Rate of the gather kernel's arithmetic, used to choose between it and the split-TF32 dense kernel (measured).
@@ -996,16 +1045,20 @@ int choose_variant(const cfi_layer* l, int batch) {
         // variant does for any batch up to 128 (measured 4096 x 4096 at 80 %, batch 16: 31 against 25 us; 3072 -> 768:
         // 22 against 11 us).  A pass of eight batch rows costs about 2.3 us plus the larger of staging x (90 ns per KB
         // of the 8-row tile, every CTA stages all of it) and the weights (176 G entries per second).
-        if (batch > 8 && l->tc_ok && l->dtype == CFI_F32) {
+        if (batch > 8 && l->tc_ok) {
             const double t_stage = (double)l->d.in * 8 * 4 / 1024.0 * 90e-9, t_fma = (double)l->d.n_active * l->d.k / 176e9;
             const double t_splitk = ((batch + 7) / 8) * (2.3e-6 + std::max(t_stage, t_fma));
-            if (tf32_shape(l, batch).seconds < t_splitk) return CFI_VARIANT_DENSE_TC;
+            double t_dense = 0.0;
+            if (l->dtype == CFI_F32) t_dense = tf32_shape(l, batch).seconds;
+            else tc_bf16_split(l, batch, &t_dense);
+            if (t_dense < t_splitk) return CFI_VARIANT_DENSE_TC;
         }
         return CFI_VARIANT_SPLITK;
     }
-    // bf16 at large batch: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
-    // (10 TFLOP/s effective for the gather against several hundred dense); below a full 128-row tile it does not pay.
-    if (l->tc_ok && l->dtype == CFI_BF16 && batch >= 96) return CFI_VARIANT_DENSE_TC;
+    // bf16 above 24 rows: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
+    // (10 TFLOP/s effective for the gather against several hundred dense), also with a partly empty 128-row tile
+    // now that K can be split over a cluster (3072 -> 768 at batch 64: 8.5 against 33 us).
+    if (l->tc_ok && l->dtype == CFI_BF16) return CFI_VARIANT_DENSE_TC;
     if (l->tc_ok && l->dtype == CFI_F32) {
         // fp32: the split-TF32 kernel takes a fixed time per 32-column block of K and tile (it is bound by the
         // number of MMA instructions), whatever the fill of its 128-row batch tile, and can split K over a cluster
@@ -1335,7 +1388,8 @@ extern "C" cfi_status_t cfi_dense_tile_shape(const cfi_layer_t* layer, int32_t b
     if (!layer->tc_ok || batch < 1) return CFI_ERR_SHAPE;
     DeviceGuard g(layer->device);
     if (layer->dtype == CFI_BF16) {
-        *tile_n = tc_bf16_persistent(layer, batch) ? kTpN : kTcN, *cluster = 1;
+        const bool persistent = tc_bf16_persistent(layer, batch);
+        *tile_n = persistent ? kTpN : kTcN, *cluster = persistent ? 1 : tc_bf16_split(layer, batch);
     } else {
         const Tf32Shape sh = tf32_shape(layer, batch);
         *tile_n = sh.tile_n, *cluster = sh.split;

@@ -69,7 +69,7 @@ def test_dense_tc_bf16_many_tiles_per_sm(in_f, out_f, k, nabl, B, act):
     y_ref, S = oracle_layer(L, x, "bf16", act)
     dl = device_layer(L, "bf16", act)
     assert cfi.cfi_dense_tile_shape(dl, B) == (256, 1)
-    assert cfi.cfi_dense_tile_shape(dl, 256) == (128, 1)
+    assert cfi.cfi_dense_tile_shape(dl, 256)[0] == 128   # few tiles: one tile per CTA, K possibly split over a cluster
     y = run_device(dl, x, "bf16", "dense_tc")
     y2 = run_device(dl, x, "bf16", "dense_tc")
     dl.close()

@@ -196,3 +196,13 @@ def test_stack_matches_chained_oracle(dtype):
     st.close()
     for dl in dls:
         dl.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B", [8, 16, 24])
+def test_splitk_long_rows_full_batch_tile(dtype, B):
+    """A long x (4096 columns) with full tiles of eight batch rows: the split-k launch shape with the most threads per
+    CTA and the most registers per thread (bf16 widening); it must launch and match on every tile."""
+    L = inputs.make_layer(4096, 1024, 205, n_ablated=30, seed=B)
+    x = inputs.make_x(B, 4096, seed=B + 3)
+    check_layer(L, x, dtype, "gelu", variants=("splitk",))
