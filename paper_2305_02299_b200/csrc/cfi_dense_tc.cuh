@@ -125,6 +125,12 @@ __device__ __forceinline__ void cluster_sync_all() {
     __syncwarp();
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The same meeting point without ordering any memory: for "every CTA is done reading its peers' shared memory", where
+// nothing is published.  (A releasing arrival would first wait for the CTA's outstanding global stores.)
+__device__ __forceinline__ void cluster_sync_all_relaxed() {
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
 // 16 bytes at the same shared-memory offset in CTA `rank` of the cluster.
 __device__ __forceinline__ float4 ld_cluster_f4(uint32_t local_addr, uint32_t rank) {
     uint32_t remote;
@@ -321,7 +327,7 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
                 }
             }
         }
-        cluster_sync_all();  // no CTA leaves while another may still read its tile
+        cluster_sync_all_relaxed();  // no CTA leaves while another may still read its tile
     }
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

@@ -280,7 +280,7 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             }
         }
     }
-    if (n_split > 1) cluster_sync_all();  // no CTA leaves while another may still read its tile
+    if (n_split > 1) cluster_sync_all_relaxed();  // no CTA leaves while another may still read its tile
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
