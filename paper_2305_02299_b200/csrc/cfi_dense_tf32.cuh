@@ -80,6 +80,34 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         : "memory");
 }
 
+// Sum of the 16 bytes at shared-memory address `addr` over the S CTAs of the cluster, in rank order, for each of
+// ITER rows that are `row_step` bytes apart.  All S * ITER loads are issued before the first sum needs one, so the
+// latency of distributed shared memory is paid once, and the CTA's own tile is read as ordinary shared memory.
+template <int S, int ITER>
+__device__ __forceinline__ void cluster_sum_rows(uint32_t addr, uint32_t row_step, uint32_t own_rank, float4 (&out)[ITER]) {
+    float4 t[ITER][S];
+#pragma unroll
+    for (int it = 0; it < ITER; ++it)
+#pragma unroll
+        for (int p = 0; p < S; ++p) {
+            const uint32_t a = addr + (uint32_t)it * row_step;
+            if ((uint32_t)p == own_rank) {
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(t[it][p].x), "=f"(t[it][p].y), "=f"(t[it][p].z), "=f"(t[it][p].w)
+                             : "r"(a)
+                             : "memory");
+            } else {
+                t[it][p] = ld_cluster_f4(a, (uint32_t)p);
+            }
+        }
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        out[it] = t[it][0];
+#pragma unroll
+        for (int p = 1; p < S; ++p) out[it].x += t[it][p].x, out[it].y += t[it][p].y, out[it].z += t[it][p].z, out[it].w += t[it][p].w;
+    }
+}
+
 // hi = v with the 13 low mantissa bits cleared; lo = the same of (v - hi).  Both are exact TF32 numbers.
 __device__ __forceinline__ void split_tf32(float v, float& hi, float& lo) {
     hi = __uint_as_float(__float_as_uint(v) & 0xFFFFE000u);
@@ -258,8 +286,38 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         constexpr int kPerRow = TN / 4, kRowsPerPass = 32 * kTfWorkerWarps / kPerRow;
         const int wt = tid - 64, ch = wt % kPerRow, rows_per = (kTfM + n_split - 1) / n_split;
         const float4 bv = *reinterpret_cast<const float4*>(bias_s + 4 * ch);
+        const int n = n0 + 4 * ch;
+        // Clusters of 2, 4 and 8: the thread's rows are kRowsPerPass apart (a multiple of 16, so the chunk
+        // permutation is the same for all of them) and all their loads are issued together.
+        auto fast = [&](auto s_tag, auto iter_tag) {
+            constexpr int S = decltype(s_tag)::value, ITER = decltype(iter_tag)::value;
+            const int rr0 = wt / kPerRow;
+            if (rr0 >= kTfM / S) return;
+            const int r0 = split * (kTfM / S) + rr0;
+            float4 acc[ITER];
+            cluster_sum_rows<S, ITER>(smem_u32(ring + r0 * (4 * TN) + ((ch ^ (r0 & 15)) << 4)), kRowsPerPass * 4 * TN,
+                                      (uint32_t)split, acc);
+#pragma unroll
+            for (int it = 0; it < ITER; ++it) {
+                const int m = m0 + r0 + it * kRowsPerPass;
+                if (m < batch && n < L.out) {
+                    float4 a = acc[it];
+                    a.x = activate(a.x + bv.x, L.act);
+                    a.y = activate(a.y + bv.y, L.act);
+                    a.z = activate(a.z + bv.z, L.act);
+                    a.w = activate(a.w + bv.w, L.act);
+                    *reinterpret_cast<float4*>(y + (size_t)m * L.out + n) = a;
+                }
+            }
+        };
+        using std::integral_constant;
+        constexpr int kIter2 = kTfM / 2 / kRowsPerPass, kIter4 = kTfM / 4 / kRowsPerPass;
+        if (n_split == 2) fast(integral_constant<int, 2>{}, integral_constant<int, kIter2>{});
+        else if (n_split == 4) fast(integral_constant<int, 4>{}, integral_constant<int, (kIter4 > 0 ? kIter4 : 1)>{});
+        else if (n_split == 8) fast(integral_constant<int, 8>{}, integral_constant<int, 1>{});
+        else
         for (int rr = wt / kPerRow; rr < rows_per; rr += kRowsPerPass) {
-            const int r = split * rows_per + rr, m = m0 + r, n = n0 + 4 * ch;
+            const int r = split * rows_per + rr, m = m0 + r;
             if (r < kTfM && m < batch && n < L.out) {
                 const uint32_t off = ring + r * (4 * TN) + ((ch ^ (r & 15)) << 4);
                 float4 a;
