@@ -66,6 +66,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, uint32
     }
     return false;
 }
+// Asks for a tensor map's 128 bytes ahead of the first TMA that uses it.
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t mbar, int c0, int c1) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
@@ -188,6 +192,8 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
     const int k_blocks = (int)(((int64_t)k_blocks_all * (split + 1)) / n_split) - kb0;
 
     if (tid == 0) {
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_w);
         for (int s = 0; s < kTcStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);

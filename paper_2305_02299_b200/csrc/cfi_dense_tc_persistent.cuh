@@ -59,6 +59,8 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
     const int first = blockIdx.x, stride = gridDim.x;
 
     if (tid == 0) {
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_w);
         for (int s = 0; s < kTpStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);

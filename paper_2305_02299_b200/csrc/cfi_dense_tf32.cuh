@@ -138,6 +138,8 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     const int n_local = (int)(((int64_t)k_blocks * (split + 1)) / n_split) - kb0;
 
     if (tid == 0) {
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_w);
         for (int s = 0; s < kTfStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(ready0 + 8 * s, 128);
