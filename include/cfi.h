@@ -24,6 +24,7 @@
 #ifndef CFI_H_
 #define CFI_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -130,6 +131,35 @@ cfi_status_t cfi_compact_producer(const float* bias, const int32_t* active_rows,
 cfi_status_t cfi_compact_consumer(const int32_t* prod_active_rows, int32_t prod_n_active, int32_t prod_out,
                                   const float* prod_const, float* values, int32_t* indices, const int32_t* active_rows,
                                   int32_t n_active, int32_t k, float* bias, int32_t out_features);
+
+/*
+ * cfi_srigl_update — one SRigL mask update of one layer, on the device (Sec. 3.1, the seven steps "for each
+ * layer": magnitudes and gradient magnitudes; K; salient weights per neuron; ablation below gamma_sal * k; the new
+ * fan-in k'; global pruning of the K smallest; regrowth per neuron to k').  Outside the forward path: it produces
+ * the masks that cfi_pack / cfi_create consume.
+ *
+ *   w       device, float [out_features, in_features], in/out: zero where masked; survivors keep their value,
+ *           grown weights are 0
+ *   mask    device, uint8 [out_features, in_features], in/out: 0/1, the same number k of ones in every non-empty row
+ *   grad    device, float [out_features, in_features]: dense gradient of the loss with respect to w
+ *   K       weights to prune and to grow (clipped to the number of active weights and of inactive positions)
+ *   gamma_sal  ablation threshold in [0, 1]: a neuron with fewer than max(1, gamma_sal * k) salient weights is ablated
+ *   workspace  device, 256-byte aligned, at least cfi_srigl_workspace_bytes(out_features, in_features) bytes
+ *   k_new, n_active_new  host, written: the new fan-in k' = min(in, floor(k * live_before / live_after)) and the
+ *           number of neurons that are still active
+ *
+ * Readings where the paper leaves a choice: ties in magnitude go to the smaller position (row-major); a weight is
+ * salient if it is active and not among the K smallest of the layer, or inactive and among the K largest gradients
+ * of the layer (live neurons only); neurons without weights stay ablated; regrowth may use any position of the
+ * neuron that is not active at that moment, a weight pruned in this very update included, and grown weights start
+ * at 0; a neuron left with more than k' weights after the global pruning loses its smallest down to k'.
+ * Runs on `stream` and waits for it.  CFI_ERR_NULL, CFI_ERR_SHAPE (sizes < 1, more than 2^31 entries, gamma_sal
+ * negative or NaN), CFI_ERR_ALIGNMENT, CFI_ERR_BUFFER_TOO_SMALL (workspace), CFI_ERR_CUDA.
+ */
+cfi_status_t cfi_srigl_workspace_bytes(int32_t out_features, int32_t in_features, size_t* bytes);
+cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* grad, int32_t out_features, int32_t in_features,
+                              int64_t K, float gamma_sal, void* workspace, size_t workspace_bytes, int32_t* k_new,
+                              int32_t* n_active_new, cfi_stream_t stream);
 
 /*
  * cfi_create — build a device-resident layer from condensed arrays (the inputs w and indx of

@@ -24,7 +24,8 @@ _DTYPES = {"f32": F32, "fp32": F32, "float32": F32, "bf16": BF16, "bfloat16": BF
 _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE, ACT_GELU: ACT_GELU}
 _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
 
-EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
+EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_srigl_workspace_bytes",
+           "cfi_srigl_update", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_dense_tile_shape", "cfi_device_status", "cfi_destroy",
            "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static",
            "cfi_probe_device")
@@ -71,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.cfi_pack.argtypes = [f32p, u8p, ci, ci, i32p, i32p, f32p, i32p, i32p]
     lib.cfi_compact_producer.argtypes = [f32p, i32p, ci, ci, f32p, i32p]
     lib.cfi_compact_consumer.argtypes = [i32p, ci, ci, f32p, f32p, i32p, i32p, ci, ci, f32p, ci]
+    lib.cfi_srigl_workspace_bytes.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_size_t)]
+    lib.cfi_srigl_update.argtypes = [vp, vp, vp, ci, ci, ctypes.c_int64, ctypes.c_float, vp, ctypes.c_size_t, i32p, i32p, vp]
     lib.cfi_create.argtypes = [f32p, i32p, i32p, f32p, ci, ci, ci, ci, ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
     lib.cfi_forward.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_forward_variant.argtypes = [vp, vp, vp, ci, vp, ctypes.c_int]
@@ -208,6 +211,22 @@ def cfi_compact_consumer(prod_active_rows, prod_out: int, prod_const, values, in
                                      _hp(v, ctypes.c_float), _hp(ix, ctypes.c_int32), _hp(rows, ctypes.c_int32), n_active, k,
                                      _hp(b, ctypes.c_float), b.shape[0]), "cfi_compact_consumer")
     return v, ix, b
+
+
+def cfi_srigl_update(w, mask, grad, K: int, gamma_sal: float, stream=None):
+    """One SRigL mask update in place on device tensors w (float32), mask (uint8), grad (float32), all [out, in] and
+    contiguous.  Returns (k_new, n_active_new).  The workspace is a torch allocation made here."""
+    import torch
+    out_f, in_f = w.shape
+    nbytes = ctypes.c_size_t(0)
+    _check(_lib.cfi_srigl_workspace_bytes(out_f, in_f, ctypes.byref(nbytes)), "cfi_srigl_workspace_bytes")
+    ws = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=w.device)
+    base = (ws.data_ptr() + 255) & ~255
+    k_new, n_act = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_lib.cfi_srigl_update(_dev_ptr(w), _dev_ptr(mask), _dev_ptr(grad), out_f, in_f, int(K), float(gamma_sal), base,
+                                 nbytes.value, ctypes.byref(k_new), ctypes.byref(n_act), _stream_handle(stream)),
+           "cfi_srigl_update")
+    return k_new.value, n_act.value
 
 
 def cfi_forward(layer: Layer, x, y, batch: int, stream=None) -> None:

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_PKG, "libcfi.so")
-SOURCES = ["cfi_pack.cpp", "cfi_layer.cu", "cfi_probe.cu"]
+SOURCES = ["cfi_pack.cpp", "cfi_layer.cu", "cfi_probe.cu", "cfi_srigl_update.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -1,0 +1,446 @@
+// cfi_srigl_update: one SRigL mask update of one layer on the device (Sec. 3.1, steps 1-7 "for each layer").
+//
+// Dense layout, as a training loop holds it: w[out][in] (zero where masked), mask[out][in] (0/1), grad[out][in].
+// The update needs two selections over the whole layer -- the K smallest magnitudes among the active weights and the
+// K largest gradient magnitudes among the inactive positions of live neurons -- and one selection per neuron (regrow
+// to the new fan-in k', or trim down to it).  All of them are "the m smallest of a set of (32-bit key, position)
+// pairs, ties to the smaller position", with key = the bits of |w| (a non-negative float orders like its bits) or
+// the complement of the bits of |grad| (so that a larger gradient is a smaller key).  They are done by radix
+// selection: four passes of 256-bin histograms over the digits of the key from the top, each pass narrowing to the
+// bin that holds the m-th element, then the ties on the final key are cut in position order with a prefix count.
+//
+// Readings where Sec. 3.1 leaves a choice (the same as the CPU oracle used by the tests takes): already ablated
+// neurons stay out; a weight is salient if it is active and not among the K smallest, or inactive and among the K
+// largest gradients; a neuron is ablated if its salient count is below max(1, gamma_sal * k);
+// k' = min(in, floor(k * live_before / live_after)); step 7 may regrow any position of the neuron that is not active
+// at that moment (a weight pruned in step 6 included; grown weights start at 0); a neuron left with more than k'
+// weights after step 6 loses its smallest down to k'.
+#include "cfi.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace {
+
+constexpr int kThreads = 256, kChunk = 16 * kThreads;  // a block marks ties over 4096 consecutive positions
+
+struct SelectState {
+    unsigned long long want;     // elements still to take inside the current prefix bin (1-based rank of the cut)
+    unsigned long long below;    // elements with a key below the current prefix
+    unsigned int prefix, prefix_mask;
+    unsigned int hist[256];
+};
+
+struct Scalars {
+    long long active_total, inactive_total;
+    int k, k_new, live_before, live_after;
+};
+
+__device__ __forceinline__ unsigned int mag_bits(float v) { return __float_as_uint(fabsf(v)); }
+
+// SEL 0: active weights, key = bits |w|.  SEL 1: inactive positions of live rows, key = ~bits |grad|.
+template <int SEL>
+__device__ __forceinline__ bool sel_key(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
+                                        long long p, unsigned int& key) {
+    if (SEL == 0) {
+        if (!mask[p]) return false;
+        key = mag_bits(w[p]);
+        return true;
+    }
+    if (mask[p] || row_count[p / in_f] == 0) return false;
+    key = ~mag_bits(grad[p]);
+    return true;
+}
+
+__global__ void row_count_kernel(const uint8_t* mask, int out_f, int in_f, int* row_count) {
+    __shared__ int s;
+    const int r = blockIdx.x;
+    if (threadIdx.x == 0) s = 0;
+    __syncthreads();
+    int c = 0;
+    for (int j = threadIdx.x; j < in_f; j += blockDim.x) c += mask[(size_t)r * in_f + j] ? 1 : 0;
+    atomicAdd(&s, c);
+    __syncthreads();
+    if (threadIdx.x == 0) row_count[r] = s;
+}
+
+// Single block: totals, k, and the initial state of the two layer-wide selections (K clipped to both pools).
+__global__ void setup_kernel(const int* row_count, int out_f, int in_f, long long K, Scalars* sc, SelectState* st) {
+    __shared__ long long act;
+    __shared__ int live, k;
+    if (threadIdx.x == 0) act = 0, live = 0, k = 0;
+    __syncthreads();
+    for (int r = threadIdx.x; r < out_f; r += blockDim.x)
+        if (row_count[r] > 0) {
+            atomicAdd((unsigned long long*)&act, (unsigned long long)row_count[r]);
+            atomicAdd(&live, 1);
+            atomicMax(&k, row_count[r]);
+        }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        sc->active_total = act;
+        sc->inactive_total = (long long)live * in_f - act;
+        sc->k = k, sc->live_before = live, sc->k_new = 0, sc->live_after = 0;
+        long long kk = K < 0 ? 0 : K;
+        if (kk > act) kk = act;
+        if (kk > sc->inactive_total) kk = sc->inactive_total;
+        for (int s = 0; s < 2; ++s) st[s].want = (unsigned long long)kk, st[s].below = 0, st[s].prefix = 0, st[s].prefix_mask = 0;
+    }
+    for (int s = 0; s < 2; ++s)
+        for (int b = threadIdx.x; b < 256; b += blockDim.x) st[s].hist[b] = 0;
+}
+
+// Histogram of digit `pass` (0 = top byte) over the valid elements whose key matches the prefix found so far.
+template <int SEL>
+__global__ void hist_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f, long long n,
+                            int pass, SelectState* st) {
+    __shared__ unsigned int h[256];
+    for (int b = threadIdx.x; b < 256; b += blockDim.x) h[b] = 0;
+    __syncthreads();
+    if (st->want != 0) {
+        const unsigned int prefix = st->prefix, pmask = st->prefix_mask;
+        const int shift = 24 - 8 * pass;
+        for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (long long)gridDim.x * blockDim.x) {
+            unsigned int key;
+            if (sel_key<SEL>(w, mask, grad, row_count, in_f, p, key) && (key & pmask) == prefix) atomicAdd(&h[(key >> shift) & 255u], 1u);
+        }
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < 256; b += blockDim.x)
+        if (h[b]) atomicAdd(&st->hist[b], h[b]);
+}
+
+// One thread: the bin that holds the `want`-th element; narrow the prefix to it and clear the histogram.
+__global__ void pick_kernel(int pass, SelectState* st) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (st->want != 0) {
+        unsigned long long seen = 0;
+        int b = 0;
+        for (; b < 255; ++b) {
+            if (seen + st->hist[b] >= st->want) break;
+            seen += st->hist[b];
+        }
+        const int shift = 24 - 8 * pass;
+        st->want -= seen;
+        st->below += seen;
+        st->prefix |= (unsigned int)b << shift;
+        st->prefix_mask |= 255u << shift;
+    }
+    for (int b = 0; b < 256; ++b) st->hist[b] = 0;
+}
+
+// After the four passes prefix is the key of the cut and `want` of the elements equal to it are taken, the first ones
+// in position order.  Per chunk of kChunk positions: how many equal the cut key.
+template <int SEL>
+__global__ void tie_count_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
+                                 long long n, const SelectState* st, unsigned int* chunk_ties) {
+    __shared__ unsigned int s;
+    if (threadIdx.x == 0) s = 0;
+    __syncthreads();
+    const long long base = (long long)blockIdx.x * kChunk + (long long)threadIdx.x * 16;
+    unsigned int c = 0;
+    if (st->want != 0)
+        for (int e = 0; e < 16; ++e) {
+            unsigned int key;
+            if (base + e < n && sel_key<SEL>(w, mask, grad, row_count, in_f, base + e, key) && key == st->prefix) ++c;
+        }
+    if (c) atomicAdd(&s, c);
+    __syncthreads();
+    if (threadIdx.x == 0) chunk_ties[blockIdx.x] = s;
+}
+
+// Single block: exclusive prefix sum of the per-chunk tie counts, in place.
+__global__ void chunk_scan_kernel(unsigned int* chunk_ties, int n_chunks) {
+    __shared__ unsigned long long carry;
+    __shared__ unsigned int part[kThreads];
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int c0 = 0; c0 < n_chunks; c0 += kThreads) {
+        const int c = c0 + threadIdx.x;
+        const unsigned int v = c < n_chunks ? chunk_ties[c] : 0u;
+        part[threadIdx.x] = v;
+        __syncthreads();
+        for (int off = 1; off < kThreads; off <<= 1) {  // inclusive scan of the block's values
+            const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
+            __syncthreads();
+            part[threadIdx.x] += add;
+            __syncthreads();
+        }
+        const unsigned long long before = carry + part[threadIdx.x] - v;
+        if (c < n_chunks) chunk_ties[c] = (unsigned int)(before > 0xFFFFFFFFull ? 0xFFFFFFFFull : before);
+        __syncthreads();
+        if (threadIdx.x == kThreads - 1) carry += part[kThreads - 1];
+        __syncthreads();
+    }
+}
+
+// flag[p] = 1 for the selected elements: key below the cut, or equal to it and among the first `want` in position order.
+template <int SEL>
+__global__ void mark_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f, long long n,
+                            const SelectState* st, const unsigned int* chunk_ties, uint8_t* flag) {
+    __shared__ unsigned int part[kThreads];
+    const long long base = (long long)blockIdx.x * kChunk + (long long)threadIdx.x * 16;
+    const unsigned long long want = st->want;
+    const unsigned int cut = st->prefix;
+    unsigned int keys[16];
+    bool valid[16];
+    unsigned int mine = 0;
+    for (int e = 0; e < 16; ++e) {
+        valid[e] = base + e < n && sel_key<SEL>(w, mask, grad, row_count, in_f, base + e, keys[e]);
+        if (want != 0 && valid[e] && keys[e] == cut) ++mine;
+    }
+    part[threadIdx.x] = mine;
+    __syncthreads();
+    for (int off = 1; off < kThreads; off <<= 1) {
+        const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
+        __syncthreads();
+        part[threadIdx.x] += add;
+        __syncthreads();
+    }
+    unsigned long long rank = (unsigned long long)chunk_ties[blockIdx.x] + part[threadIdx.x] - mine;  // ties before this thread's first
+    for (int e = 0; e < 16; ++e) {
+        if (base + e >= n) break;
+        uint8_t f = 0;
+        if (want != 0 && valid[e]) {
+            if (keys[e] < cut) f = 1;
+            else if (keys[e] == cut) f = rank++ < want ? 1 : 0;
+        }
+        flag[base + e] = f;
+    }
+}
+
+// Step 3: salient weights per neuron.
+__global__ void salient_kernel(const uint8_t* mask, const uint8_t* drop, const uint8_t* grow_top, int in_f, int* salient) {
+    __shared__ int s;
+    const int r = blockIdx.x;
+    if (threadIdx.x == 0) s = 0;
+    __syncthreads();
+    int c = 0;
+    for (int j = threadIdx.x; j < in_f; j += blockDim.x) {
+        const size_t p = (size_t)r * in_f + j;
+        c += ((mask[p] && !drop[p]) || grow_top[p]) ? 1 : 0;
+    }
+    atomicAdd(&s, c);
+    __syncthreads();
+    if (threadIdx.x == 0) salient[r] = s;
+}
+
+// Steps 4 and 5 (single block): who is ablated, and the new fan-in.
+__global__ void ablate_kernel(const int* row_count, const int* salient, int out_f, int in_f, float gamma_sal, Scalars* sc,
+                              uint8_t* survives) {
+    __shared__ int after;
+    if (threadIdx.x == 0) after = 0;
+    __syncthreads();
+    const double threshold = fmax(1.0, (double)gamma_sal * (double)sc->k);
+    for (int r = threadIdx.x; r < out_f; r += blockDim.x) {
+        const bool live = row_count[r] > 0 && !((double)salient[r] < threshold);
+        survives[r] = live ? 1 : 0;
+        if (live) atomicAdd(&after, 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        sc->live_after = after;
+        long long kn = after > 0 ? ((long long)sc->k * sc->live_before) / after : 0;
+        if (kn > in_f) kn = in_f;
+        sc->k_new = (int)kn;
+    }
+}
+
+// Block-wide selection inside one row: the `m` smallest keys (ties to the smaller column) among the columns for which
+// `key_of` returns true.  Returns through shared memory the cut key and how many ties on it to take; `take(c, key)`
+// then answers for a column in increasing column order within the calling pattern below.
+struct RowCut {
+    unsigned int cut;
+    unsigned int ties;   // elements equal to the cut to take, the first ones in column order
+    int any;             // 0: nothing to select
+};
+
+template <typename KeyOf>
+__device__ void row_select(int in_f, int m, KeyOf key_of, unsigned int* hist /*256, shared*/, RowCut* out /*shared*/) {
+    __shared__ unsigned int prefix, pmask, want;
+    if (threadIdx.x == 0) prefix = 0, pmask = 0, want = (unsigned int)(m > 0 ? m : 0);
+    __syncthreads();
+    for (int pass = 0; pass < 4 && m > 0; ++pass) {
+        for (int b = threadIdx.x; b < 256; b += blockDim.x) hist[b] = 0;
+        __syncthreads();
+        const int shift = 24 - 8 * pass;
+        for (int c = threadIdx.x; c < in_f; c += blockDim.x) {
+            unsigned int key;
+            if (key_of(c, key) && (key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned int seen = 0;
+            int b = 0;
+            for (; b < 255; ++b) {
+                if (seen + hist[b] >= want) break;
+                seen += hist[b];
+            }
+            want -= seen;
+            prefix |= (unsigned int)b << shift;
+            pmask |= 255u << shift;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) out->cut = prefix, out->ties = want, out->any = m > 0 ? 1 : 0;
+    __syncthreads();
+}
+
+// Steps 6 and 7 for one neuron per block: prune, then trim or regrow to k'.
+__global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, const uint8_t* drop, const uint8_t* survives,
+                                int in_f, const Scalars* sc) {
+    __shared__ unsigned int hist[256];
+    __shared__ RowCut cut;
+    __shared__ int kept_count;
+    __shared__ unsigned int part[kThreads];
+    __shared__ unsigned int carry;
+    const int r = blockIdx.x;
+    float* wr = w + (size_t)r * in_f;
+    uint8_t* mr = mask + (size_t)r * in_f;
+    const float* gr = grad + (size_t)r * in_f;
+    const uint8_t* dr = drop + (size_t)r * in_f;
+    if (!survives[r]) {  // ablated now or before: nothing left
+        for (int c = threadIdx.x; c < in_f; c += blockDim.x) wr[c] = 0.0f, mr[c] = 0;
+        return;
+    }
+    const int k_new = sc->k_new;
+    if (threadIdx.x == 0) kept_count = 0;
+    __syncthreads();
+    int mine = 0;
+    for (int c = threadIdx.x; c < in_f; c += blockDim.x) mine += (mr[c] && !dr[c]) ? 1 : 0;
+    atomicAdd(&kept_count, mine);
+    __syncthreads();
+    const int kept = kept_count;
+    const bool trim = kept > k_new;
+    const int m = trim ? kept - k_new : k_new - kept;
+    if (trim)  // the kept weights with the smallest magnitudes go
+        row_select(in_f, m, [&](int c, unsigned int& key) { key = mag_bits(wr[c]); return mr[c] && !dr[c]; }, hist, &cut);
+    else       // the free positions with the largest gradient magnitudes come
+        row_select(in_f, m, [&](int c, unsigned int& key) { key = ~mag_bits(gr[c]); return !(mr[c] && !dr[c]); }, hist, &cut);
+    // Apply, walking the row in column order so that ties on the cut key go to the smaller columns.
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int c0 = 0; c0 < in_f; c0 += kThreads) {
+        const int c = c0 + threadIdx.x;
+        bool is_kept = false, candidate = false;
+        unsigned int key = 0;
+        if (c < in_f) {
+            is_kept = mr[c] && !dr[c];
+            candidate = trim ? is_kept : !is_kept;
+            key = trim ? mag_bits(wr[c]) : ~mag_bits(gr[c]);
+        }
+        const unsigned int tie = (cut.any && candidate && key == cut.cut) ? 1u : 0u;
+        part[threadIdx.x] = tie;
+        __syncthreads();
+        for (int off = 1; off < kThreads; off <<= 1) {
+            const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
+            __syncthreads();
+            part[threadIdx.x] += add;
+            __syncthreads();
+        }
+        const unsigned int rank = carry + part[threadIdx.x] - tie;
+        if (c < in_f) {
+            const bool selected = cut.any && candidate && (key < cut.cut || (tie && rank < cut.ties));
+            bool on;
+            float val;
+            if (trim) on = is_kept && !selected, val = on ? wr[c] : 0.0f;
+            else on = is_kept || selected, val = is_kept ? wr[c] : 0.0f;
+            mr[c] = on ? 1 : 0;
+            wr[c] = val;
+        }
+        __syncthreads();
+        if (threadIdx.x == kThreads - 1) carry += part[kThreads - 1];
+        __syncthreads();
+    }
+}
+
+size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct Workspace {
+    int* row_count;
+    int* salient;
+    uint8_t* survives;
+    uint8_t* drop;
+    uint8_t* grow_top;
+    unsigned int* chunk_ties;
+    SelectState* state;
+    Scalars* scalars;
+    size_t bytes;
+};
+
+Workspace carve(void* base, int out_f, int in_f) {
+    const size_t n = (size_t)out_f * in_f, chunks = (n + kChunk - 1) / kChunk;
+    size_t off = 0;
+    auto take = [&](size_t b) {
+        const size_t at = off;
+        off += align_up(b);
+        return static_cast<char*>(base) + at;
+    };
+    Workspace w{};
+    w.row_count = reinterpret_cast<int*>(take((size_t)out_f * 4));
+    w.salient = reinterpret_cast<int*>(take((size_t)out_f * 4));
+    w.survives = reinterpret_cast<uint8_t*>(take((size_t)out_f));
+    w.drop = reinterpret_cast<uint8_t*>(take(n));
+    w.grow_top = reinterpret_cast<uint8_t*>(take(n));
+    w.chunk_ties = reinterpret_cast<unsigned int*>(take(chunks * 4));
+    w.state = reinterpret_cast<SelectState*>(take(2 * sizeof(SelectState)));
+    w.scalars = reinterpret_cast<Scalars*>(take(sizeof(Scalars)));
+    w.bytes = off;
+    return w;
+}
+
+template <int SEL>
+bool layer_select(const float* w, const uint8_t* mask, const float* grad, const Workspace& ws, int in_f, long long n,
+                  uint8_t* flag, cudaStream_t st) {
+    const int chunks = (int)((n + kChunk - 1) / kChunk);
+    const long long want_blocks = (n + kThreads * 8 - 1) / (kThreads * 8);
+    const int blocks = (int)(want_blocks < 1 ? 1 : want_blocks > 1184 ? 1184 : want_blocks);  // 8 CTAs per SM at most
+    for (int pass = 0; pass < 4; ++pass) {
+        hist_kernel<SEL><<<blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, pass, ws.state + SEL);
+        pick_kernel<<<1, 32, 0, st>>>(pass, ws.state + SEL);
+    }
+    tie_count_kernel<SEL><<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state + SEL, ws.chunk_ties);
+    chunk_scan_kernel<<<1, kThreads, 0, st>>>(ws.chunk_ties, chunks);
+    mark_kernel<SEL><<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state + SEL, ws.chunk_ties, flag);
+    return cudaGetLastError() == cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" cfi_status_t cfi_srigl_workspace_bytes(int32_t out_features, int32_t in_features, size_t* bytes) {
+    if (!bytes) return CFI_ERR_NULL;
+    if (out_features < 1 || in_features < 1 || (int64_t)out_features * in_features > ((int64_t)1 << 31)) return CFI_ERR_SHAPE;
+    *bytes = carve(nullptr, out_features, in_features).bytes;
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* grad, int32_t out_features, int32_t in_features,
+                                         int64_t K, float gamma_sal, void* workspace, size_t workspace_bytes, int32_t* k_new,
+                                         int32_t* n_active_new, cfi_stream_t stream) {
+    if (!w || !mask || !grad || !workspace || !k_new || !n_active_new) return CFI_ERR_NULL;
+    if (out_features < 1 || in_features < 1 || (int64_t)out_features * in_features > ((int64_t)1 << 31) || !(gamma_sal >= 0.0f))
+        return CFI_ERR_SHAPE;
+    if (((uintptr_t)workspace & 255) != 0) return CFI_ERR_ALIGNMENT;
+    const Workspace ws = carve(workspace, out_features, in_features);
+    if (workspace_bytes < ws.bytes) return CFI_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const long long n = (long long)out_features * in_features;
+    row_count_kernel<<<out_features, kThreads, 0, st>>>(mask, out_features, in_features, ws.row_count);
+    setup_kernel<<<1, kThreads, 0, st>>>(ws.row_count, out_features, in_features, (long long)K, ws.scalars, ws.state);
+    if (!layer_select<0>(w, mask, grad, ws, in_features, n, ws.drop, st)) return CFI_ERR_CUDA;       // step 3, first half (= step 6)
+    if (!layer_select<1>(w, mask, grad, ws, in_features, n, ws.grow_top, st)) return CFI_ERR_CUDA;   // step 3, second half
+    salient_kernel<<<out_features, kThreads, 0, st>>>(mask, ws.drop, ws.grow_top, in_features, ws.salient);
+    ablate_kernel<<<1, kThreads, 0, st>>>(ws.row_count, ws.salient, out_features, in_features, gamma_sal, ws.scalars, ws.survives);
+    finalize_kernel<<<out_features, kThreads, 0, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
+    Scalars host{};
+    if (cudaGetLastError() != cudaSuccess ||
+        cudaMemcpyAsync(&host, ws.scalars, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
+    *k_new = host.k_new;
+    *n_active_new = host.live_after;
+    return CFI_OK;
+}

@@ -1,0 +1,83 @@
+"""cfi_srigl_update (device) against the oracle of Sec. 3.1's seven steps: masks and weights bit for bit, k' and the
+number of live neurons equal.  Index and integer work: no tolerance."""
+import numpy as np
+import pytest
+
+from oracle.srigl_update import srigl_update
+from paper_2305_02299_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer(out_f, in_f, k, n_abl, seed):
+    L = inputs.make_layer(in_f, out_f, k, n_ablated=n_abl, seed=seed, bias=False)
+    g = inputs.make_x(out_f, in_f, seed=seed + 77)
+    return L.w_dense.copy(), L.mask.copy(), g
+
+
+def _run_device(w, m, g, K, gamma):
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    wd, md, gd = torch.from_numpy(w).cuda(), torch.from_numpy(m).cuda(), torch.from_numpy(g).cuda()
+    k_new, n_act = cfi.cfi_srigl_update(wd, md, gd, K, gamma)
+    torch.cuda.synchronize()
+    return wd.cpu().numpy(), md.cpu().numpy(), k_new, n_act
+
+
+def _compare(w, m, g, K, gamma):
+    gamma = float(np.float32(gamma))
+    w_ref, m_ref, k_ref, abl = srigl_update(w, m, g, K, gamma)
+    w_dev, m_dev, k_dev, n_dev = _run_device(w, m, g, K, gamma)
+    assert k_dev == k_ref
+    assert n_dev == int((m_ref.sum(1) > 0).sum())
+    assert np.array_equal(m_dev, m_ref)
+    assert np.array_equal(w_dev, w_ref)
+    return k_ref, abl
+
+
+@pytest.mark.parametrize("out_f,in_f,k,n_abl,K,gamma", [
+    (24, 40, 6, 0, 30, 0.3), (24, 40, 6, 3, 60, 0.5), (16, 16, 2, 0, 8, 1.0), (64, 96, 10, 5, 200, 0.3),
+    (8, 8, 8, 0, 0, 0.3), (12, 30, 3, 0, 36, 0.0), (1, 5, 2, 0, 1, 0.5), (7, 4099, 33, 1, 100, 0.25),
+    (768, 3072, 307, 38, 70_000, 0.3), (3072, 768, 77, 154, 60_000, 0.3), (300, 1000, 10, 0, 2990, 0.9)])
+def test_matches_oracle(out_f, in_f, k, n_abl, K, gamma):
+    w, m, g = _layer(out_f, in_f, k, n_abl, seed=out_f + in_f)
+    _compare(w, m, g, K, gamma)
+
+
+def test_ablation_case_and_chained_updates():
+    """A neuron with tiny weights and gradients is ablated and k' rises; a second update on the result still matches."""
+    w, m, g = _layer(64, 256, 16, 0, seed=9)
+    w[5] *= 1e-6
+    g[5] *= 1e-6
+    w[40] *= 1e-6
+    g[40] *= 1e-6
+    k2, abl = _compare(w, m, g, 32, 0.3)
+    assert set(abl) == {5, 40} and k2 == (16 * 64) // 62
+    w2, m2, _, _ = srigl_update(w, m, g, 32, float(np.float32(0.3)))
+    g2 = inputs.make_x(64, 256, seed=123)
+    _compare(w2, m2, g2, 50, 0.3)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_many_ties(seed):
+    """Quantised magnitudes and gradients: most selections are decided by position."""
+    rng = np.random.default_rng(seed)
+    out_f, in_f, k = int(rng.integers(3, 40)), int(rng.integers(8, 300)), 0
+    k = int(rng.integers(1, min(in_f, 20)))
+    w, m, g = _layer(out_f, in_f, k, int(rng.integers(0, out_f // 3 + 1)), seed=200 + seed)
+    w = (np.round(w * 2) / 2 * (m == 1)).astype(np.float32)
+    g = np.round(g).astype(np.float32)
+    _compare(w, m, g, int(rng.integers(0, out_f * k + 1)), float(rng.choice([0.0, 0.25, 0.5, 1.0])))
+
+
+def test_workspace_and_argument_checks():
+    import ctypes
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    w = torch.zeros((4, 8), device="cuda")
+    m = torch.zeros((4, 8), device="cuda", dtype=torch.uint8)
+    with pytest.raises(cfi.CfiError) as e:
+        cfi.cfi_srigl_update(w, m, w, 1, -0.5)
+    assert e.value.status == 2
+    k_new, n_act = cfi.cfi_srigl_update(w, m, w, 3, 0.3)      # a layer with no active weight stays empty
+    assert (k_new, n_act) == (0, 0) and int(m.sum()) == 0
