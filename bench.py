@@ -427,6 +427,7 @@ def main():
         except Exception as exc:
             line["device_probe"] = str(exc)
         line["stack_batch1"] = stack_batch1_leg(cfi, torch, l2, peaks)
+        line["srigl_update"] = srigl_update_leg(cfi, torch, peaks)
     if rank == 0:
         print(json.dumps(line))
     if dist:
@@ -569,6 +570,32 @@ def stack_batch1_leg(cfi, torch, l2, peaks, blocks=12, replicas=4):
             "us_per_pass_eager_warm": eager * 1e6, "algorithmic_bytes": bytes_,
             "hbm_frac": bytes_ / sec / 1e9 / peaks["hbm_gbs"], "gflops": flops / sec / 1e9,
             "l2": f"{replicas} rotating stacks, {replicas * bytes_ / 1e6:.0f} MB vs L2 {l2 / 1e6:.0f} MB"}
+
+
+def srigl_update_leg(cfi, torch, peaks):
+    """One SRigL mask update (Sec. 3.1, steps 1-7) on the device for the two ViT MLP layer shapes and the 4096 x 4096
+    layer at 80 % sparsity; K = 30 % of the active weights, gamma_sal = 0.3.  Algorithmic bytes: w, mask and grad
+    read once (9 B per entry), w and mask written once (5 B)."""
+    import time
+    out = {}
+    for name, (out_f, in_f, k) in {"768x3072_k77": (3072, 768, 77), "3072x768_k307": (768, 3072, 307),
+                                   "4096x4096_k819": (4096, 4096, 819)}.items():
+        L = inputs.make_layer(in_f, out_f, k, seed=11, bias=False)
+        g = torch.from_numpy(inputs.make_x(out_f, in_f, seed=12)).cuda()
+        w0, m0 = torch.from_numpy(L.w_dense).cuda(), torch.from_numpy(L.mask).cuda()
+        K = int(0.3 * out_f * k)
+        times = []
+        for it in range(6):
+            w, m = w0.clone(), m0.clone()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            k_new, n_act = cfi.cfi_srigl_update(w, m, g, K, 0.3)     # returns after its stream has drained
+            times.append(time.perf_counter() - t0)
+        sec = float(np.median(times[1:]))
+        nbytes = 14 * out_f * in_f
+        out[name] = {"us_per_update": sec * 1e6, "K": K, "k_new": k_new, "n_active_new": n_act,
+                     "algorithmic_bytes": nbytes, "hbm_frac": nbytes / sec / 1e9 / peaks["hbm_gbs"]}
+    return out
 
 
 def batch1_leg(W, cfi, torch, l2, peaks, peak_kind):

@@ -39,18 +39,14 @@ struct Scalars {
 
 __device__ __forceinline__ unsigned int mag_bits(float v) { return __float_as_uint(fabsf(v)); }
 
-// SEL 0: active weights, key = bits |w|.  SEL 1: inactive positions of live rows, key = ~bits |grad|.
-template <int SEL>
-__device__ __forceinline__ bool sel_key(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
-                                        long long p, unsigned int& key) {
-    if (SEL == 0) {
-        if (!mask[p]) return false;
-        key = mag_bits(w[p]);
-        return true;
+// h[bin] += 1 for every lane that takes part; lanes of the warp with the same bin are counted by one of them.  (The top
+// digits of float magnitudes fall into a handful of bins, and a plain atomic per lane would serialise on them.)
+__device__ __forceinline__ void hist_add(unsigned int* h, bool take, unsigned int bin) {
+    const unsigned int active = __ballot_sync(0xffffffffu, take);
+    if (take) {
+        const unsigned int peers = __match_any_sync(active, bin);
+        if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&h[bin], (unsigned int)__popc(peers));
     }
-    if (mask[p] || row_count[p / in_f] == 0) return false;
-    key = ~mag_bits(grad[p]);
-    return true;
 }
 
 __global__ void row_count_kernel(const uint8_t* mask, int out_f, int in_f, int* row_count) {
@@ -71,12 +67,20 @@ __global__ void setup_kernel(const int* row_count, int out_f, int in_f, long lon
     __shared__ int live, k;
     if (threadIdx.x == 0) act = 0, live = 0, k = 0;
     __syncthreads();
+    long long my_act = 0;
+    int my_live = 0, my_k = 0;
     for (int r = threadIdx.x; r < out_f; r += blockDim.x)
-        if (row_count[r] > 0) {
-            atomicAdd((unsigned long long*)&act, (unsigned long long)row_count[r]);
-            atomicAdd(&live, 1);
-            atomicMax(&k, row_count[r]);
-        }
+        if (row_count[r] > 0) my_act += row_count[r], ++my_live, my_k = max(my_k, row_count[r]);
+    for (int off = 16; off > 0; off >>= 1) {  // one set of atomics per warp
+        my_act += __shfl_down_sync(0xffffffffu, my_act, off);
+        my_live += __shfl_down_sync(0xffffffffu, my_live, off);
+        my_k = max(my_k, __shfl_down_sync(0xffffffffu, my_k, off));
+    }
+    if ((threadIdx.x & 31) == 0 && my_live) {
+        atomicAdd((unsigned long long*)&act, (unsigned long long)my_act);
+        atomicAdd(&live, my_live);
+        atomicMax(&k, my_k);
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         sc->active_total = act;
@@ -91,29 +95,46 @@ __global__ void setup_kernel(const int* row_count, int out_f, int in_f, long lon
         for (int b = threadIdx.x; b < 256; b += blockDim.x) st[s].hist[b] = 0;
 }
 
-// Histogram of digit `pass` (0 = top byte) over the valid elements whose key matches the prefix found so far.
-template <int SEL>
+// Histograms of digit `pass` (0 = top byte) for both layer-wide selections in one sweep over the layer: over the valid
+// elements of each whose key matches the prefix found so far.  Every position is valid for at most one of the two.
 __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f, long long n,
                             int pass, SelectState* st) {
-    __shared__ unsigned int h[256];
-    for (int b = threadIdx.x; b < 256; b += blockDim.x) h[b] = 0;
+    __shared__ unsigned int h[2][256];
+    for (int b = threadIdx.x; b < 512; b += blockDim.x) h[b >> 8][b & 255] = 0;
     __syncthreads();
-    if (st->want != 0) {
-        const unsigned int prefix = st->prefix, pmask = st->prefix_mask;
+    const bool on0 = st[0].want != 0, on1 = st[1].want != 0;
+    if (on0 || on1) {
+        const unsigned int prefix0 = st[0].prefix, pmask0 = st[0].prefix_mask, prefix1 = st[1].prefix, pmask1 = st[1].prefix_mask;
         const int shift = 24 - 8 * pass;
-        for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (long long)gridDim.x * blockDim.x) {
-            unsigned int key;
-            if (sel_key<SEL>(w, mask, grad, row_count, in_f, p, key) && (key & pmask) == prefix) atomicAdd(&h[(key >> shift) & 255u], 1u);
+        const long long stride = (long long)gridDim.x * blockDim.x;
+        const long long rounds = (n + stride - 1) / stride;  // the same trip count for every lane: the warp votes inside
+        for (long long i = 0; i < rounds; ++i) {
+            const long long p = i * stride + (long long)blockIdx.x * blockDim.x + threadIdx.x;
+            bool take0 = false, take1 = false;
+            unsigned int key = 0;
+            if (p < n) {
+                if (mask[p]) {
+                    key = mag_bits(w[p]);
+                    take0 = on0 && (key & pmask0) == prefix0;
+                } else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) {
+                    key = ~mag_bits(grad[p]);
+                    take1 = on1 && (key & pmask1) == prefix1;
+                }
+            }
+            const unsigned int bin = (key >> shift) & 255u;
+            hist_add(h[0], take0, bin);
+            hist_add(h[1], take1, bin);
         }
     }
     __syncthreads();
-    for (int b = threadIdx.x; b < 256; b += blockDim.x)
-        if (h[b]) atomicAdd(&st->hist[b], h[b]);
+    for (int b = threadIdx.x; b < 512; b += blockDim.x)
+        if (h[b >> 8][b & 255]) atomicAdd(&st[b >> 8].hist[b & 255], h[b >> 8][b & 255]);
 }
 
 // One thread: the bin that holds the `want`-th element; narrow the prefix to it and clear the histogram.
-__global__ void pick_kernel(int pass, SelectState* st) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+__global__ void pick_kernel(int pass, SelectState* both) {
+    if (threadIdx.x > 1 || blockIdx.x != 0) return;
+    SelectState* st = both + threadIdx.x;  // one thread per selection
     if (st->want != 0) {
         unsigned long long seen = 0;
         int b = 0;
@@ -131,27 +152,30 @@ __global__ void pick_kernel(int pass, SelectState* st) {
 }
 
 // After the four passes prefix is the key of the cut and `want` of the elements equal to it are taken, the first ones
-// in position order.  Per chunk of kChunk positions: how many equal the cut key.
-template <int SEL>
+// in position order.  Per chunk of kChunk positions and per selection: how many equal the cut key.
 __global__ void tie_count_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
-                                 long long n, const SelectState* st, unsigned int* chunk_ties) {
-    __shared__ unsigned int s;
-    if (threadIdx.x == 0) s = 0;
+                                 long long n, const SelectState* st, unsigned int* chunk_ties, int n_chunks) {
+    __shared__ unsigned int s[2];
+    if (threadIdx.x < 2) s[threadIdx.x] = 0;
     __syncthreads();
     const long long base = (long long)blockIdx.x * kChunk + (long long)threadIdx.x * 16;
-    unsigned int c = 0;
-    if (st->want != 0)
-        for (int e = 0; e < 16; ++e) {
-            unsigned int key;
-            if (base + e < n && sel_key<SEL>(w, mask, grad, row_count, in_f, base + e, key) && key == st->prefix) ++c;
-        }
-    if (c) atomicAdd(&s, c);
+    const bool on0 = st[0].want != 0, on1 = st[1].want != 0;
+    const unsigned int cut0 = st[0].prefix, cut1 = st[1].prefix;
+    unsigned int c0 = 0, c1 = 0;
+    for (int e = 0; e < 16 && base + e < n; ++e) {
+        const long long p = base + e;
+        if (mask[p]) c0 += (on0 && mag_bits(w[p]) == cut0) ? 1u : 0u;
+        else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) c1 += (on1 && ~mag_bits(grad[p]) == cut1) ? 1u : 0u;
+    }
+    if (c0) atomicAdd(&s[0], c0);
+    if (c1) atomicAdd(&s[1], c1);
     __syncthreads();
-    if (threadIdx.x == 0) chunk_ties[blockIdx.x] = s;
+    if (threadIdx.x < 2) chunk_ties[(size_t)threadIdx.x * n_chunks + blockIdx.x] = s[threadIdx.x];
 }
 
-// Single block: exclusive prefix sum of the per-chunk tie counts, in place.
-__global__ void chunk_scan_kernel(unsigned int* chunk_ties, int n_chunks) {
+// One block per selection: exclusive prefix sum of its per-chunk tie counts, in place.
+__global__ void chunk_scan_kernel(unsigned int* chunk_ties_both, int n_chunks) {
+    unsigned int* chunk_ties = chunk_ties_both + (size_t)blockIdx.x * n_chunks;
     __shared__ unsigned long long carry;
     __shared__ unsigned int part[kThreads];
     if (threadIdx.x == 0) carry = 0;
@@ -175,38 +199,54 @@ __global__ void chunk_scan_kernel(unsigned int* chunk_ties, int n_chunks) {
     }
 }
 
-// flag[p] = 1 for the selected elements: key below the cut, or equal to it and among the first `want` in position order.
-template <int SEL>
+// drop[p] / grow_top[p] = 1 for the selected elements of the two selections: key below the cut, or equal to it and among
+// the first `want` in position order.
 __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f, long long n,
-                            const SelectState* st, const unsigned int* chunk_ties, uint8_t* flag) {
-    __shared__ unsigned int part[kThreads];
+                            const SelectState* st, const unsigned int* chunk_ties, int n_chunks, uint8_t* drop,
+                            uint8_t* grow_top) {
+    __shared__ unsigned int part[2][kThreads];
     const long long base = (long long)blockIdx.x * kChunk + (long long)threadIdx.x * 16;
-    const unsigned long long want = st->want;
-    const unsigned int cut = st->prefix;
+    const unsigned long long want0 = st[0].want, want1 = st[1].want;
+    const unsigned int cut0 = st[0].prefix, cut1 = st[1].prefix;
     unsigned int keys[16];
-    bool valid[16];
-    unsigned int mine = 0;
+    uint8_t kind[16];  // 0: in neither pool, 1: active weight, 2: inactive position of a live neuron
+    unsigned int mine0 = 0, mine1 = 0;
     for (int e = 0; e < 16; ++e) {
-        valid[e] = base + e < n && sel_key<SEL>(w, mask, grad, row_count, in_f, base + e, keys[e]);
-        if (want != 0 && valid[e] && keys[e] == cut) ++mine;
+        kind[e] = 0, keys[e] = 0;
+        const long long p = base + e;
+        if (p < n) {
+            if (mask[p]) kind[e] = 1, keys[e] = mag_bits(w[p]);
+            else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) kind[e] = 2, keys[e] = ~mag_bits(grad[p]);
+        }
+        if (kind[e] == 1 && want0 != 0 && keys[e] == cut0) ++mine0;
+        if (kind[e] == 2 && want1 != 0 && keys[e] == cut1) ++mine1;
     }
-    part[threadIdx.x] = mine;
+    part[0][threadIdx.x] = mine0;
+    part[1][threadIdx.x] = mine1;
     __syncthreads();
     for (int off = 1; off < kThreads; off <<= 1) {
-        const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
+        const unsigned int add0 = threadIdx.x >= off ? part[0][threadIdx.x - off] : 0u;
+        const unsigned int add1 = threadIdx.x >= off ? part[1][threadIdx.x - off] : 0u;
         __syncthreads();
-        part[threadIdx.x] += add;
+        part[0][threadIdx.x] += add0;
+        part[1][threadIdx.x] += add1;
         __syncthreads();
     }
-    unsigned long long rank = (unsigned long long)chunk_ties[blockIdx.x] + part[threadIdx.x] - mine;  // ties before this thread's first
+    // ties of each selection before this thread's first element
+    unsigned long long rank0 = (unsigned long long)chunk_ties[blockIdx.x] + part[0][threadIdx.x] - mine0;
+    unsigned long long rank1 = (unsigned long long)chunk_ties[(size_t)n_chunks + blockIdx.x] + part[1][threadIdx.x] - mine1;
     for (int e = 0; e < 16; ++e) {
         if (base + e >= n) break;
-        uint8_t f = 0;
-        if (want != 0 && valid[e]) {
-            if (keys[e] < cut) f = 1;
-            else if (keys[e] == cut) f = rank++ < want ? 1 : 0;
+        uint8_t f0 = 0, f1 = 0;
+        if (kind[e] == 1 && want0 != 0) {
+            if (keys[e] < cut0) f0 = 1;
+            else if (keys[e] == cut0) f0 = rank0++ < want0 ? 1 : 0;
+        } else if (kind[e] == 2 && want1 != 0) {
+            if (keys[e] < cut1) f1 = 1;
+            else if (keys[e] == cut1) f1 = rank1++ < want1 ? 1 : 0;
         }
-        flag[base + e] = f;
+        drop[base + e] = f0;
+        grow_top[base + e] = f1;
     }
 }
 
@@ -383,26 +423,27 @@ Workspace carve(void* base, int out_f, int in_f) {
     w.survives = reinterpret_cast<uint8_t*>(take((size_t)out_f));
     w.drop = reinterpret_cast<uint8_t*>(take(n));
     w.grow_top = reinterpret_cast<uint8_t*>(take(n));
-    w.chunk_ties = reinterpret_cast<unsigned int*>(take(chunks * 4));
+    w.chunk_ties = reinterpret_cast<unsigned int*>(take(2 * chunks * 4));
     w.state = reinterpret_cast<SelectState*>(take(2 * sizeof(SelectState)));
     w.scalars = reinterpret_cast<Scalars*>(take(sizeof(Scalars)));
     w.bytes = off;
     return w;
 }
 
-template <int SEL>
-bool layer_select(const float* w, const uint8_t* mask, const float* grad, const Workspace& ws, int in_f, long long n,
-                  uint8_t* flag, cudaStream_t st) {
+// Step 3's two selections over the whole layer (the first is also step 6's pruning set), in shared sweeps.
+bool layer_select_both(const float* w, const uint8_t* mask, const float* grad, const Workspace& ws, int in_f, long long n,
+                       cudaStream_t st) {
     const int chunks = (int)((n + kChunk - 1) / kChunk);
     const long long want_blocks = (n + kThreads * 8 - 1) / (kThreads * 8);
     const int blocks = (int)(want_blocks < 1 ? 1 : want_blocks > 1184 ? 1184 : want_blocks);  // 8 CTAs per SM at most
     for (int pass = 0; pass < 4; ++pass) {
-        hist_kernel<SEL><<<blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, pass, ws.state + SEL);
-        pick_kernel<<<1, 32, 0, st>>>(pass, ws.state + SEL);
+        hist_kernel<<<blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, pass, ws.state);
+        pick_kernel<<<1, 32, 0, st>>>(pass, ws.state);
     }
-    tie_count_kernel<SEL><<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state + SEL, ws.chunk_ties);
-    chunk_scan_kernel<<<1, kThreads, 0, st>>>(ws.chunk_ties, chunks);
-    mark_kernel<SEL><<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state + SEL, ws.chunk_ties, flag);
+    tie_count_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks);
+    chunk_scan_kernel<<<2, kThreads, 0, st>>>(ws.chunk_ties, chunks);
+    mark_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks, ws.drop,
+                                             ws.grow_top);
     return cudaGetLastError() == cudaSuccess;
 }
 
@@ -428,8 +469,7 @@ extern "C" cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* g
     const long long n = (long long)out_features * in_features;
     row_count_kernel<<<out_features, kThreads, 0, st>>>(mask, out_features, in_features, ws.row_count);
     setup_kernel<<<1, kThreads, 0, st>>>(ws.row_count, out_features, in_features, (long long)K, ws.scalars, ws.state);
-    if (!layer_select<0>(w, mask, grad, ws, in_features, n, ws.drop, st)) return CFI_ERR_CUDA;       // step 3, first half (= step 6)
-    if (!layer_select<1>(w, mask, grad, ws, in_features, n, ws.grow_top, st)) return CFI_ERR_CUDA;   // step 3, second half
+    if (!layer_select_both(w, mask, grad, ws, in_features, n, st)) return CFI_ERR_CUDA;
     salient_kernel<<<out_features, kThreads, 0, st>>>(mask, ws.drop, ws.grow_top, in_features, ws.salient);
     ablate_kernel<<<1, kThreads, 0, st>>>(ws.row_count, ws.salient, out_features, in_features, gamma_sal, ws.scalars, ws.survives);
     finalize_kernel<<<out_features, kThreads, 0, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
