@@ -96,39 +96,64 @@ __global__ void setup_kernel(const int* row_count, int out_f, int in_f, long lon
 }
 
 // Histograms of digit `pass` (0 = top byte) for both layer-wide selections in one sweep over the layer: over the valid
-// elements of each whose key matches the prefix found so far.  Every position is valid for at most one of the two.
-__global__ void hist_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f, long long n,
+// elements of each whose key matches the prefix found so far.  Every position is valid for at most one of the two, so
+// one histogram of 512 bins (selection * 256 + digit) serves both.  A block takes whole rows, four columns per thread
+// and step when the row length is a multiple of four (16-byte loads of w and grad, 4-byte loads of the mask).
+__global__ void hist_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int out_f, int in_f,
                             int pass, SelectState* st) {
-    __shared__ unsigned int h[2][256];
-    for (int b = threadIdx.x; b < 512; b += blockDim.x) h[b >> 8][b & 255] = 0;
+    __shared__ unsigned int h[512];
+    for (int b = threadIdx.x; b < 512; b += blockDim.x) h[b] = 0;
     __syncthreads();
     const bool on0 = st[0].want != 0, on1 = st[1].want != 0;
     if (on0 || on1) {
         const unsigned int prefix0 = st[0].prefix, pmask0 = st[0].prefix_mask, prefix1 = st[1].prefix, pmask1 = st[1].prefix_mask;
         const int shift = 24 - 8 * pass;
-        const long long stride = (long long)gridDim.x * blockDim.x;
-        const long long rounds = (n + stride - 1) / stride;  // the same trip count for every lane: the warp votes inside
-        for (long long i = 0; i < rounds; ++i) {
-            const long long p = i * stride + (long long)blockIdx.x * blockDim.x + threadIdx.x;
-            bool take0 = false, take1 = false;
-            unsigned int key = 0;
-            if (p < n) {
-                if (mask[p]) {
-                    key = mag_bits(w[p]);
-                    take0 = on0 && (key & pmask0) == prefix0;
-                } else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) {
-                    key = ~mag_bits(grad[p]);
-                    take1 = on1 && (key & pmask1) == prefix1;
+        auto one = [&](bool inside, uint8_t m, float wv, float gv) {  // every lane of the warp calls it the same number of times
+            bool take = false;
+            unsigned int bin = 0;
+            if (inside) {
+                const unsigned int key = m ? mag_bits(wv) : ~mag_bits(gv);
+                take = m ? (on0 && (key & pmask0) == prefix0) : (on1 && (key & pmask1) == prefix1);
+                bin = (m ? 0u : 256u) + ((key >> shift) & 255u);
+            }
+            hist_add(h, take, bin);
+        };
+        for (int r = blockIdx.x; r < out_f; r += gridDim.x) {
+            if (row_count[r] == 0) continue;  // a neuron without weights is in neither pool
+            const size_t base = (size_t)r * in_f;
+            if ((in_f & 3) == 0) {
+                const uchar4* m4 = reinterpret_cast<const uchar4*>(mask + base);
+                const float4* w4 = reinterpret_cast<const float4*>(w + base);
+                const float4* g4 = reinterpret_cast<const float4*>(grad + base);
+                const int n4 = in_f >> 2;
+                for (int v0 = 0; v0 < n4; v0 += blockDim.x) {
+                    const int v = v0 + threadIdx.x;
+                    const bool inside = v < n4;
+                    uchar4 m = make_uchar4(0, 0, 0, 0);
+                    float4 wv = make_float4(0.f, 0.f, 0.f, 0.f), gv = wv;
+                    if (inside) {
+                        m = m4[v];
+                        if (m.x | m.y | m.z | m.w) wv = w4[v];
+                        if (!(m.x && m.y && m.z && m.w)) gv = g4[v];
+                    }
+                    one(inside, m.x, wv.x, gv.x);
+                    one(inside, m.y, wv.y, gv.y);
+                    one(inside, m.z, wv.z, gv.z);
+                    one(inside, m.w, wv.w, gv.w);
+                }
+            } else {
+                for (int c0 = 0; c0 < in_f; c0 += blockDim.x) {
+                    const int c = c0 + threadIdx.x;
+                    const bool inside = c < in_f;
+                    const uint8_t m = inside ? mask[base + c] : 0;
+                    one(inside, m, inside && m ? w[base + c] : 0.f, inside && !m ? grad[base + c] : 0.f);
                 }
             }
-            const unsigned int bin = (key >> shift) & 255u;
-            hist_add(h[0], take0, bin);
-            hist_add(h[1], take1, bin);
         }
     }
     __syncthreads();
     for (int b = threadIdx.x; b < 512; b += blockDim.x)
-        if (h[b >> 8][b & 255]) atomicAdd(&st[b >> 8].hist[b & 255], h[b >> 8][b & 255]);
+        if (h[b]) atomicAdd(&st[b >> 8].hist[b & 255], h[b]);
 }
 
 // One thread: the bin that holds the `want`-th element; narrow the prefix to it and clear the histogram.
@@ -162,10 +187,13 @@ __global__ void tie_count_kernel(const float* w, const uint8_t* mask, const floa
     const bool on0 = st[0].want != 0, on1 = st[1].want != 0;
     const unsigned int cut0 = st[0].prefix, cut1 = st[1].prefix;
     unsigned int c0 = 0, c1 = 0;
-    for (int e = 0; e < 16 && base + e < n; ++e) {
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
         const long long p = base + e;
-        if (mask[p]) c0 += (on0 && mag_bits(w[p]) == cut0) ? 1u : 0u;
-        else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) c1 += (on1 && ~mag_bits(grad[p]) == cut1) ? 1u : 0u;
+        if (p < n) {
+            if (mask[p]) c0 += (on0 && mag_bits(w[p]) == cut0) ? 1u : 0u;
+            else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) c1 += (on1 && ~mag_bits(grad[p]) == cut1) ? 1u : 0u;
+        }
     }
     if (c0) atomicAdd(&s[0], c0);
     if (c1) atomicAdd(&s[1], c1);
@@ -211,6 +239,7 @@ __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* gr
     unsigned int keys[16];
     uint8_t kind[16];  // 0: in neither pool, 1: active weight, 2: inactive position of a live neuron
     unsigned int mine0 = 0, mine1 = 0;
+#pragma unroll
     for (int e = 0; e < 16; ++e) {
         kind[e] = 0, keys[e] = 0;
         const long long p = base + e;
@@ -235,8 +264,9 @@ __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* gr
     // ties of each selection before this thread's first element
     unsigned long long rank0 = (unsigned long long)chunk_ties[blockIdx.x] + part[0][threadIdx.x] - mine0;
     unsigned long long rank1 = (unsigned long long)chunk_ties[(size_t)n_chunks + blockIdx.x] + part[1][threadIdx.x] - mine1;
+#pragma unroll
     for (int e = 0; e < 16; ++e) {
-        if (base + e >= n) break;
+        if (base + e >= n) continue;
         uint8_t f0 = 0, f1 = 0;
         if (kind[e] == 1 && want0 != 0) {
             if (keys[e] < cut0) f0 = 1;
@@ -257,9 +287,17 @@ __global__ void salient_kernel(const uint8_t* mask, const uint8_t* drop, const u
     if (threadIdx.x == 0) s = 0;
     __syncthreads();
     int c = 0;
-    for (int j = threadIdx.x; j < in_f; j += blockDim.x) {
-        const size_t p = (size_t)r * in_f + j;
-        c += ((mask[p] && !drop[p]) || grow_top[p]) ? 1 : 0;
+    const size_t base = (size_t)r * in_f;
+    if ((in_f & 3) == 0) {
+        const uchar4 *m4 = reinterpret_cast<const uchar4*>(mask + base), *d4 = reinterpret_cast<const uchar4*>(drop + base),
+                     *g4 = reinterpret_cast<const uchar4*>(grow_top + base);
+        for (int v = threadIdx.x; v < (in_f >> 2); v += blockDim.x) {
+            const uchar4 m = m4[v], d = d4[v], g = g4[v];
+            c += ((m.x && !d.x) || g.x) + ((m.y && !d.y) || g.y) + ((m.z && !d.z) || g.z) + ((m.w && !d.w) || g.w);
+        }
+    } else {
+        for (int j = threadIdx.x; j < in_f; j += blockDim.x)
+            c += ((mask[base + j] && !drop[base + j]) || grow_top[base + j]) ? 1 : 0;
     }
     atomicAdd(&s, c);
     __syncthreads();
@@ -431,13 +469,12 @@ Workspace carve(void* base, int out_f, int in_f) {
 }
 
 // Step 3's two selections over the whole layer (the first is also step 6's pruning set), in shared sweeps.
-bool layer_select_both(const float* w, const uint8_t* mask, const float* grad, const Workspace& ws, int in_f, long long n,
-                       cudaStream_t st) {
+bool layer_select_both(const float* w, const uint8_t* mask, const float* grad, const Workspace& ws, int out_f, int in_f,
+                       long long n, cudaStream_t st) {
     const int chunks = (int)((n + kChunk - 1) / kChunk);
-    const long long want_blocks = (n + kThreads * 8 - 1) / (kThreads * 8);
-    const int blocks = (int)(want_blocks < 1 ? 1 : want_blocks > 1184 ? 1184 : want_blocks);  // 8 CTAs per SM at most
+    const int hist_blocks = out_f < 1184 ? out_f : 1184;  // whole rows per block, 8 CTAs per SM at most
     for (int pass = 0; pass < 4; ++pass) {
-        hist_kernel<<<blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, pass, ws.state);
+        hist_kernel<<<hist_blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, out_f, in_f, pass, ws.state);
         pick_kernel<<<1, 32, 0, st>>>(pass, ws.state);
     }
     tie_count_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks);
@@ -469,7 +506,7 @@ extern "C" cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* g
     const long long n = (long long)out_features * in_features;
     row_count_kernel<<<out_features, kThreads, 0, st>>>(mask, out_features, in_features, ws.row_count);
     setup_kernel<<<1, kThreads, 0, st>>>(ws.row_count, out_features, in_features, (long long)K, ws.scalars, ws.state);
-    if (!layer_select_both(w, mask, grad, ws, in_features, n, st)) return CFI_ERR_CUDA;
+    if (!layer_select_both(w, mask, grad, ws, out_features, in_features, n, st)) return CFI_ERR_CUDA;
     salient_kernel<<<out_features, kThreads, 0, st>>>(mask, ws.drop, ws.grow_top, in_features, ws.salient);
     ablate_kernel<<<1, kThreads, 0, st>>>(ws.row_count, ws.salient, out_features, in_features, gamma_sal, ws.scalars, ws.survives);
     finalize_kernel<<<out_features, kThreads, 0, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
