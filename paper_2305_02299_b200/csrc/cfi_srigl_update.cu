@@ -365,9 +365,15 @@ __device__ void row_select(int in_f, int m, KeyOf key_of, unsigned int* hist /*2
     __syncthreads();
 }
 
-// Steps 6 and 7 for one neuron per block: prune, then trim or regrow to k'.
+// Steps 6 and 7 for one neuron per block: prune, then trim or regrow to k'.  The row's keys for the selection that turns
+// out to be needed (magnitudes of the kept weights when trimming, complemented gradient magnitudes of the free positions
+// when regrowing) are put in shared memory once, next to a byte per column that says whether the column is kept, so
+// that every 32-bit key value stays usable.  CACHED = false reads the operands from global memory on every pass
+// instead (rows too long for shared memory).
+template <bool CACHED>
 __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, const uint8_t* drop, const uint8_t* survives,
                                 int in_f, const Scalars* sc) {
+    extern __shared__ __align__(16) unsigned char row_smem[];  // CACHED: keys[in_f] (4 bytes each), then state[in_f] (1 byte each)
     __shared__ unsigned int hist[256];
     __shared__ RowCut cut;
     __shared__ int kept_count;
@@ -382,20 +388,41 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
         for (int c = threadIdx.x; c < in_f; c += blockDim.x) wr[c] = 0.0f, mr[c] = 0;
         return;
     }
+    unsigned int* keys = reinterpret_cast<unsigned int*>(row_smem);
+    uint8_t* state = row_smem + (size_t)in_f * 4;  // 1 = kept after step 6, 0 = free
     const int k_new = sc->k_new;
     if (threadIdx.x == 0) kept_count = 0;
     __syncthreads();
     int mine = 0;
-    for (int c = threadIdx.x; c < in_f; c += blockDim.x) mine += (mr[c] && !dr[c]) ? 1 : 0;
+    for (int c = threadIdx.x; c < in_f; c += blockDim.x) {
+        const bool is_kept = mr[c] && !dr[c];
+        if (CACHED) state[c] = is_kept ? 1 : 0;
+        mine += is_kept ? 1 : 0;
+    }
     atomicAdd(&kept_count, mine);
     __syncthreads();
     const int kept = kept_count;
     const bool trim = kept > k_new;
     const int m = trim ? kept - k_new : k_new - kept;
-    if (trim)  // the kept weights with the smallest magnitudes go
-        row_select(in_f, m, [&](int c, unsigned int& key) { key = mag_bits(wr[c]); return mr[c] && !dr[c]; }, hist, &cut);
-    else       // the free positions with the largest gradient magnitudes come
-        row_select(in_f, m, [&](int c, unsigned int& key) { key = ~mag_bits(gr[c]); return !(mr[c] && !dr[c]); }, hist, &cut);
+    if (CACHED && m > 0) {
+        for (int c = threadIdx.x; c < in_f; c += blockDim.x) {
+            const bool candidate = trim ? state[c] != 0 : state[c] == 0;
+            keys[c] = candidate ? (trim ? mag_bits(wr[c]) : ~mag_bits(gr[c])) : 0u;
+        }
+        __syncthreads();
+    }
+    auto key_of = [&](int c, unsigned int& key) {
+        if (CACHED) {
+            key = keys[c];
+            return trim ? state[c] != 0 : state[c] == 0;
+        }
+        const bool is_kept = mr[c] && !dr[c];
+        key = trim ? mag_bits(wr[c]) : ~mag_bits(gr[c]);
+        return trim ? is_kept : !is_kept;
+    };
+    // trim: the kept weights with the smallest magnitudes go; otherwise the free positions with the largest gradient
+    // magnitudes come
+    row_select(in_f, m, key_of, hist, &cut);
     // Apply, walking the row in column order so that ties on the cut key go to the smaller columns.
     if (threadIdx.x == 0) carry = 0;
     __syncthreads();
@@ -404,9 +431,9 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
         bool is_kept = false, candidate = false;
         unsigned int key = 0;
         if (c < in_f) {
-            is_kept = mr[c] && !dr[c];
+            is_kept = CACHED ? state[c] != 0 : (mr[c] && !dr[c]);
             candidate = trim ? is_kept : !is_kept;
-            key = trim ? mag_bits(wr[c]) : ~mag_bits(gr[c]);
+            if (cut.any && candidate) key = CACHED ? keys[c] : (trim ? mag_bits(wr[c]) : ~mag_bits(gr[c]));
         }
         const unsigned int tie = (cut.any && candidate && key == cut.cut) ? 1u : 0u;
         part[threadIdx.x] = tie;
@@ -421,11 +448,10 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
         if (c < in_f) {
             const bool selected = cut.any && candidate && (key < cut.cut || (tie && rank < cut.ties));
             bool on;
-            float val;
-            if (trim) on = is_kept && !selected, val = on ? wr[c] : 0.0f;
-            else on = is_kept || selected, val = is_kept ? wr[c] : 0.0f;
+            if (trim) on = is_kept && !selected;
+            else on = is_kept || selected;
+            if (!on || !is_kept) wr[c] = 0.0f;  // pruned, trimmed, free, or grown (starts at 0); a survivor keeps its value
             mr[c] = on ? 1 : 0;
-            wr[c] = val;
         }
         __syncthreads();
         if (threadIdx.x == kThreads - 1) carry += part[kThreads - 1];
@@ -509,7 +535,11 @@ extern "C" cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* g
     if (!layer_select_both(w, mask, grad, ws, out_features, in_features, n, st)) return CFI_ERR_CUDA;
     salient_kernel<<<out_features, kThreads, 0, st>>>(mask, ws.drop, ws.grow_top, in_features, ws.salient);
     ablate_kernel<<<1, kThreads, 0, st>>>(ws.row_count, ws.salient, out_features, in_features, gamma_sal, ws.scalars, ws.survives);
-    finalize_kernel<<<out_features, kThreads, 0, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
+    const size_t row_bytes = (size_t)in_features * 5;  // keys and one state byte per column
+    if (row_bytes <= 40 * 1024)
+        finalize_kernel<true><<<out_features, kThreads, row_bytes, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
+    else
+        finalize_kernel<false><<<out_features, kThreads, 0, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
     Scalars host{};
     if (cudaGetLastError() != cudaSuccess ||
         cudaMemcpyAsync(&host, ws.scalars, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess ||

@@ -38,7 +38,8 @@ def _compare(w, m, g, K, gamma):
 @pytest.mark.parametrize("out_f,in_f,k,n_abl,K,gamma", [
     (24, 40, 6, 0, 30, 0.3), (24, 40, 6, 3, 60, 0.5), (16, 16, 2, 0, 8, 1.0), (64, 96, 10, 5, 200, 0.3),
     (8, 8, 8, 0, 0, 0.3), (12, 30, 3, 0, 36, 0.0), (1, 5, 2, 0, 1, 0.5), (7, 4099, 33, 1, 100, 0.25),
-    (768, 3072, 307, 38, 70_000, 0.3), (3072, 768, 77, 154, 60_000, 0.3), (300, 1000, 10, 0, 2990, 0.9)])
+    (768, 3072, 307, 38, 70_000, 0.3), (3072, 768, 77, 154, 60_000, 0.3), (300, 1000, 10, 0, 2990, 0.9),
+    (6, 9000, 50, 1, 120, 0.25), (5, 9001, 40, 0, 199, 0.5)])   # rows too long for the shared-memory copy of the keys
 def test_matches_oracle(out_f, in_f, k, n_abl, K, gamma):
     w, m, g = _layer(out_f, in_f, k, n_abl, seed=out_f + in_f)
     _compare(w, m, g, K, gamma)
