@@ -298,6 +298,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
     ap.add_argument("--stack-only", type=int, default=0, metavar="ROWS",
                     help="run only the bf16 MLP stack leg on ROWS batch rows (for profiling) and print its JSON")
+    ap.add_argument("--srigl-only", action="store_true",
+                    help="run only the SRigL mask-update leg (for profiling) and print its JSON")
     args = ap.parse_args()
     W = inputs.workloads()
     w = W[args.workload]
@@ -313,6 +315,11 @@ def main():
     import torch
     from paper_2305_02299_b200 import binding as cfi   # raises if the CUDA library is missing
 
+    if args.srigl_only:
+        torch.cuda.set_device(0)
+        peaks, _ = measured_peaks()
+        print(json.dumps(srigl_update_leg(cfi, torch, peaks)))
+        return
     if args.stack_only:
         torch.cuda.set_device(0)
         peaks, _ = measured_peaks()
