@@ -82,3 +82,31 @@ def test_workspace_and_argument_checks():
     assert e.value.status == 2
     k_new, n_act = cfi.cfi_srigl_update(w, m, w, 3, 0.3)      # a layer with no active weight stays empty
     assert (k_new, n_act) == (0, 0) and int(m.sum()) == 0
+
+
+def test_update_then_pack_create_forward():
+    """The update's output is a constant-fan-in mask that the forward path accepts as is: cfi_pack (mask given, so grown
+    weights with value 0 count), cfi_create, cfi_forward, against the oracle forward on the oracle's updated layer."""
+    import torch
+    import oracle
+    from paper_2305_02299_b200 import binding as cfi
+    from parity import TOL, scaled_error
+    w, m, g = _layer(384, 512, 51, 20, seed=31)
+    w[7] *= 1e-6
+    g[7] *= 1e-6
+    gamma = float(np.float32(0.3))
+    w_ref, m_ref, k_ref, _ = srigl_update(w, m, g, 3000, gamma)
+    w_dev, m_dev, k_dev, n_dev = _run_device(w, m, g, 3000, gamma)
+    assert k_dev == k_ref and np.array_equal(m_dev, m_ref)
+    v, ix, rows = cfi.cfi_pack(w_dev, m_dev)
+    assert v.shape == (n_dev, k_dev) and np.any(v == 0.0)            # freshly grown weights are kept entries of value 0
+    bias = inputs.make_layer(512, 384, 51, seed=32).bias
+    x = inputs.make_x(40, 512, seed=33)
+    vr, ir, rr = oracle.pack(w_ref, m_ref)
+    y_ref, S = oracle.forward(vr, ir, rr, bias, 512, 384, x, want_scale=True)
+    layer = cfi.cfi_create(v, ix, rows, bias, 512, 384)
+    y = torch.empty((40, 384), device="cuda")
+    cfi.cfi_forward(layer, torch.from_numpy(x).cuda(), y, 40)
+    torch.cuda.synchronize()
+    layer.close()
+    assert scaled_error(y.cpu().numpy(), y_ref, S) <= TOL["f32"]
