@@ -162,6 +162,23 @@ cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* grad, int32_
                               int32_t* n_active_new, cfi_stream_t stream);
 
 /*
+ * cfi_pack_device — cfi_pack for a weight and mask that live in device memory (e.g. right after cfi_srigl_update):
+ * the same condensed arrays, the same order (columns ascending within a row, rows ascending), written to device
+ * memory.  The mask is required and defines the structure.
+ *
+ *   w_dense, mask   device, [out_features, in_features] float / uint8
+ *   workspace       device, 256-byte aligned, at least 8 * out_features + 256 bytes
+ *   k, n_active     host, written on every successful call
+ *   values, indices, active_rows   device, [n_active, k] / [n_active, k] / [n_active]; all three NULL: size query
+ *
+ * Runs on `stream` and waits for it.  CFI_ERR_NOT_CONSTANT_FAN_IN as for cfi_pack; CFI_ERR_NULL, CFI_ERR_SHAPE,
+ * CFI_ERR_ALIGNMENT, CFI_ERR_BUFFER_TOO_SMALL, CFI_ERR_CUDA.
+ */
+cfi_status_t cfi_pack_device(const float* w_dense, const uint8_t* mask, int32_t out_features, int32_t in_features,
+                             void* workspace, size_t workspace_bytes, int32_t* k, int32_t* n_active, float* values,
+                             int32_t* indices, int32_t* active_rows, cfi_stream_t stream);
+
+/*
  * cfi_create — build a device-resident layer from condensed arrays (the inputs w and indx of
  * Algorithm 1, plus the bias that Sec. 4.4 extracts with the weights).
  *

@@ -7,7 +7,7 @@ loaded on first use so that the input generators stay importable on their own.
 """
 import importlib
 
-_BINDING_NAMES = ("cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_srigl_update", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
+_BINDING_NAMES = ("cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_srigl_update", "cfi_pack_device", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
                   "cfi_destroy", "cfi_device_status", "cfi_status_string", "cfi_layer_info",
                   "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static", "cfi_probe_device", "cfi_choose_variant",
                   "cfi_dense_tile_shape",

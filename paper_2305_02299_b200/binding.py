@@ -25,7 +25,7 @@ _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE,
 _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_srigl_workspace_bytes",
-           "cfi_srigl_update", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
+           "cfi_srigl_update", "cfi_pack_device", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_dense_tile_shape", "cfi_device_status", "cfi_destroy",
            "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static",
            "cfi_probe_device")
@@ -74,6 +74,7 @@ def _load() -> ctypes.CDLL:
     lib.cfi_compact_consumer.argtypes = [i32p, ci, ci, f32p, f32p, i32p, i32p, ci, ci, f32p, ci]
     lib.cfi_srigl_workspace_bytes.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_size_t)]
     lib.cfi_srigl_update.argtypes = [vp, vp, vp, ci, ci, ctypes.c_int64, ctypes.c_float, vp, ctypes.c_size_t, i32p, i32p, vp]
+    lib.cfi_pack_device.argtypes = [vp, vp, ci, ci, vp, ctypes.c_size_t, i32p, i32p, vp, vp, vp, vp]
     lib.cfi_create.argtypes = [f32p, i32p, i32p, f32p, ci, ci, ci, ci, ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
     lib.cfi_forward.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_forward_variant.argtypes = [vp, vp, vp, ci, vp, ctypes.c_int]
@@ -227,6 +228,26 @@ def cfi_srigl_update(w, mask, grad, K: int, gamma_sal: float, stream=None):
                                  nbytes.value, ctypes.byref(k_new), ctypes.byref(n_act), _stream_handle(stream)),
            "cfi_srigl_update")
     return k_new.value, n_act.value
+
+
+def cfi_pack_device(w, mask, stream=None):
+    """cfi_pack on device tensors w (float32) and mask (uint8), both [out, in] and contiguous.  Returns device tensors
+    (values [n_active, k] float32, indices [n_active, k] int32, active_rows [n_active] int32)."""
+    import torch
+    out_f, in_f = w.shape
+    ws = torch.empty(8 * out_f + 512, dtype=torch.uint8, device=w.device)
+    base = (ws.data_ptr() + 255) & ~255
+    k, na = ctypes.c_int32(0), ctypes.c_int32(0)
+    st = _stream_handle(stream)
+    _check(_lib.cfi_pack_device(_dev_ptr(w), _dev_ptr(mask), out_f, in_f, base, 8 * out_f + 256, ctypes.byref(k),
+                                ctypes.byref(na), None, None, None, st), "cfi_pack_device")
+    values = torch.empty((na.value, k.value), dtype=torch.float32, device=w.device)
+    indices = torch.empty((na.value, k.value), dtype=torch.int32, device=w.device)
+    rows = torch.empty((na.value,), dtype=torch.int32, device=w.device)
+    if na.value:
+        _check(_lib.cfi_pack_device(_dev_ptr(w), _dev_ptr(mask), out_f, in_f, base, 8 * out_f + 256, ctypes.byref(k),
+                                    ctypes.byref(na), _dev_ptr(values), _dev_ptr(indices), _dev_ptr(rows), st), "cfi_pack_device")
+    return values, indices, rows
 
 
 def cfi_forward(layer: Layer, x, y, batch: int, stream=None) -> None:

@@ -510,6 +510,70 @@ bool layer_select_both(const float* w, const uint8_t* mask, const float* grad, c
     return cudaGetLastError() == cudaSuccess;
 }
 
+// ---- cfi_pack_device: the condensed arrays straight from device-resident w and mask -------------------------------
+
+// Single block: rank of every non-empty row among the non-empty rows, their number, the common fan-in, and whether the
+// fan-in really is common.  info = {n_active, k, constant (1/0)}.
+__global__ void pack_rows_kernel(const int* row_count, int out_f, int* row_rank, int* info) {
+    __shared__ unsigned int part[kThreads];
+    __shared__ unsigned int carry;
+    __shared__ int k_min, k_max;
+    if (threadIdx.x == 0) carry = 0, k_min = 0x7fffffff, k_max = 0;
+    __syncthreads();
+    for (int r0 = 0; r0 < out_f; r0 += kThreads) {
+        const int r = r0 + threadIdx.x;
+        const int cnt = r < out_f ? row_count[r] : 0;
+        const unsigned int live = cnt > 0 ? 1u : 0u;
+        if (live) atomicMin(&k_min, cnt), atomicMax(&k_max, cnt);
+        part[threadIdx.x] = live;
+        __syncthreads();
+        for (int off = 1; off < kThreads; off <<= 1) {
+            const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
+            __syncthreads();
+            part[threadIdx.x] += add;
+            __syncthreads();
+        }
+        if (r < out_f) row_rank[r] = live ? (int)(carry + part[threadIdx.x] - 1) : -1;
+        __syncthreads();
+        if (threadIdx.x == kThreads - 1) carry += part[kThreads - 1];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) info[0] = (int)carry, info[1] = k_max, info[2] = (carry == 0 || k_min == k_max) ? 1 : 0;
+}
+
+// One block per row: its kept entries in increasing column order to values / indices of its rank.
+__global__ void pack_fill_kernel(const float* w, const uint8_t* mask, const int* row_rank, int in_f, int k, float* values,
+                                 int32_t* indices, int32_t* active_rows) {
+    __shared__ unsigned int part[kThreads];
+    __shared__ unsigned int carry;
+    const int r = blockIdx.x, rank = row_rank[r];
+    if (rank < 0) return;
+    if (threadIdx.x == 0) carry = 0, active_rows[rank] = r;
+    __syncthreads();
+    const float* wr = w + (size_t)r * in_f;
+    const uint8_t* mr = mask + (size_t)r * in_f;
+    for (int c0 = 0; c0 < in_f; c0 += kThreads) {
+        const int c = c0 + threadIdx.x;
+        const unsigned int kept = (c < in_f && mr[c]) ? 1u : 0u;
+        part[threadIdx.x] = kept;
+        __syncthreads();
+        for (int off = 1; off < kThreads; off <<= 1) {
+            const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
+            __syncthreads();
+            part[threadIdx.x] += add;
+            __syncthreads();
+        }
+        if (kept) {
+            const size_t at = (size_t)rank * k + carry + part[threadIdx.x] - 1;
+            values[at] = wr[c];
+            indices[at] = c;
+        }
+        __syncthreads();
+        if (threadIdx.x == kThreads - 1) carry += part[kThreads - 1];
+        __syncthreads();
+    }
+}
+
 }  // namespace
 
 extern "C" cfi_status_t cfi_srigl_workspace_bytes(int32_t out_features, int32_t in_features, size_t* bytes) {
@@ -549,5 +613,38 @@ extern "C" cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* g
     }
     *k_new = host.k_new;
     *n_active_new = host.live_after;
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_pack_device(const float* w_dense, const uint8_t* mask, int32_t out_features, int32_t in_features,
+                                        void* workspace, size_t workspace_bytes, int32_t* k, int32_t* n_active, float* values,
+                                        int32_t* indices, int32_t* active_rows, cfi_stream_t stream) {
+    if (!w_dense || !mask || !workspace || !k || !n_active) return CFI_ERR_NULL;
+    if (out_features < 1 || in_features < 1 || (int64_t)out_features * in_features > ((int64_t)1 << 31)) return CFI_ERR_SHAPE;
+    const bool fill = values || indices || active_rows;
+    if (fill && !(values && indices && active_rows)) return CFI_ERR_NULL;
+    if (((uintptr_t)workspace & 255) != 0) return CFI_ERR_ALIGNMENT;
+    if (workspace_bytes < (size_t)out_features * 8 + 256) return CFI_ERR_BUFFER_TOO_SMALL;
+    int* row_count = static_cast<int*>(workspace);
+    int* row_rank = row_count + out_features;
+    int* info = row_rank + out_features;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    row_count_kernel<<<out_features, kThreads, 0, st>>>(mask, out_features, in_features, row_count);
+    pack_rows_kernel<<<1, kThreads, 0, st>>>(row_count, out_features, row_rank, info);
+    int host[3] = {0, 0, 0};
+    if (cudaGetLastError() != cudaSuccess || cudaMemcpyAsync(host, info, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
+    if (!host[2]) return CFI_ERR_NOT_CONSTANT_FAN_IN;
+    *n_active = host[0];
+    *k = host[0] ? host[1] : 0;
+    if (!fill || host[0] == 0) return CFI_OK;
+    pack_fill_kernel<<<out_features, kThreads, 0, st>>>(w_dense, mask, row_rank, in_features, host[1], values, indices, active_rows);
+    if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
     return CFI_OK;
 }

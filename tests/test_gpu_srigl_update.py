@@ -110,3 +110,33 @@ def test_update_then_pack_create_forward():
     torch.cuda.synchronize()
     layer.close()
     assert scaled_error(y.cpu().numpy(), y_ref, S) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("out_f,in_f,k,n_abl", [(24, 40, 6, 0), (300, 1000, 10, 37), (7, 4099, 33, 1), (768, 3072, 307, 38), (5, 9, 9, 0)])
+def test_pack_device_equals_host_pack(out_f, in_f, k, n_abl):
+    """cfi_pack_device on device-resident w and mask gives exactly cfi_pack's arrays (and the oracle's)."""
+    import torch
+    import oracle
+    from paper_2305_02299_b200 import binding as cfi
+    w, m, _ = _layer(out_f, in_f, k, n_abl, seed=out_f)
+    zr, zc = np.nonzero(m == 1)
+    w[zr[::7], zc[::7]] = 0.0                                    # kept entries of value 0 still count (the mask decides)
+    v, ix, rows = cfi.cfi_pack_device(torch.from_numpy(w).cuda(), torch.from_numpy(m).cuda())
+    vh, ih, rh = cfi.cfi_pack(w, m)
+    vo, io, ro = oracle.pack(w, m)
+    assert np.array_equal(v.cpu().numpy(), vh) and np.array_equal(ix.cpu().numpy(), ih) and np.array_equal(rows.cpu().numpy(), rh)
+    assert np.array_equal(vh, vo) and np.array_equal(ih, io) and np.array_equal(rh, ro)
+
+
+def test_pack_device_errors_and_empty():
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    w, m, _ = _layer(10, 20, 4, 2, seed=3)
+    m2 = m.copy()
+    row = int(np.nonzero(m2.sum(1))[0][0])
+    m2[row, np.nonzero(m2[row])[0][0]] = 0                        # one row keeps one entry fewer
+    with pytest.raises(cfi.CfiError) as e:
+        cfi.cfi_pack_device(torch.from_numpy(w).cuda(), torch.from_numpy(m2).cuda())
+    assert e.value.status == 3
+    v, ix, rows = cfi.cfi_pack_device(torch.zeros((4, 8), device="cuda"), torch.zeros((4, 8), device="cuda", dtype=torch.uint8))
+    assert v.shape == (0, 0) and rows.shape == (0,)
