@@ -207,6 +207,14 @@ cfi_status_t cfi_create(const float* values, const int32_t* indices, const int32
  *
  * Every element of y is written (ablated columns too).  batch == 0 succeeds and launches nothing.
  * The return value reports argument and launch errors only.
+ *
+ * Non-finite inputs.  The condensed kernels (CFI_VARIANT_SIMPLE, SPLITK, BATCH) read only the columns a row
+ * indexes, so an inf or NaN in a column that no row (or not this row) uses leaves that row's output alone.
+ * CFI_VARIANT_DENSE_TC computes the dense masked product, in which such a column meets weights of 0 and
+ * 0 * inf = NaN reaches every output of that batch row (for fp32 layers also through the operand split).  The two
+ * agree for finite x, which is the equivalence the paper states (appendix "Condensed matrix multiplication").
+ * cfi_forward picks by speed; a caller that needs the condensed behaviour for non-finite activations calls
+ * cfi_forward_variant with one of the condensed variants.
  */
 cfi_status_t cfi_forward(const cfi_layer_t* layer, const void* x, void* y, int32_t batch, cfi_stream_t stream);
 
