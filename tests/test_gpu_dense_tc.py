@@ -78,6 +78,26 @@ def test_dense_tc_bf16_many_tiles_per_sm(in_f, out_f, k, nabl, B, act):
     assert np.array_equal(y, y2)
 
 
+def test_dense_tc_bf16_cluster_split_is_exercised():
+    """bf16, few tiles and a long K: the one-tile kernel with K split over clusters of several sizes (asserted through
+    cfi_dense_tile_shape), each case against the oracle; and a case with enough tiles that it does not split."""
+    from paper_2305_02299_b200 import binding as cfi
+    seen = set()
+    for in_f, out_f, k, nabl, B, act in [(3072, 768, 307, 77, 256, "none"), (3072, 768, 307, 77, 64, "gelu"), (4096, 256, 41, 3, 100, "gelu"),
+                                          (1000, 72, 100, 5, 257, "none"), (520, 640, 52, 30, 128, "gelu"), (256, 3072, 26, 0, 700, "gelu")]:
+        L = inputs.make_layer(in_f, out_f, k, n_ablated=nabl, seed=in_f + B)
+        x = inputs.make_x(B, in_f, seed=B)
+        y_ref, S = oracle_layer(L, x, "bf16", act)
+        dl = device_layer(L, "bf16", act)
+        shape = cfi.cfi_dense_tile_shape(dl, B)
+        seen.add(shape)
+        y = run_device(dl, x, "bf16", "dense_tc")
+        dl.close()
+        assert scaled_error(y, y_ref, S) <= TOL["bf16"], (in_f, out_f, B, shape)
+    clusters = {c for t, c in seen if t == 128}
+    assert 1 in clusters and len([c for c in clusters if c > 1]) >= 2, seen
+
+
 def test_dense_tf32_wide_dynamic_range():
     """Inputs spread over many binades: the split must hold for every magnitude, not only for N(0,1)."""
     L = inputs.make_layer(512, 128, 51, n_ablated=7, seed=9)
