@@ -169,6 +169,67 @@ __device__ __forceinline__ float activate_tc(float v) {
     }
 }
 
+// Two fp32 numbers in one 64-bit register, for the packed fp32 instructions of sm_100 (one issue slot for two
+// results: the epilogue of a GELU layer is bound by instruction issue, not by the tensor pipe).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// act(acc + bias) of two neighbouring outputs, rounded to bf16 and packed (first output in the low half).
+// The GELU is the formula of activate_tc with its polynomial and products in packed fp32, and with the two
+// signs of v merged into one expression: with q = p t e (a function of |v|, 0 < q <= 1/2),
+// v Phi(v) = max(v, 0) - |v| q for either sign, and the negative tail is still a plain product.
+template <int ACT>
+__device__ __forceinline__ uint32_t bias_act_bf16x2(float a0, float a1, float b0, float b1) {
+    float r0, r1;
+    if constexpr (ACT != CFI_ACT_GELU_ERF) {
+        r0 = a0 + b0;
+        r1 = a1 + b1;
+    } else {
+        float v0, v1, t0, t1, e0, e1, q0, q1;
+        const uint64_t v = f2_add(f2_pack(a0, a1), f2_pack(b0, b1));
+        f2_unpack(v, v0, v1);
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t0) : "f"(fmaf(fabsf(v0), 0.23164189f, 1.0f)));
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t1) : "f"(fmaf(fabsf(v1), 0.23164189f, 1.0f)));
+        const uint64_t t = f2_pack(t0, t1);
+        uint64_t p = f2_fma(f2_pack(0.5307027145f, 0.5307027145f), t, f2_pack(-0.7265760135f, -0.7265760135f));
+        p = f2_fma(p, t, f2_pack(0.7107068705f, 0.7107068705f));
+        p = f2_fma(p, t, f2_pack(-0.142248368f, -0.142248368f));
+        p = f2_fma(p, t, f2_pack(0.127414796f, 0.127414796f));
+        const uint64_t x2 = f2_mul(f2_mul(v, f2_pack(-0.72134752f, -0.72134752f)), v);  // -v^2 log2(e) / 2
+        float s0, s1;
+        f2_unpack(x2, s0, s1);
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(s0));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(s1));
+        const uint64_t q = f2_mul(f2_mul(p, t), f2_pack(e0, e1));
+        f2_unpack(q, q0, q1);
+        r0 = fmaf(-fabsf(v0), q0, fmaxf(v0, 0.0f));
+        r1 = fmaf(-fabsf(v1), q1, fmaxf(v1, 0.0f));
+    }
+    const __nv_bfloat162 pk = __floats2bfloat162_rn(r0, r1);
+    return *reinterpret_cast<const uint32_t*>(&pk);
+}
+
 // Shared memory (offsets from the first 1024-byte boundary): the ring, then barriers and small tables.
 //   ring      kTcStages x [A 128 x 64 bf16 | B 128 x 64 bf16]; after the main loop its first 32 KB hold the y tile
 //   +0        full[kTcStages], +32 empty[kTcStages], +64 accumulator barrier, +72 tensor-memory base address
@@ -281,13 +342,8 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
 #pragma unroll
                     for (int e4 = 0; e4 < 4; ++e4) {
                         const float4 bv = *reinterpret_cast<const float4*>(bias_s + c + 16 * h + 4 * e4);
-                        const float r0 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 0]) + bv.x);
-                        const float r1 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 1]) + bv.y);
-                        const float r2 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 2]) + bv.z);
-                        const float r3 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 3]) + bv.w);
-                        const __nv_bfloat162 p01 = __floats2bfloat162_rn(r0, r1), p23 = __floats2bfloat162_rn(r2, r3);
-                        packed[2 * e4] = *reinterpret_cast<const uint32_t*>(&p01);
-                        packed[2 * e4 + 1] = *reinterpret_cast<const uint32_t*>(&p23);
+                        packed[2 * e4] = bias_act_bf16x2<ACT>(__uint_as_float(v[h][4 * e4 + 0]), __uint_as_float(v[h][4 * e4 + 1]), bv.x, bv.y);
+                        packed[2 * e4 + 1] = bias_act_bf16x2<ACT>(__uint_as_float(v[h][4 * e4 + 2]), __uint_as_float(v[h][4 * e4 + 3]), bv.z, bv.w);
                     }
                     const int ch = (c + 16 * h) >> 3;  // 16-byte chunk of columns .. +7; the next one holds +8 .. +15
                     *reinterpret_cast<uint4*>(smem_at(ring + row * 256 + ((ch ^ (row & 15)) << 4))) =

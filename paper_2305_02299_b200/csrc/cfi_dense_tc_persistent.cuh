@@ -166,13 +166,8 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
 #pragma unroll
                         for (int e4 = 0; e4 < 4; ++e4) {
                             const float4 bv = *reinterpret_cast<const float4*>(bias_s + 128 * half + c + 16 * h + 4 * e4);
-                            const float r0 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 0]) + bv.x);
-                            const float r1 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 1]) + bv.y);
-                            const float r2 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 2]) + bv.z);
-                            const float r3 = activate_tc<ACT>(__uint_as_float(v[h][4 * e4 + 3]) + bv.w);
-                            const __nv_bfloat162 p01 = __floats2bfloat162_rn(r0, r1), p23 = __floats2bfloat162_rn(r2, r3);
-                            packed[2 * e4] = *reinterpret_cast<const uint32_t*>(&p01);
-                            packed[2 * e4 + 1] = *reinterpret_cast<const uint32_t*>(&p23);
+                            packed[2 * e4] = bias_act_bf16x2<ACT>(__uint_as_float(v[h][4 * e4 + 0]), __uint_as_float(v[h][4 * e4 + 1]), bv.x, bv.y);
+                            packed[2 * e4 + 1] = bias_act_bf16x2<ACT>(__uint_as_float(v[h][4 * e4 + 2]), __uint_as_float(v[h][4 * e4 + 3]), bv.z, bv.w);
                         }
                         const int ch = (c + 16 * h) >> 3;
                         *reinterpret_cast<uint4*>(smem_at(staging + row * 256 + ((ch ^ (row & 15)) << 4))) =
