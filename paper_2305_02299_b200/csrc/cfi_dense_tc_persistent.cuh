@@ -14,9 +14,13 @@
 //                       does not drain between tiles);
 //   warp 1, one lane    MMA issuer (M = 128, N = 256, K = 16): tile i accumulates into tensor-memory buffer i mod 2
 //                       (2 x 256 columns); before reusing a buffer it waits until the epilogue has read it;
-//   warps 2..17         epilogue of tile i while the MMAs of tile i + 1 run, in two halves of 128 columns:
-//                       tcgen05.ld (one batch row and 32 columns per thread), bias, activation, bf16, a staging
-//                       half-tile in shared memory, 256-byte runs per batch row to y.
+//   warps 2..17         epilogue of tile i while the MMAs of tile i + 1 run, in four quarters of 64 columns:
+//                       tcgen05.ld (one batch row and 16 columns per thread), bias (read from global memory, the same
+//                       64 bytes for a whole warp), activation in packed fp32, bf16, one of two 16 KB staging boxes in
+//                       shared memory (128-byte swizzle), and a TMA store of the box issued by one thread, which
+//                       clips rows past the batch and columns past out.  While the store of one box drains, the
+//                       next quarter is computed into the other; the issuing thread waits for a box's store to have
+//                       read shared memory (cp.async.bulk.wait_group.read) one barrier before the box is written again.
 //
 // Tiles are numbered with the output tile fastest, and CTA c takes tiles c, c + gridDim.x, ...: CTAs running at the
 // same time share a batch tile of x, and Wd (4.7 MB for 768 x 3072) stays in L2.
@@ -28,7 +32,8 @@
 
 constexpr int kTpN = 256, kTpStages = 4, kTpEpilogueWarps = 16, kTpThreads = 64 + 32 * kTpEpilogueWarps;
 constexpr uint32_t kTpABytes = kTcM * kTcK * 2, kTpBBytes = kTpN * kTcK * 2, kTpStageBytes = kTpABytes + kTpBBytes;  // 16 + 32 KB
-constexpr uint32_t kTpStagingBytes = kTcM * 128 * 2;  // half a y tile, bf16: 32 KB
+constexpr uint32_t kTpStoreBoxBytes = kTcM * 64 * 2;       // one TMA store box of y: 128 rows x 64 bf16 = 16 KB
+constexpr uint32_t kTpStagingBytes = 2 * kTpStoreBoxBytes;  // two boxes, written and stored alternately
 constexpr size_t kTpSmemBytes = 1024 + kTpStages * kTpStageBytes + kTpStagingBytes + 2048;  // exactly 227 KB
 constexpr uint32_t kTpTmemCols = 512;
 constexpr uint32_t kTpInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTpN >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
@@ -41,12 +46,12 @@ __device__ __forceinline__ void umma_bf16_n256(uint32_t tmem_d, uint64_t desc_a,
         : "memory");
 }
 
-// Shared memory from the first 1024-byte boundary: ring (4 x 48 KB) | staging (32 KB) | control:
-//   +0 full[4], +32 empty[4], +64 acc_full[2], +80 acc_empty[2], +96 tensor-memory base, +128 bias[256].
+// Shared memory from the first 1024-byte boundary: ring (4 x 48 KB) | two store boxes (2 x 16 KB) | control:
+//   +0 full[4], +32 empty[4], +64 acc_full[2], +80 acc_empty[2], +96 tensor-memory base.
 template <int ACT>
 __global__ void __launch_bounds__(kTpThreads, 1)
 cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                               __nv_bfloat16* __restrict__ y, int batch, int n_tiles_n, int n_tiles) {
+                               const __grid_constant__ CUtensorMap map_y, int batch, int n_tiles_n, int n_tiles) {
     pdl_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t base = ((smem_u32(0) + 1023u) & ~1023u) - smem_u32(0);
@@ -54,13 +59,13 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
     const uint32_t full0 = smem_u32(ctl), empty0 = smem_u32(ctl + 32), acc_full0 = smem_u32(ctl + 64),
                    acc_empty0 = smem_u32(ctl + 80);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_at(ctl + 96));
-    float* bias_s = reinterpret_cast<float*>(smem_at(ctl + 128));  // [kTpN], of the tile in the epilogue
     const int k_blocks = (L.in + kTcK - 1) / kTcK;
     const int first = blockIdx.x, stride = gridDim.x;
 
     if (tid == 0) {
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_w);
+        prefetch_tensormap(&map_y);
         for (int s = 0; s < kTpStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
@@ -75,10 +80,6 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(ctl + 96)), "r"(kTpTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (tid >= 64 && tid < 64 + kTpN && first < n_tiles) {  // bias of the first tile
-        const int n = (first % n_tiles_n) * kTpN + tid - 64;
-        bias_s[tid - 64] = n < L.out ? L.bias[n] : 0.0f;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -129,67 +130,60 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
         // ---------------------------------------------------------------- epilogue
         const int et = tid - 64;
         const int q = warp & 3;             // tensor-memory lanes 32 q .. 32 q + 31
-        const int cq = (warp - 2) >> 2;     // which 32 of a half's 128 columns
+        const int cq = (warp - 2) >> 2;     // which 16 of a quarter's 64 columns
         const int row = 32 * q + lane;      // batch row of the tile held by this thread
-        uint32_t i = 0;
+        uint32_t i = 0, step = 0;           // tiles and quarter-tiles so far
         for (int t = first; t < n_tiles; t += stride, ++i) {
             const int m0 = (t / n_tiles_n) * kTcM, n0 = (t % n_tiles_n) * kTpN;
             const uint32_t b = i & 1u;
-            // Bias of the next tile: requested now, put into bias_s when this tile no longer reads it.
-            const int t_next = t + stride;
-            float bias_next = 0.0f;
-            if (et < kTpN && t_next < n_tiles) {
-                const int n = (t_next % n_tiles_n) * kTpN + et;
-                bias_next = n < L.out ? L.bias[n] : 0.0f;
-            }
             if (ok) ok = mbar_wait(acc_full0 + 8 * b, (i >> 1) & 1u, kTcSpinLimit);
             ok = __all_sync(0xffffffffu, ok);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
+            for (int qs = 0; qs < 4; ++qs, ++step) {
+                // Staging buffer step mod 2: one TMA box of 128 rows x 64 bf16 columns in the 128-byte swizzle.  Its
+                // last store (two steps ago) was waited for by thread 0 before the barrier of the step in between.
+                const uint32_t stage = staging + (step & 1u) * kTpStoreBoxBytes;
+                const int c = 64 * qs + 16 * cq;  // column within the tile
                 if (ok) {
-                    // Staging half-tile: 128 rows x 256 bytes, 16-byte chunks permuted by chunk ^ (row & 15).
-                    const int c = 32 * cq;  // column within the half
-                    uint32_t v[2][16];
-                    const uint32_t t_acc =
-                        tmem_base + ((uint32_t)(32 * q) << 16) + b * (uint32_t)kTpN + (uint32_t)(128 * half + c);
-                    tmem_ld16(t_acc, v[0]);
-                    tmem_ld16(t_acc + 16u, v[1]);
+                    float4 bv[4];  // bias straight from global memory: every lane of a warp reads the same 64 bytes
+#pragma unroll
+                    for (int e4 = 0; e4 < 4; ++e4) {
+                        const int n = n0 + c + 4 * e4;
+                        bv[e4] = n < L.out ? __ldg(reinterpret_cast<const float4*>(L.bias + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    uint32_t v[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(32 * q) << 16) + b * (uint32_t)kTpN + (uint32_t)c, v);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (half == 1) {  // the buffer is free for tile i + 2 once every epilogue warp has its values
+                    if (qs == 3) {  // the buffer is free for tile i + 2 once every epilogue warp has its values
                         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                         if (lane == 0) mbar_arrive(acc_empty0 + 8 * b);
                     }
+                    uint32_t packed[8];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t packed[8];
-#pragma unroll
-                        for (int e4 = 0; e4 < 4; ++e4) {
-                            const float4 bv = *reinterpret_cast<const float4*>(bias_s + 128 * half + c + 16 * h + 4 * e4);
-                            packed[2 * e4] = bias_act_bf16x2<ACT>(__uint_as_float(v[h][4 * e4 + 0]), __uint_as_float(v[h][4 * e4 + 1]), bv.x, bv.y);
-                            packed[2 * e4 + 1] = bias_act_bf16x2<ACT>(__uint_as_float(v[h][4 * e4 + 2]), __uint_as_float(v[h][4 * e4 + 3]), bv.z, bv.w);
-                        }
-                        const int ch = (c + 16 * h) >> 3;
-                        *reinterpret_cast<uint4*>(smem_at(staging + row * 256 + ((ch ^ (row & 15)) << 4))) =
-                            make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                        *reinterpret_cast<uint4*>(smem_at(staging + row * 256 + (((ch + 1) ^ (row & 15)) << 4))) =
-                            make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                    for (int e4 = 0; e4 < 4; ++e4) {
+                        packed[2 * e4] = bias_act_bf16x2<ACT>(__uint_as_float(v[4 * e4 + 0]), __uint_as_float(v[4 * e4 + 1]), bv[e4].x, bv[e4].y);
+                        packed[2 * e4 + 1] = bias_act_bf16x2<ACT>(__uint_as_float(v[4 * e4 + 2]), __uint_as_float(v[4 * e4 + 3]), bv[e4].z, bv[e4].w);
                     }
+                    const int ch = 2 * cq;  // 16-byte chunk of the row's 128 bytes; chunk j sits at j ^ (row & 7)
+                    *reinterpret_cast<uint4*>(smem_at(stage + row * 128 + ((ch ^ (row & 7)) << 4))) =
+                        make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    *reinterpret_cast<uint4*>(smem_at(stage + row * 128 + (((ch + 1) ^ (row & 7)) << 4))) =
+                        make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the TMA store reads these writes
                 }
-                asm volatile("bar.sync 1, %0;" ::"n"(32 * kTpEpilogueWarps) : "memory");  // staging half-tile complete
-                if (ok) {
-                    for (int r = et >> 4; r < kTcM; r += 2 * kTpEpilogueWarps) {  // 16 threads per row, 32 rows per pass
-                        const int ch = et & 15, m = m0 + r, n = n0 + 128 * half + 8 * ch;
-                        if (m < batch && n < L.out) {
-                            const uint4 val = *reinterpret_cast<const uint4*>(smem_at(staging + r * 256 + ((ch ^ (r & 15)) << 4)));
-                            *reinterpret_cast<uint4*>(y + (size_t)m * L.out + n) = val;
-                        }
-                    }
+                if (et == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the other buffer's store has read it
+                asm volatile("bar.sync 1, %0;" ::"n"(32 * kTpEpilogueWarps) : "memory");  // the box is complete
+                if (et == 0 && ok && n0 + 64 * qs < L.out) {  // rows past the batch and columns past out are clipped
+                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                                     reinterpret_cast<uint64_t>(&map_y)),
+                                 "r"(smem_u32(stage)), "r"(n0 + 64 * qs), "r"(m0)
+                                 : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
-                if (half == 1 && et < kTpN) bias_s[et] = bias_next;  // every read of this tile's bias is behind the barrier above
-                asm volatile("bar.sync 1, %0;" ::"n"(32 * kTpEpilogueWarps) : "memory");  // staging (and bias) may be rewritten
             }
         }
+        if (et == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // every store has landed before the CTA ends
     }
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

@@ -1014,14 +1014,16 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
     const int64_t n_tiles = (int64_t)wide_x * grid_y;
     if (tc_bf16_persistent(l, batch)) {
         const int ctas = l->sm_count;
+        CUtensorMap map_y;  // y leaves through TMA stores of 128-row x 64-column boxes
+        if (!encode_map(&map_y, y, (uint64_t)batch, (uint64_t)l->d.out, 2, kTcM)) return CFI_ERR_SHAPE;
         if (l->d.act == CFI_ACT_GELU_ERF) {
             if (cfi_status_t e = set_smem<cfi_dense_tc_persistent_kernel<CFI_ACT_GELU_ERF>>(kTpSmemBytes, l->device)) return e;
             return launch_pdl(cfi_dense_tc_persistent_kernel<CFI_ACT_GELU_ERF>, dim3(ctas), kTpThreads, kTpSmemBytes, st, l->d,
-                              map_x, l->map_w_wide, static_cast<__nv_bfloat16*>(y), batch, wide_x, (int)n_tiles);
+                              map_x, l->map_w_wide, map_y, batch, wide_x, (int)n_tiles);
         }
         if (cfi_status_t e = set_smem<cfi_dense_tc_persistent_kernel<CFI_ACT_NONE>>(kTpSmemBytes, l->device)) return e;
         return launch_pdl(cfi_dense_tc_persistent_kernel<CFI_ACT_NONE>, dim3(ctas), kTpThreads, kTpSmemBytes, st, l->d, map_x,
-                          l->map_w_wide, static_cast<__nv_bfloat16*>(y), batch, wide_x, (int)n_tiles);
+                          l->map_w_wide, map_y, batch, wide_x, (int)n_tiles);
     }
     const int split = tc_bf16_split(l, batch);
     if (l->d.act == CFI_ACT_GELU_ERF) {
