@@ -161,6 +161,15 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    // The layer's weight belongs to no earlier kernel: the Wd boxes of the first ring round are requested before
+    // the wait for the kernel ahead (their slots' barriers already expect the x box as well), so a cold weight
+    // streams in while that kernel finishes.
+    if (warp == 0 && lane == 0) {
+        for (int i = 0; i < n_local && i < kTfStages; ++i) {
+            mbar_expect_tx(full0 + 8 * i, kTfABytes + kBBytes);
+            tma_load_2d(smem_u32(ring + i * kStageBytes) + kTfABytes, &map_w, full0 + 8 * i, (kb0 + i) * kTfK, n0);
+        }
+    }
     pdl_wait();  // x and y may belong to the kernel before this one
     if (tid >= 64 && tid < 64 + TN) bias_s[tid - 64] = bias_v;
     bool ok = true;
@@ -172,9 +181,9 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             if (i >= kTfStages) ok = mbar_wait(empty0 + 8 * s, (uint32_t)(i / kTfStages - 1) & 1u, kTcSpinLimit);
             if (!ok) break;
             const uint32_t a_dst = smem_u32(ring + s * kStageBytes), b_dst = a_dst + kTfABytes;
-            mbar_expect_tx(full0 + 8 * s, kTfABytes + kBBytes);
+            if (i >= kTfStages) mbar_expect_tx(full0 + 8 * s, kTfABytes + kBBytes);
             tma_load_2d(a_dst, &map_x, full0 + 8 * s, (kb0 + i) * kTfK, m0);
-            tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + i) * kTfK, n0);
+            if (i >= kTfStages) tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + i) * kTfK, n0);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
