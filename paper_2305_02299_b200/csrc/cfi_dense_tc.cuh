@@ -275,6 +275,14 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    // The weight belongs to no earlier kernel: its boxes of the first ring round are requested before the wait for
+    // the kernel ahead (each slot's barrier already expects the x box too).
+    if (warp == 0 && lane == 0) {
+        for (int kb = 0; kb < k_blocks && kb < kTcStages; ++kb) {
+            mbar_expect_tx(full0 + 8 * kb, kTcStageBytes);
+            tma_load_2d(smem_u32(ring + kb * kTcStageBytes) + kTcM * kTcK * 2, &map_w, full0 + 8 * kb, (kb0 + kb) * kTcK, n0);
+        }
+    }
     pdl_wait();  // x and y may belong to the kernel before this one
     bool ok = true;
 
@@ -285,9 +293,9 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
             if (kb >= kTcStages) ok = mbar_wait(empty0 + 8 * s, (uint32_t)(kb / kTcStages - 1) & 1u, kTcSpinLimit);
             if (!ok) break;
             const uint32_t a_dst = smem_u32(ring + s * kTcStageBytes), b_dst = a_dst + kTcM * kTcK * 2;
-            mbar_expect_tx(full0 + 8 * s, kTcStageBytes);
+            if (kb >= kTcStages) mbar_expect_tx(full0 + 8 * s, kTcStageBytes);
             tma_load_2d(a_dst, &map_x, full0 + 8 * s, (kb0 + kb) * kTcK, m0);
-            tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + kb) * kTcK, n0);
+            if (kb >= kTcStages) tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + kb) * kTcK, n0);
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
