@@ -42,7 +42,7 @@
 // them.  The barrier is the hardware cluster barrier (no flags, no global workspace), the order of additions is
 // fixed, and the layer stays read-only, so concurrent calls on one layer remain safe.
 
-constexpr int kTfM = 128, kTfK = 32, kTfStages = 4;  // the output tile is kTfM x TN with TN = 64 or 128 (template)
+constexpr int kTfM = 128, kTfK = 32, kTfStages = 4;  // the output tile is kTfM x TN with TN = 64, 96 or 128 (template)
 constexpr int kTfGroups = 4;  // groups of four worker warps; group g splits the K blocks kb with kb % kTfGroups == g
 constexpr int kTfWorkerWarps = 4 * kTfGroups, kTfThreads = 64 + 32 * kTfWorkerWarps;
 // A ring slot is always split by the same group, so that one phase bit per barrier is enough: a group that ran a
@@ -123,7 +123,10 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     pdl_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t base = ((smem_u32(0) + 1023u) & ~1023u) - smem_u32(0);
-    static_assert(TN == 64 || TN == 128, "tile width");
+    static_assert(TN == 64 || TN == 96 || TN == 128, "tile width");
+    // Partial tile in shared memory: 16-byte chunk c of row r sits at c ^ (r & kPermMask); the mask keeps the chunk
+    // inside its aligned group of 16 (or of 8 where a row has 24 chunks).
+    constexpr uint32_t kPermMask = TN % 64 == 0 ? 15u : 7u;
     constexpr uint32_t kBBytes = tf_b_bytes(TN), kStageBytes = tf_stage_bytes(TN), kAccCols = 2 * TN;
     static_assert(kAccCols + 64 * kTfStages <= kTfTmemCols, "tensor memory: accumulators + x slots");
     const uint32_t ring = base, ctl = base + kTfStages * kStageBytes;
@@ -266,8 +269,9 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
             // This CTA's partial tile (no bias yet) in shared memory: 128 rows of 4 TN bytes, 16-byte chunks permuted
             // by chunk ^ (row & 15).  The two accumulator halves are the two groups of products.
 #pragma unroll
-            for (int c16 = 0; c16 < TN / 64; ++c16) {
-                const int col0 = (TN / 4) * group + 16 * c16;
+            for (int ck = 0; ck < (TN / 16 + kTfGroups - 1) / kTfGroups; ++ck) {
+                const int col0 = 16 * (group + kTfGroups * ck);  // the groups take the 16-column pieces in turn
+                if (col0 >= TN) break;                           // (the same for a whole warp)
                 uint32_t v[16], v1[16];
                 const uint32_t t_acc = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)col0;
                 tmem_ld16(t_acc, v);
@@ -283,7 +287,7 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
                         r.z = __uint_as_float(v[4 * e4 + 2]) + __uint_as_float(v1[4 * e4 + 2]);
                         r.w = __uint_as_float(v[4 * e4 + 3]) + __uint_as_float(v1[4 * e4 + 3]);
                     }
-                    *reinterpret_cast<float4*>(smem_at(ring + row * (4 * TN) + (((col >> 2) ^ (row & 15)) << 4))) = r;
+                    *reinterpret_cast<float4*>(smem_at(ring + row * (4 * TN) + (((col >> 2) ^ (row & kPermMask)) << 4))) = r;
                 }
             }
         }
@@ -294,7 +298,8 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
     if (warp >= 2 && ok) {
         // Rows [split * rows_per, (split + 1) * rows_per) of the tile: sum over the cluster in rank order, bias,
         // activation, store.  TN / 4 threads per row, runs of 4 TN bytes.
-        constexpr int kPerRow = TN / 4, kRowsPerPass = 32 * kTfWorkerWarps / kPerRow;
+        // (24 threads per row do not divide the 512 workers: at TN = 96 the first 384 take 16 rows per pass.)
+        constexpr int kPerRow = TN / 4, kRowsPerPass = TN == 96 ? 16 : 32 * kTfWorkerWarps / kPerRow;
         const int wt = tid - 64, ch = wt % kPerRow, rows_per = (kTfM + n_split - 1) / n_split;
         const float4 bv = *reinterpret_cast<const float4*>(bias_s + 4 * ch);
         const int n = n0 + 4 * ch;
@@ -303,10 +308,10 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         auto fast = [&](auto s_tag, auto iter_tag) {
             constexpr int S = decltype(s_tag)::value, ITER = decltype(iter_tag)::value;
             const int rr0 = wt / kPerRow;
-            if (rr0 >= kTfM / S) return;
+            if (rr0 >= kTfM / S || rr0 >= kRowsPerPass) return;
             const int r0 = split * (kTfM / S) + rr0;
             float4 acc[ITER];
-            cluster_sum_rows<S, ITER>(smem_u32(ring + r0 * (4 * TN) + ((ch ^ (r0 & 15)) << 4)), kRowsPerPass * 4 * TN,
+            cluster_sum_rows<S, ITER>(smem_u32(ring + r0 * (4 * TN) + ((ch ^ (r0 & kPermMask)) << 4)), kRowsPerPass * 4 * TN,
                                       (uint32_t)split, acc);
 #pragma unroll
             for (int it = 0; it < ITER; ++it) {
@@ -326,11 +331,11 @@ cfi_dense_tf32_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, con
         if (n_split == 2) fast(integral_constant<int, 2>{}, integral_constant<int, kIter2>{});
         else if (n_split == 4) fast(integral_constant<int, 4>{}, integral_constant<int, (kIter4 > 0 ? kIter4 : 1)>{});
         else if (n_split == 8) fast(integral_constant<int, 8>{}, integral_constant<int, 1>{});
-        else
+        else if (wt < kRowsPerPass * kPerRow)
         for (int rr = wt / kPerRow; rr < rows_per; rr += kRowsPerPass) {
             const int r = split * rows_per + rr, m = m0 + r;
             if (r < kTfM && m < batch && n < L.out) {
-                const uint32_t off = ring + r * (4 * TN) + ((ch ^ (r & 15)) << 4);
+                const uint32_t off = ring + r * (4 * TN) + ((ch ^ (r & kPermMask)) << 4);
                 float4 a;
                 if (n_split == 1) {
                     a = *reinterpret_cast<const float4*>(smem_at(off));

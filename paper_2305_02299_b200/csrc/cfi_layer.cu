@@ -62,6 +62,7 @@ struct cfi_layer {
     bool tc_ok = false;
     CUtensorMap map_w{};       // dense copy in boxes of 128 rows (bf16) or 64 rows (fp32)
     CUtensorMap map_w_wide{};  // boxes of 128 rows (fp32) or 256 rows (bf16) for the wide tiles
+    CUtensorMap map_w_mid{};   // boxes of 96 rows (fp32 only)
 };
 
 struct cfi_stack {
@@ -861,6 +862,8 @@ bool encode_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols
 // again), larger for the wide tile; the cluster reduction when K is split; and the launch itself.
 constexpr double kDenseTf32SecondsPerBlock64 = 0.45e-6, kDenseTf32SecondsPerBlock128 = 0.61e-6, kDenseTf32Wave64 = 3.0e-6,
                  kDenseTf32Wave128 = 4.5e-6, kDenseTf32Reduce = 1.0e-6, kDenseTf32Launch = 0.7e-6;
+// 96-wide tiles: MMAs of N = 192 and N = 96, between the two by the same cost law.
+constexpr double kDenseTf32SecondsPerBlock96 = 0.53e-6, kDenseTf32Wave96 = 3.75e-6;
 constexpr int kTfMaxSplit = 8;
 
 template <int TN>
@@ -886,13 +889,15 @@ int tf32_query_clusters(const cfi_layer* l, int split) {
 // Clusters of `split` CTAs of the split-TF32 kernel that the device can hold at once; 0 if it cannot launch that
 // cluster size (cached per device; -1 in the cache stands for 0).
 int tf32_resident_clusters(const cfi_layer* l, int tile_n, int split) {
-    static std::atomic<int> cache[64][2][kTfMaxSplit + 1];
+    static std::atomic<int> cache[64][3][kTfMaxSplit + 1];
     if (split == 1) return std::max(1, l->sm_count);
     if (l->device < 0 || l->device >= 64) return 0;
-    std::atomic<int>& c = cache[l->device][tile_n == 128 ? 1 : 0][split];
+    std::atomic<int>& c = cache[l->device][tile_n == 128 ? 2 : tile_n == 96 ? 1 : 0][split];
     int v = c.load(std::memory_order_acquire);
     if (v == 0) {
-        v = tile_n == 128 ? tf32_query_clusters<128>(l, split) : tf32_query_clusters<64>(l, split);
+        v = tile_n == 128  ? tf32_query_clusters<128>(l, split)
+            : tile_n == 96 ? tf32_query_clusters<96>(l, split)
+                           : tf32_query_clusters<64>(l, split);
         if (v <= 0) v = -1;
         c.store(v, std::memory_order_release);
     }
@@ -900,7 +905,7 @@ int tf32_resident_clusters(const cfi_layer* l, int tile_n, int split) {
 }
 
 struct Tf32Shape {
-    int tile_n;      // outputs per tile: 64 or 128
+    int tile_n;      // outputs per tile: 64, 96 or 128
     int split;       // CTAs per output tile (cluster size along z): 1 .. 8
     double seconds;  // modelled time of the launch
 };
@@ -911,10 +916,12 @@ Tf32Shape tf32_shape(const cfi_layer* l, int batch) {
     const int k_blocks = (l->d.in + kTfK - 1) / kTfK;
     Tf32Shape best{64, 1, 0.0};
     bool have = false;
-    for (int tile_n = 64; tile_n <= 128; tile_n *= 2) {
+    for (int tile_n = 64; tile_n <= 128; tile_n += 32) {
         const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + tile_n - 1) / tile_n);
-        const double per_block = tile_n == 128 ? kDenseTf32SecondsPerBlock128 : kDenseTf32SecondsPerBlock64;
-        const double per_wave = tile_n == 128 ? kDenseTf32Wave128 : kDenseTf32Wave64;
+        const double per_block = tile_n == 128  ? kDenseTf32SecondsPerBlock128
+                                 : tile_n == 96 ? kDenseTf32SecondsPerBlock96
+                                                : kDenseTf32SecondsPerBlock64;
+        const double per_wave = tile_n == 128 ? kDenseTf32Wave128 : tile_n == 96 ? kDenseTf32Wave96 : kDenseTf32Wave64;
         for (int split = 1; split <= kTfMaxSplit; ++split) {
             if (split > 1 && (k_blocks < 4 * split || tiles * split > 2 * (int64_t)l->sm_count)) break;
             const int64_t resident = tf32_resident_clusters(l, tile_n, split);
@@ -943,6 +950,7 @@ cfi_status_t launch_dense_tf32(const cfi_layer* l, const void* x, void* y, int b
     if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 4, kTfM)) return CFI_ERR_SHAPE;
     const Tf32Shape sh = tf32_shape(l, batch);
     if (sh.tile_n == 128) return launch_dense_tf32_n<128>(l, map_x, l->map_w_wide, sh.split, y, batch, st);
+    if (sh.tile_n == 96) return launch_dense_tf32_n<96>(l, map_x, l->map_w_mid, sh.split, y, batch, st);
     return launch_dense_tf32_n<64>(l, map_x, l->map_w, sh.split, y, batch, st);
 }
 
@@ -1349,6 +1357,8 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                 if (l->tc_ok)  // the same copy in the boxes of the wide tiles: 128 rows (fp32), 256 rows (bf16)
                     l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb,
                                           dtype == CFI_BF16 ? kTpN : 128);
+                if (l->tc_ok && dtype != CFI_BF16)
+                    l->tc_ok = encode_map(&l->map_w_mid, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb, 96);
             }
         }
 
