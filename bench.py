@@ -385,7 +385,7 @@ def main():
                          # dram__bytes_read.sum + dram__bytes_write.sum of one launch (ncu capture summarised under
                          # profiles/); only valid for the kernel and workload it was taken on
                          "traffic": 10.29e6 if (tile_shape is not None and w.name == "c2"
-                                                and tile_shape["tile"][1] == 128 and tile_shape["cluster_k_split"] == 2) else None,
+                                                and tile_shape["tile"][1] == 96 and tile_shape["cluster_k_split"] == 2) else None,
                          "peak_source": f"{sm_count} SMs x {FMA_LANES_PER_SM} fp32 FMA lanes x 2 x {sm_max_mhz:.0f} MHz",
                          "kernel": {"batch": "cfi_batch_kernel<float>",
                                     "dense_tc": f"cfi_dense_tf32_kernel<{tile_shape['tile'][1] if tile_shape else 64}>"}.get(
