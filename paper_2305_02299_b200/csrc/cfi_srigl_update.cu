@@ -30,6 +30,7 @@ struct SelectState {
     unsigned long long below;    // elements with a key below the current prefix
     unsigned int prefix, prefix_mask;
     unsigned int hist[256];
+    unsigned int blocks_done;    // blocks of the running histogram sweep that have added their counts (first state only)
 };
 
 struct Scalars {
@@ -89,10 +90,54 @@ __global__ void setup_kernel(const int* row_count, int out_f, int in_f, long lon
         long long kk = K < 0 ? 0 : K;
         if (kk > act) kk = act;
         if (kk > sc->inactive_total) kk = sc->inactive_total;
-        for (int s = 0; s < 2; ++s) st[s].want = (unsigned long long)kk, st[s].below = 0, st[s].prefix = 0, st[s].prefix_mask = 0;
+        for (int s = 0; s < 2; ++s)
+            st[s].want = (unsigned long long)kk, st[s].below = 0, st[s].prefix = 0, st[s].prefix_mask = 0, st[s].blocks_done = 0;
     }
     for (int s = 0; s < 2; ++s)
         for (int b = threadIdx.x; b < 256; b += blockDim.x) st[s].hist[b] = 0;
+}
+
+// One warp per selection: the bin that holds the `want`-th element (the first bin whose running count reaches it;
+// the last bin if none before it does); narrow the prefix to it and clear the histogram for the next pass.  Called by
+// the last block of a histogram sweep, after every block's counts have arrived.
+__device__ void pick_bin(int pass, SelectState* st) {
+    const int lane = threadIdx.x & 31;
+    const unsigned long long want = st->want;
+    unsigned int v[8];
+    unsigned long long mine = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = __ldcg(&st->hist[8 * lane + e]), mine += v[e];
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    unsigned long long seen = incl - mine;  // count in the bins before this lane's
+    int found = 256;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        if (found == 256) {
+            if (seen + v[e] >= want) found = 8 * lane + e;
+            else seen += v[e];
+        }
+    }
+    int bin = found;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) bin = min(bin, __shfl_xor_sync(0xffffffffu, bin, off));
+    if (bin > 255) bin = 255;
+    // `seen` of the lane that owns the bin is the count below it (for the last bin without a hit: lane 31 stopped there)
+    if (found == 256 && lane == 31) seen -= v[7];
+    const unsigned long long below_bin = __shfl_sync(0xffffffffu, seen, bin >> 3);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) st->hist[8 * lane + e] = 0;
+    if (lane == 0 && want != 0) {
+        const int shift = 24 - 8 * pass;
+        st->want = want - below_bin;
+        st->below += below_bin;
+        st->prefix |= (unsigned int)bin << shift;
+        st->prefix_mask |= 255u << shift;
+    }
 }
 
 // Histograms of digit `pass` (0 = top byte) for both layer-wide selections in one sweep over the layer: over the valid
@@ -154,26 +199,17 @@ __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* gr
     __syncthreads();
     for (int b = threadIdx.x; b < 512; b += blockDim.x)
         if (h[b]) atomicAdd(&st[b >> 8].hist[b & 255], h[b]);
-}
-
-// One thread: the bin that holds the `want`-th element; narrow the prefix to it and clear the histogram.
-__global__ void pick_kernel(int pass, SelectState* both) {
-    if (threadIdx.x > 1 || blockIdx.x != 0) return;
-    SelectState* st = both + threadIdx.x;  // one thread per selection
-    if (st->want != 0) {
-        unsigned long long seen = 0;
-        int b = 0;
-        for (; b < 255; ++b) {
-            if (seen + st->hist[b] >= st->want) break;
-            seen += st->hist[b];
-        }
-        const int shift = 24 - 8 * pass;
-        st->want -= seen;
-        st->below += seen;
-        st->prefix |= (unsigned int)b << shift;
-        st->prefix_mask |= 255u << shift;
+    // The block whose counts arrive last narrows both selections to their bins (no separate launch, nobody waits).
+    __shared__ bool last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&st[0].blocks_done, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (last) {
+        __threadfence();
+        if (threadIdx.x < 64) pick_bin(pass, st + (threadIdx.x >> 5));
+        if (threadIdx.x == 0) st[0].blocks_done = 0;
     }
-    for (int b = 0; b < 256; ++b) st->hist[b] = 0;
 }
 
 // After the four passes prefix is the key of the cut and `want` of the elements equal to it are taken, the first ones
@@ -501,7 +537,6 @@ bool layer_select_both(const float* w, const uint8_t* mask, const float* grad, c
     const int hist_blocks = out_f < 1184 ? out_f : 1184;  // whole rows per block, 8 CTAs per SM at most
     for (int pass = 0; pass < 4; ++pass) {
         hist_kernel<<<hist_blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, out_f, in_f, pass, ws.state);
-        pick_kernel<<<1, 32, 0, st>>>(pass, ws.state);
     }
     tie_count_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks);
     chunk_scan_kernel<<<2, kThreads, 0, st>>>(ws.chunk_ties, chunks);
