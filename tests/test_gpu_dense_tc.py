@@ -58,11 +58,13 @@ def test_dense_tf32_launch_shapes_cover_wide_tiles_and_clusters():
 
 
 @pytest.mark.parametrize("in_f,out_f,k,nabl,B,act", [(768, 1000, 77, 50, 9601, "gelu"), (1024, 512, 102, 0, 19001, "none"),
-                                                     (200, 2048, 20, 100, 4801, "gelu"), (768, 3072, 77, 154, 7000, "gelu")])
+                                                     (200, 2048, 20, 100, 4801, "gelu"), (768, 3072, 77, 154, 7000, "gelu"),
+                                                     (256, 2120, 26, 60, 2200, "gelu")])
 def test_dense_tc_bf16_many_tiles_per_sm(in_f, out_f, k, nabl, B, act):
     """Enough 128 x 256 tiles for the persistent bf16 kernel (at least two per SM): ragged last batch tile and last
-    output tile (also one that ends in the first half of a tile), ablated rows, more tiles than CTAs so that both
-    accumulator buffers and the bias buffer are reused."""
+    output tile (also one that ends in the first half of a tile, and one whose last 64-column store boxes lie partly
+    and wholly past the outputs), ablated rows, more tiles than CTAs so that both accumulator buffers and both store
+    boxes are reused.  run_device keeps guard bands around y, so a store that is not clipped at the end of y fails."""
     from paper_2305_02299_b200 import binding as cfi
     L = inputs.make_layer(in_f, out_f, k, n_ablated=nabl, seed=B)
     x = inputs.make_x(B, in_f, seed=B + 1)
