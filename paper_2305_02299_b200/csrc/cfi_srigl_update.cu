@@ -370,6 +370,36 @@ struct RowCut {
     int any;             // 0: nothing to select
 };
 
+// One warp: the first of 256 shared-memory bins whose running count reaches `want` (the last bin if none before it
+// does) and the count in the bins before it; eight bins per lane, one scan over the lanes.
+__device__ __forceinline__ void row_pick(const unsigned int* hist, unsigned int want, int& bin, unsigned int& below) {
+    const int lane = threadIdx.x & 31;
+    unsigned int v[8], mine = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = hist[8 * lane + e], mine += v[e];
+    unsigned int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int up = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    unsigned int seen = incl - mine;
+    int found = 256;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        if (found == 256) {
+            if (seen + v[e] >= want) found = 8 * lane + e;
+            else seen += v[e];
+        }
+    }
+    bin = found;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) bin = min(bin, __shfl_xor_sync(0xffffffffu, bin, off));
+    if (bin > 255) bin = 255;
+    if (found == 256 && lane == 31) seen -= v[7];  // no bin before the last reaches `want`: the count below the last bin
+    below = __shfl_sync(0xffffffffu, seen, bin >> 3);
+}
+
 template <typename KeyOf>
 __device__ void row_select(int in_f, int m, KeyOf key_of, unsigned int* hist /*256, shared*/, RowCut* out /*shared*/) {
     __shared__ unsigned int prefix, pmask, want;
@@ -379,21 +409,21 @@ __device__ void row_select(int in_f, int m, KeyOf key_of, unsigned int* hist /*2
         for (int b = threadIdx.x; b < 256; b += blockDim.x) hist[b] = 0;
         __syncthreads();
         const int shift = 24 - 8 * pass;
+        const unsigned int pre = prefix, pm = pmask;
         for (int c = threadIdx.x; c < in_f; c += blockDim.x) {
             unsigned int key;
-            if (key_of(c, key) && (key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+            if (key_of(c, key) && (key & pm) == pre) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned int seen = 0;
-            int b = 0;
-            for (; b < 255; ++b) {
-                if (seen + hist[b] >= want) break;
-                seen += hist[b];
+        if (threadIdx.x < 32) {
+            int b;
+            unsigned int seen;
+            row_pick(hist, want, b, seen);
+            if (threadIdx.x == 0) {
+                want -= seen;
+                prefix |= (unsigned int)b << shift;
+                pmask |= 255u << shift;
             }
-            want -= seen;
-            prefix |= (unsigned int)b << shift;
-            pmask |= 255u << shift;
         }
         __syncthreads();
     }
@@ -413,8 +443,7 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
     __shared__ unsigned int hist[256];
     __shared__ RowCut cut;
     __shared__ int kept_count;
-    __shared__ unsigned int part[kThreads];
-    __shared__ unsigned int carry;
+    __shared__ unsigned int part[kThreads / 32];
     const int r = blockIdx.x;
     float* wr = w + (size_t)r * in_f;
     uint8_t* mr = mask + (size_t)r * in_f;
@@ -459,9 +488,10 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
     // trim: the kept weights with the smallest magnitudes go; otherwise the free positions with the largest gradient
     // magnitudes come
     row_select(in_f, m, key_of, hist, &cut);
-    // Apply, walking the row in column order so that ties on the cut key go to the smaller columns.
-    if (threadIdx.x == 0) carry = 0;
-    __syncthreads();
+    // Apply, walking the row in column order so that ties on the cut key go to the smaller columns: a tie's rank is
+    // the ties of the chunks before (carried by every thread), of the warps before in this chunk (one count per warp
+    // in shared memory) and of the lanes before in its warp (a ballot).
+    unsigned int carry = 0;
     for (int c0 = 0; c0 < in_f; c0 += kThreads) {
         const int c = c0 + threadIdx.x;
         bool is_kept = false, candidate = false;
@@ -472,15 +502,17 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
             if (cut.any && candidate) key = CACHED ? keys[c] : (trim ? mag_bits(wr[c]) : ~mag_bits(gr[c]));
         }
         const unsigned int tie = (cut.any && candidate && key == cut.cut) ? 1u : 0u;
-        part[threadIdx.x] = tie;
+        const unsigned int ties_in_warp = __ballot_sync(0xffffffffu, tie != 0);
+        const int wid = threadIdx.x >> 5, ln = threadIdx.x & 31;
+        if (ln == 0) part[wid] = (unsigned int)__popc(ties_in_warp);
         __syncthreads();
-        for (int off = 1; off < kThreads; off <<= 1) {
-            const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
-            __syncthreads();
-            part[threadIdx.x] += add;
-            __syncthreads();
+        unsigned int rank = carry + (unsigned int)__popc(ties_in_warp & ((1u << ln) - 1u)), in_chunk = 0;
+#pragma unroll
+        for (int i = 0; i < kThreads / 32; ++i) {
+            const unsigned int p = part[i];
+            rank += i < wid ? p : 0u;
+            in_chunk += p;
         }
-        const unsigned int rank = carry + part[threadIdx.x] - tie;
         if (c < in_f) {
             const bool selected = cut.any && candidate && (key < cut.cut || (tie && rank < cut.ties));
             bool on;
@@ -489,9 +521,8 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
             if (!on || !is_kept) wr[c] = 0.0f;  // pruned, trimmed, free, or grown (starts at 0); a survivor keeps its value
             mr[c] = on ? 1 : 0;
         }
-        __syncthreads();
-        if (threadIdx.x == kThreads - 1) carry += part[kThreads - 1];
-        __syncthreads();
+        carry += in_chunk;
+        __syncthreads();  // part[] is rewritten by the next chunk
     }
 }
 
