@@ -161,7 +161,10 @@ __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* gr
                 take = m ? (on0 && (key & pmask0) == prefix0) : (on1 && (key & pmask1) == prefix1);
                 bin = (m ? 0u : 256u) + ((key >> shift) & 255u);
             }
-            hist_add(h, take, bin);
+            // The top digit falls into a handful of bins (aggregate per warp); the later digits of the few elements that
+            // still match the prefix spread out, and a plain atomic is cheaper there.
+            if (pass == 0) hist_add(h, take, bin);
+            else if (take) atomicAdd(&h[bin], 1u);
         };
         for (int r = blockIdx.x; r < out_f; r += gridDim.x) {
             if (row_count[r] == 0) continue;  // a neuron without weights is in neither pool
