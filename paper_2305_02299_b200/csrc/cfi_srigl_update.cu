@@ -56,8 +56,17 @@ __global__ void row_count_kernel(const uint8_t* mask, int out_f, int in_f, int* 
     if (threadIdx.x == 0) s = 0;
     __syncthreads();
     int c = 0;
-    for (int j = threadIdx.x; j < in_f; j += blockDim.x) c += mask[(size_t)r * in_f + j] ? 1 : 0;
-    atomicAdd(&s, c);
+    if ((in_f & 15) == 0) {  // 16 mask bytes per load; __vcmpne4 turns every nonzero byte into 0xff
+        const uint4* m16 = reinterpret_cast<const uint4*>(mask + (size_t)r * in_f);
+        for (int v = threadIdx.x; v < (in_f >> 4); v += blockDim.x) {
+            const uint4 m = m16[v];
+            c += (__popc(__vcmpne4(m.x, 0u)) + __popc(__vcmpne4(m.y, 0u)) + __popc(__vcmpne4(m.z, 0u)) + __popc(__vcmpne4(m.w, 0u))) >> 3;
+        }
+    } else {
+        for (int j = threadIdx.x; j < in_f; j += blockDim.x) c += mask[(size_t)r * in_f + j] ? 1 : 0;
+    }
+    for (int off = 16; off > 0; off >>= 1) c += __shfl_down_sync(0xffffffffu, c, off);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s, c);
     __syncthreads();
     if (threadIdx.x == 0) row_count[r] = s;
 }
