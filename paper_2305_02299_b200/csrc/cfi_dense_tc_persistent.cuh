@@ -139,7 +139,7 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
             if (ok) ok = mbar_wait(acc_full0 + 8 * b, (i >> 1) & 1u, kTcSpinLimit);
             ok = __all_sync(0xffffffffu, ok);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll 1
+#pragma unroll
             for (int qs = 0; qs < 4; ++qs, ++step) {
                 // Staging buffer step mod 2: one TMA box of 128 rows x 64 bf16 columns in the 128-byte swizzle.  Its
                 // last store (two steps ago) was waited for by thread 0 before the barrier of the step in between.
