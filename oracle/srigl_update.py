@@ -4,7 +4,7 @@ TEST INFRASTRUCTURE ONLY, like the rest of this package: plain numpy, whole-arra
 code shared with the CUDA library.  Steps are taken in the paper's order and notation (K = weights pruned and grown
 in this step, k = fan-in before, k' = fan-in after, gamma_sal = ablation threshold).
 
-Where the paper leaves a choice open, the reading is the one listed in DESIGN.md (section 2, "SRigL update"):
+Where the paper leaves a choice open, the reading taken is:
   * ties in magnitude are broken by position: among equal magnitudes the entry with the smaller flat index
     (row * in + column) counts as the smaller weight when pruning and as the larger gradient when growing;
   * "salient" (step 3): an active weight that is NOT among the K smallest magnitudes of the layer, or an inactive

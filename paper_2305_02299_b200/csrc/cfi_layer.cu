@@ -44,6 +44,7 @@ struct DevLayer {
     int32_t* status;
     int in, out, n_active, k, kp, act;
     int cs, n_slabs, stride_q, maxq;  // slab width, slabs, quads per row, most quads of a row in one slab
+    int identity_rows;                // 1 if output row o is condensed row o for every o (no ablated row, rows in order)
 };
 
 }  // namespace
@@ -210,7 +211,7 @@ __global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* _
     const int nb = min(BT, batch - b0);
     const int groups = nthr / G, g = tid / G, lg = tid % G;
     const int nvec = L.kp / CK::VEC;
-    const bool dense_rows = L.n_active == L.out;  // no ablated row: output row o is condensed row o
+    const bool dense_rows = L.identity_rows != 0;  // output row o is condensed row o: no look-up through slot[]
     int o = blockIdx.x * (groups * rows_per_group) + g;
     int r = o < L.out ? (dense_rows ? o : L.slot[o]) : -1;
 
@@ -1047,6 +1048,15 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
 // Rate of the gather kernel's arithmetic, used to choose between it and the split-TF32 dense kernel (measured).
 constexpr double kGatherTflops = 12.5;
 
+// The split-k kernel keeps at least one whole row of x (+ one zero element) in shared memory.
+bool splitk_fits(const cfi_layer* l, int batch) { return splitk_shape(l, batch).smem <= (size_t)l->smem_optin; }
+
+// What remains when the preferred kernel cannot hold its tile: the gather kernel (column slabs), else one thread per output.
+int fallback_variant(const cfi_layer* l, int batch) {
+    if (batch_shape(l, batch).ok) return CFI_VARIANT_BATCH;
+    return splitk_fits(l, batch) ? CFI_VARIANT_SPLITK : CFI_VARIANT_SIMPLE;
+}
+
 int choose_variant(const cfi_layer* l, int batch) {
     // Up to three batch tiles of 8 the split-k kernel (weights re-read from L2 per tile) beats the 64-wide tiles of
     // the batch kernel, which would be mostly empty.
@@ -1063,7 +1073,7 @@ int choose_variant(const cfi_layer* l, int batch) {
             else tc_bf16_split(l, batch, &t_dense);
             if (t_dense < t_splitk) return CFI_VARIANT_DENSE_TC;
         }
-        return CFI_VARIANT_SPLITK;
+        return splitk_fits(l, batch) ? CFI_VARIANT_SPLITK : fallback_variant(l, batch);
     }
     // bf16 above 24 rows: the dense contraction on the tensor cores beats the gather kernel even at 99 % sparsity
     // (10 TFLOP/s effective for the gather against several hundred dense), also with a partly empty 128-row tile
@@ -1083,7 +1093,7 @@ int choose_variant(const cfi_layer* l, int batch) {
         const double t_gather = t_fma + t_stage - 0.5 * std::min(t_fma, t_stage) + 5e-6;
         if (t_dense < t_gather) return CFI_VARIANT_DENSE_TC;
     }
-    return batch_shape(l, batch).ok ? CFI_VARIANT_BATCH : CFI_VARIANT_SPLITK;
+    return fallback_variant(l, batch);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1201,6 +1211,8 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
         if (o < 0 || o >= out_features || slot[o] != -1) return CFI_ERR_INDEX_RANGE;
         slot[o] = r;
     }
+    bool identity_rows = n_active == out_features;
+    for (int32_t r = 0; identity_rows && r < n_active; ++r) identity_rows = active_rows[r] == r;
 
     cfi_layer* l = new (std::nothrow) cfi_layer();
     if (!l) return CFI_ERR_ALLOC;
@@ -1215,6 +1227,7 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
     l->dtype = dtype;
     DevLayer& d = l->d;
     d.in = in_features, d.out = out_features, d.n_active = n_active, d.k = k, d.act = act;
+    d.identity_rows = identity_rows ? 1 : 0;
 
     try {
         // Each row sorted by column (stable, so repeated columns keep the caller's order).
@@ -1416,6 +1429,7 @@ extern "C" cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void
     if (batch == 0 || layer->d.out == 0) return CFI_OK;
     if (!y || (!x && layer->d.in > 0)) return CFI_ERR_NULL;
     if (((uintptr_t)x | (uintptr_t)y) & 15u) return CFI_ERR_ALIGNMENT;
+    DeviceGuard g(layer->device);  // kernels, tensor maps and shared-memory opt-ins belong to the layer's device
     int v = variant;
     if (v == CFI_VARIANT_AUTO) v = choose_variant(layer, batch);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);

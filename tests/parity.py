@@ -56,6 +56,20 @@ def scaled_error(y, y_ref, S):
     return float(np.max(np.abs(y - y_ref) / np.maximum(S, 1e-300)))
 
 
+def assert_parity(y, y_ref, S, dtype, what=""):
+    """The stated bound (error against the scale of the sum) and, for bf16 storage, the bound the arithmetic itself
+    allows: exact products of the rounded inputs, fp32 accumulation (a few 2^-24 of S for these fan-ins, 1e-5 of S
+    with room for the activation) and ONE rounding to nearest at the store (2^-9 of |y|, allowed 2^-8).  The second
+    bound is what catches inputs rounded the wrong way, which the first, at 2e-2 of S, would let through."""
+    err = scaled_error(y, y_ref, S)
+    assert err <= TOL[dtype], f"{what}: scaled error {err:.3e}"
+    if dtype == "bf16" and y.size:
+        excess = np.abs(y - y_ref) - (2.0 ** -8 * np.abs(y_ref) + 1e-5 * S)
+        i = np.unravel_index(np.argmax(excess), excess.shape)
+        assert excess[i] <= 0.0, f"{what}: bf16 result off by more than its store rounding at {i}: {y[i]} vs {y_ref[i]} (S {S[i]})"
+    return err
+
+
 def check_layer(layer, x_np, dtype="f32", act="none", variants=("auto",), tol=None):
     y_ref, S = oracle_layer(layer, x_np, dtype, act)
     dl = device_layer(layer, dtype, act)
@@ -64,7 +78,7 @@ def check_layer(layer, x_np, dtype="f32", act="none", variants=("auto",), tol=No
         for v in variants:
             y = run_device(dl, x_np, dtype, v)
             assert np.all(np.isfinite(y)), f"variant {v}: non-finite output"
-            errs[v] = scaled_error(y, y_ref, S)
+            errs[v] = assert_parity(y, y_ref, S, dtype, f"variant {v}")
             assert errs[v] <= (TOL[dtype] if tol is None else tol), f"variant {v}: scaled error {errs[v]:.3e}"
     finally:
         dl.close()

@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 
 from paper_2305_02299_b200 import inputs
-from parity import TOL, device_layer, oracle_layer, run_device, scaled_error
+from parity import TOL, assert_parity, device_layer, oracle_layer, run_device, scaled_error
 
 pytestmark = pytest.mark.gpu
 
@@ -28,7 +28,7 @@ def test_dense_tc_matches_oracle(in_f, out_f, k, nabl, B, act, dtype):
     y = run_device(dl, x, dtype, "dense_tc")
     dl.close()
     assert np.all(np.isfinite(y))
-    assert scaled_error(y, y_ref, S) <= TOL[dtype]
+    assert_parity(y, y_ref, S, dtype)
 
 
 # (in, out, k, ablated, batch) chosen so that together they run all three tile widths and clusters of several sizes.
@@ -76,7 +76,7 @@ def test_dense_tc_bf16_many_tiles_per_sm(in_f, out_f, k, nabl, B, act):
     y2 = run_device(dl, x, "bf16", "dense_tc")
     dl.close()
     assert np.all(np.isfinite(y))
-    assert scaled_error(y, y_ref, S) <= TOL["bf16"]
+    assert_parity(y, y_ref, S, "bf16")
     assert np.array_equal(y, y2)
 
 
@@ -95,7 +95,7 @@ def test_dense_tc_bf16_cluster_split_is_exercised():
         seen.add(shape)
         y = run_device(dl, x, "bf16", "dense_tc")
         dl.close()
-        assert scaled_error(y, y_ref, S) <= TOL["bf16"], (in_f, out_f, B, shape)
+        assert_parity(y, y_ref, S, "bf16", str((in_f, out_f, B, shape)))
     clusters = {c for t, c in seen if t == 128}
     assert 1 in clusters and len([c for c in clusters if c > 1]) >= 2, seen
 

@@ -9,7 +9,7 @@ import pytest
 
 import oracle
 from paper_2305_02299_b200 import inputs
-from parity import TOL, check_layer, device_layer, oracle_layer, run_device, scaled_error, to_device, torch_dtype
+from parity import TOL, assert_parity, check_layer, device_layer, oracle_layer, run_device, scaled_error, to_device, torch_dtype
 
 pytestmark = pytest.mark.gpu
 ALL = ("simple", "splitk", "batch", "auto")
@@ -48,7 +48,7 @@ def test_gelu_and_ablated_rows(dtype, act):
     dl = device_layer(L, dtype, act)
     for v in ALL:
         y = run_device(dl, x, dtype, v)
-        assert scaled_error(y, y_ref, S) <= TOL[dtype]
+        assert_parity(y, y_ref, S, dtype)
         # Ablated rows carry act(bias) only, identical for every batch row and rounded once to the storage type.
         expect = torch.tensor(y_ref[0, L.ablated]).to(torch_dtype(dtype)).to(torch.float64).numpy()
         got = y[:, L.ablated]
@@ -181,7 +181,7 @@ def test_stack_matches_chained_oracle(dtype):
     cur = oracle.round_bf16(x) if dtype == "bf16" else x
     for i, dl in enumerate(dls):                        # teacher-forced: layer i gets the oracle's input
         y = run_device(dl, cur, dtype)
-        assert scaled_error(y, exact[i], scales[i]) <= TOL[dtype], i
+        assert_parity(y, exact[i], scales[i], dtype, str(i))
         cur = outs[i].astype(np.float32)
     st = cfi.cfi_stack_create(dls, 70)
     y_d = torch.empty((70, 96), device="cuda", dtype=torch_dtype(dtype))
@@ -206,3 +206,81 @@ def test_splitk_long_rows_full_batch_tile(dtype, B):
     L = inputs.make_layer(4096, 1024, 205, n_ablated=30, seed=B)
     x = inputs.make_x(B, 4096, seed=B + 3)
     check_layer(L, x, dtype, "gelu", variants=("splitk",))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("order", ["reversed", "shuffled"])
+def test_every_row_active_in_any_row_order(dtype, order):
+    """n_active == out_features with active_rows that is not 0, 1, 2, ...: condensed row r belongs to output row
+    active_rows[r] in every kernel, the small-batch one included."""
+    from paper_2305_02299_b200 import binding as cfi
+    out_f, in_f, k = 64, 128, 9
+    L = inputs.make_layer(in_f, out_f, k, seed=21)
+    v, ix, rows = oracle.pack(L.w_dense, L.mask)
+    assert rows.shape[0] == out_f
+    perm = np.arange(out_f)[::-1].copy() if order == "reversed" else np.random.default_rng(5).permutation(out_f)
+    v2, ix2, rows2 = v[perm], ix[perm], rows[perm].astype(np.int32)
+    dl = cfi.cfi_create(v2, ix2, rows2, L.bias, in_f, out_f, dtype=dtype)
+    for B in (1, 2, 5, 8, 40, 130):
+        x = inputs.make_x(B, in_f, seed=B)
+        y_ref, S = oracle_layer(L, x, dtype)
+        y_perm, _ = oracle_layer(L, x, dtype, packed=(v2, ix2, rows2))
+        assert np.array_equal(y_ref, y_perm)                 # the oracle itself does not care about the row order
+        for var in ALL + ("dense_tc",):
+            assert_parity(run_device(dl, x, dtype, var), y_ref, S, dtype, f"{var} B={B}")
+    dl.close()
+
+
+@pytest.mark.parametrize("variant", ["simple", "splitk", "batch", "dense_tc", "auto"])
+def test_bf16_inputs_are_rounded_to_nearest_even(variant):
+    """Weights and activations that lie exactly half-way between two bf16 numbers.  With one-hot partners every
+    output is a single product of the rounded numbers, exact in bf16, so the device must return the oracle's
+    numbers bit for bit; truncation or round-half-up of either operand gives different bits."""
+    from paper_2305_02299_b200 import binding as cfi
+    n = 16
+    ties = np.array([1 + 1 * 2.0 ** -8, 1 + 3 * 2.0 ** -8, -(1 + 5 * 2.0 ** -8), 2 + 7 * 2.0 ** -7, 0.5 + 9 * 2.0 ** -9,
+                     -(1 + 2.0 ** -8 + 2.0 ** -20), 1 + 2.0 ** -8 - 2.0 ** -20, 3.0], dtype=np.float32)
+    r = oracle.round_bf16(ties)
+    assert r[0] == 1.0 and r[1] == 1 + 2.0 ** -6 and r[2] == -(1 + 2.0 ** -6)     # to even, not down and not up
+    assert r[5] == -(1 + 2.0 ** -7) and r[6] == 1.0                               # just past / short of half-way
+    # (a) tie-valued weights against one-hot activations.
+    vals = np.stack([np.roll(ties, i)[:2] for i in range(n)]).astype(np.float32)           # [16, 2]
+    idx = np.stack([[i, (i + 5) % n] for i in range(n)]).astype(np.int32)
+    rows = np.arange(n, dtype=np.int32)
+    x = np.eye(n, dtype=np.float32)
+    dl = cfi.cfi_create(vals, idx, rows, None, n, n, dtype="bf16")
+    y_ref = oracle.forward(oracle.round_bf16(vals), idx, rows, None, n, n, x)
+    assert np.array_equal(run_device(dl, x, "bf16", variant), y_ref)
+    dl.close()
+    # (b) tie-valued activations against weights of one.
+    ones = np.ones((n, 1), np.float32)
+    idx1 = np.arange(n, dtype=np.int32).reshape(n, 1)
+    dl = cfi.cfi_create(ones, idx1, rows, None, n, n, dtype="bf16")
+    xt = np.stack([np.roll(np.resize(ties, n), b) for b in range(24)]).astype(np.float32)
+    y_ref = oracle.forward(ones, idx1, rows, None, n, n, oracle.round_bf16(xt))
+    import torch
+    x_d = torch.from_numpy(xt).to("cuda", torch.bfloat16)          # torch rounds to nearest even as well
+    assert np.array_equal(x_d.float().cpu().numpy(), oracle.round_bf16(xt))
+    assert np.array_equal(run_device(dl, xt, "bf16", variant), y_ref)
+    dl.close()
+
+
+def test_wide_layer_small_batch_falls_back_to_a_kernel_that_fits():
+    """in_features so large that one row of x does not fit shared memory: the automatic choice must not pick the
+    small-batch kernel (which would refuse the shape) but one that can run it."""
+    from paper_2305_02299_b200 import binding as cfi
+    in_f, out_f, k = 70000, 24, 6
+    rng = np.random.default_rng(3)
+    idx = np.stack([np.sort(rng.choice(in_f, size=k, replace=False)) for _ in range(out_f)]).astype(np.int32)
+    vals = rng.standard_normal((out_f, k)).astype(np.float32)
+    rows = np.arange(out_f, dtype=np.int32)
+    bias = rng.standard_normal(out_f).astype(np.float32)
+    dl = cfi.cfi_create(vals, idx, rows, bias, in_f, out_f)
+    for B in (1, 3, 12):
+        assert cfi.cfi_choose_variant(dl, B) != 2
+        x = inputs.make_x(B, in_f, seed=B)
+        y_ref, S = oracle.forward(vals, idx, rows, bias, in_f, out_f, x, want_scale=True)
+        assert scaled_error(run_device(dl, x, "f32", "auto"), y_ref, S) <= 1e-5
+    with pytest.raises(cfi.CfiError):
+        run_device(dl, inputs.make_x(1, in_f), "f32", "splitk")
+    dl.close()

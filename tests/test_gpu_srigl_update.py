@@ -45,6 +45,13 @@ def test_matches_oracle(out_f, in_f, k, n_abl, K, gamma):
     _compare(w, m, g, K, gamma)
 
 
+def test_matches_oracle_at_the_benchmarked_size():
+    """4096 x 4096 at 80 % sparsity with K = 30 % of the active weights (about 1.0 M): the size and K the benchmark's
+    mask-update leg times."""
+    w, m, g = _layer(4096, 4096, 819, 0, seed=11)
+    _compare(w, m, g, int(0.3 * 4096 * 819), 0.3)
+
+
 def test_ablation_case_and_chained_updates():
     """A neuron with tiny weights and gradients is ablated and k' rises; a second update on the result still matches."""
     w, m, g = _layer(64, 256, 16, 0, seed=9)

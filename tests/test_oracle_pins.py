@@ -265,6 +265,60 @@ def test_stack_is_chain_of_layers():
         cur = cur.astype(np.float32).astype(np.float64)
 
 
+def _bf16_torch(a):
+    """fp32 -> bf16 -> fp32 through torch's conversion (round to nearest even), independent of the oracle's own."""
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16).to(torch.float32).numpy()
+
+
+def _is_bf16(a):
+    return bool(np.all((np.ascontiguousarray(a, dtype=np.float32).view(np.uint32) & 0xFFFF) == 0))
+
+
+def test_stack_bf16_rounds_where_a_bf16_layer_stores():
+    """bf16 chain: values and x are rounded when stored, every layer's output once at its store, the bias stays
+    fp32, sums are exact products in double.  The chain is written out here with torch's bf16 conversion and numpy
+    float64 dense products; a chain with any of the roundings left out must differ from it visibly."""
+    import torch
+    specs = [(16, 24, 5, 2, "gelu"), (24, 16, 7, 1, "none"), (16, 24, 5, 0, "gelu"), (24, 16, 7, 3, "none")]
+    layers, dense = [], []
+    for li, (i, o, k, na, act) in enumerate(specs):
+        L = inputs.make_layer(i, o, k, n_ablated=na, seed=9, stream=li)
+        v, ix, rows = oracle.pack(L.w_dense, L.mask)
+        layers.append((v, ix, rows, L.bias, i, o, act))
+        dense.append((L, act))
+    x = inputs.make_x(5, 16, seed=9)
+    outs, exact, scales = oracle.stack_forward(layers, x, dtype="bf16")
+
+    def chain(round_w, round_x, round_y):
+        cur = (_bf16_torch(x) if round_x else x).astype(np.float64)
+        ys, stored = [], []
+        for (L, act) in dense:
+            w = (_bf16_torch(L.w_dense) if round_w else L.w_dense).astype(np.float64) * L.mask
+            y = cur @ w.T + L.bias.astype(np.float64)[None, :]          # bias is NOT rounded
+            if act == "gelu":
+                y = torch.nn.functional.gelu(torch.from_numpy(y), approximate="none").numpy()
+            ys.append(y)
+            cur = (_bf16_torch(y.astype(np.float32)) if round_y else y.astype(np.float32)).astype(np.float64)
+            stored.append(cur)
+        return ys, stored
+
+    ys, stored = chain(True, True, True)
+    for i in range(len(specs)):
+        assert np.allclose(exact[i], ys[i], rtol=0, atol=1e-12), i
+        assert np.array_equal(outs[i], stored[i]), i                       # the rounded hand-over, bit for bit
+        assert _is_bf16(outs[i]), i
+        assert np.all(scales[i] >= np.abs(exact[i]) - 1e-12) or specs[i][4] == "gelu"
+    # Each rounding matters at this size: leaving one out moves the last layer by far more than 1e-12.
+    for flags in ((False, True, True), (True, False, True), (True, True, False)):
+        other, _ = chain(*flags)
+        assert np.max(np.abs(other[-1] - exact[-1])) > 1e-5, flags
+    # A bias that is not bf16-representable must come through unrounded (ablated rows of a no-activation layer).
+    L1 = dense[1][0]
+    assert not _is_bf16(L1.bias[L1.ablated])
+    assert np.array_equal(exact[1][:, L1.ablated], np.tile(L1.bias[L1.ablated].astype(np.float64), (5, 1)))
+
+
 # ---------------------------------------------------------------- generator
 def test_generator_structure_and_moments():
     L = inputs.make_layer(768, 512, 77, n_ablated=51, seed=0, stream=7)
