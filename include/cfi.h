@@ -62,9 +62,9 @@ typedef enum {
     CFI_VARIANT_SIMPLE = 1,   /* one thread per output element, no staging: a cross-check, not fast      */
     CFI_VARIANT_SPLITK = 2,   /* small batch: lanes split a row's k terms, x staged in shared memory     */
     CFI_VARIANT_BATCH = 3,    /* large batch: lanes own batch columns, x tile transposed in shared memory */
-    CFI_VARIANT_DENSE_TC = 4  /* large batch: dense copy of the weight on the tensor cores (tcgen05): bf16 layers
-                                 directly, fp32 layers as three TF32 products of split operands (K may be split over a
-                                 thread-block cluster); needs row pitches
+    CFI_VARIANT_DENSE_TC = 4  /* batch above a handful of rows: dense copy of the weight on the tensor cores (tcgen05):
+                                 bf16 layers directly, fp32 layers as three TF32 products of operands split into two
+                                 TF32-exact parts each (K may be split over a thread-block cluster); needs row pitches
                                  of x, y and the weight that are multiples of 16 bytes and no repeated column in a
                                  row, otherwise CFI_ERR_SHAPE */
 } cfi_variant_t;
@@ -224,6 +224,21 @@ cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void* x, void* 
                                  cfi_stream_t stream, cfi_variant_t variant);
 
 /*
+ * cfi_forward_dense — CFI_VARIANT_DENSE_TC with the launch shape chosen by the caller (tests and sweeps; the paper
+ * has no counterpart).  0 leaves a value to the library.
+ *
+ *   fp32 layers   tile = batch rows per tile: 16, 32, 64 or 128;  cluster = CTAs that share one tile by splitting K
+ *                 over a thread-block cluster, 1 .. 8
+ *   bf16 layers   tile = outputs per tile: 128 (one tile per CTA; cluster 1 .. 8 as above) or 256 (persistent kernel;
+ *                 cluster must be 0 or 1)
+ *
+ * CFI_ERR_SHAPE for a value outside these sets, for a cluster size the device cannot hold, or if the layer has no
+ * dense copy.  Otherwise as cfi_forward.
+ */
+cfi_status_t cfi_forward_dense(const cfi_layer_t* layer, const void* x, void* y, int32_t batch, cfi_stream_t stream,
+                               int32_t tile, int32_t cluster);
+
+/*
  * cfi_forward_host — the same operation for a caller whose activations live in host memory.
  *
  *   x_host  host (pinned memory makes the copies asynchronous), [batch, in_features]  of the layer's dtype
@@ -256,9 +271,10 @@ cfi_status_t cfi_layer_info(const cfi_layer_t* layer, cfi_layer_info_t* info);
 cfi_status_t cfi_choose_variant(const cfi_layer_t* layer, int32_t batch, int32_t* variant);
 
 /*
- * Launch shape CFI_VARIANT_DENSE_TC would use for this batch size: outputs per tile (*tile_n: 64 or 128 for fp32
- * layers; 128, or 256 for the persistent kernel, for bf16 layers) and the number of CTAs that share one output tile
- * by splitting K over a thread-block cluster (*cluster: 1 .. 8).  An introspection call for tests and benchmarks; the paper has no counterpart.
+ * Launch shape CFI_VARIANT_DENSE_TC would use for this batch size, in the terms of cfi_forward_dense: *tile_n = batch
+ * rows per tile (16, 32, 64 or 128) for fp32 layers, outputs per tile (128, or 256 for the persistent kernel) for bf16
+ * layers; *cluster = the number of CTAs that share one tile by splitting K over a thread-block cluster (1 .. 8).
+ * An introspection call for tests and benchmarks; the paper has no counterpart.
  * CFI_ERR_SHAPE if the layer has no dense copy (see CFI_VARIANT_DENSE_TC), CFI_ERR_NULL on a NULL argument.
  */
 cfi_status_t cfi_dense_tile_shape(const cfi_layer_t* layer, int32_t batch, int32_t* tile_n, int32_t* cluster);

@@ -25,7 +25,8 @@ _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE,
 _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_srigl_workspace_bytes",
-           "cfi_srigl_update", "cfi_pack_device", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_host",
+           "cfi_srigl_update", "cfi_pack_device", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_dense",
+           "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_dense_tile_shape", "cfi_device_status", "cfi_destroy",
            "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static",
            "cfi_probe_device")
@@ -78,6 +79,7 @@ def _load() -> ctypes.CDLL:
     lib.cfi_create.argtypes = [f32p, i32p, i32p, f32p, ci, ci, ci, ci, ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
     lib.cfi_forward.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_forward_variant.argtypes = [vp, vp, vp, ci, vp, ctypes.c_int]
+    lib.cfi_forward_dense.argtypes = [vp, vp, vp, ci, vp, ci, ci]
     lib.cfi_forward_host.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_layer_info.argtypes = [vp, ctypes.POINTER(LayerInfo)]
     lib.cfi_choose_variant.argtypes = [vp, ci, i32p]
@@ -257,6 +259,12 @@ def cfi_forward(layer: Layer, x, y, batch: int, stream=None) -> None:
 def cfi_forward_variant(layer: Layer, x, y, batch: int, stream=None, variant="auto") -> None:
     _check(_lib.cfi_forward_variant(layer.handle, _dev_ptr(x), _dev_ptr(y), batch, _stream_handle(stream),
                                     _VARIANTS[variant]), "cfi_forward_variant")
+
+
+def cfi_forward_dense(layer: Layer, x, y, batch: int, stream=None, tile: int = 0, cluster: int = 0) -> None:
+    """The tensor-core variant with its launch shape given (0 = chosen by the library); see include/cfi.h."""
+    _check(_lib.cfi_forward_dense(layer.handle, _dev_ptr(x), _dev_ptr(y), batch, _stream_handle(stream), tile, cluster),
+           "cfi_forward_dense")
 
 
 def cfi_forward_host(layer: Layer, x_host, y_host, batch: int, stream=None) -> None:

@@ -57,13 +57,12 @@ struct cfi_layer {
     void* stage_x = nullptr;
     void* stage_y = nullptr;
     int staged_batch = 0;
-    // Tensor-core variant (bf16 layers whose shapes TMA can address): dense copy of the weight and its tensor map.
+    // Tensor-core variant (layers whose shapes TMA can address): dense copy of the weight and its tensor map.
     const void* w_dense = nullptr;
     int out_pad = 0;
     bool tc_ok = false;
-    CUtensorMap map_w{};       // dense copy in boxes of 128 rows (bf16) or 64 rows (fp32)
-    CUtensorMap map_w_wide{};  // boxes of 128 rows (fp32) or 256 rows (bf16) for the wide tiles
-    CUtensorMap map_w_mid{};   // boxes of 96 rows (fp32 only)
+    CUtensorMap map_w{};       // dense copy in boxes of 128 rows x 128 bytes
+    CUtensorMap map_w_wide{};  // bf16 layers: boxes of 256 rows for the persistent kernel's wide tiles
 };
 
 struct cfi_stack {
@@ -617,7 +616,7 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 }
 
 #include "cfi_dense_tc.cuh"
-#include "cfi_dense_tf32.cuh"
+#include "cfi_dense_split.cuh"
 #include "cfi_dense_tc_persistent.cuh"
 
 // ------------------------------------------------------------------------------------------------
@@ -858,29 +857,31 @@ bool encode_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Time model of the split-TF32 kernel (measured): seconds per 32-column block of K and tile of 64 or 128 outputs; a
-// fixed part per wave of CTAs (prologue, pipeline fill, epilogue: CTAs are not persistent, so a second wave pays it
-// again), larger for the wide tile; the cluster reduction when K is split; and the launch itself.
-constexpr double kDenseTf32SecondsPerBlock64 = 0.45e-6, kDenseTf32SecondsPerBlock128 = 0.61e-6, kDenseTf32Wave64 = 3.0e-6,
-                 kDenseTf32Wave128 = 4.5e-6, kDenseTf32Reduce = 1.0e-6, kDenseTf32Launch = 0.7e-6;
-// 96-wide tiles: MMAs of N = 192 and N = 96, between the two by the same cost law.
-constexpr double kDenseTf32SecondsPerBlock96 = 0.53e-6, kDenseTf32Wave96 = 3.75e-6;
-constexpr int kTfMaxSplit = 8;
+constexpr int kMaxSplit = kMaxClusterSplit;
 
-template <int TN>
-int tf32_query_clusters(const cfi_layer* l, int split) {
-    if (set_smem<cfi_dense_tf32_kernel<TN>>(tf_smem_bytes(TN), l->device) != CFI_OK) return 0;
+// Time model of the split-TF32 kernel (fp32 layers on the tensor cores; measured): seconds per 32-column block of K by
+// batch tile, a fixed part per wave of CTAs (prologue, pipeline fill, epilogue: CTAs are not persistent, so a second
+// wave pays it again), the cluster reduction when K is split, and the launch itself.  The dense weight pieces
+// (4 bytes per dense entry) have to come from HBM at least once per call.
+constexpr double kSplitLaunch = 0.7e-6, kSplitWave = 4.2e-6, kSplitHbmBytesPerSecond = 5.5e12;
+double split_seconds_per_block(int bt) { return bt >= 128 ? 0.51e-6 : 0.49e-6; }  // bound by the issue of 4 + 4 MMAs and a commit
+double split_seconds_reduce(int bt) { return 0.5e-6 + 0.95e-6 * bt / 128.0; }
+int split_bt_index(int bt) { return bt >= 128 ? 3 : bt >= 64 ? 2 : bt >= 32 ? 1 : 0; }
+
+template <int BT>
+int split_query_clusters(const cfi_layer* l, int split) {
+    if (set_smem<cfi_dense_split_kernel<BT>>(sp_smem_bytes(BT), l->device) != CFI_OK) return 0;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(1, 1, (unsigned)split);
-    cfg.blockDim = dim3(kTfThreads);
-    cfg.dynamicSmemBytes = tf_smem_bytes(TN);
+    cfg.blockDim = dim3(kSpThreads);
+    cfg.dynamicSmemBytes = sp_smem_bytes(BT);
     cudaLaunchAttribute attr{};
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 1, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = (unsigned)split;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, cfi_dense_tf32_kernel<TN>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, cfi_dense_split_kernel<BT>, &cfg) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -889,70 +890,77 @@ int tf32_query_clusters(const cfi_layer* l, int split) {
 
 // Clusters of `split` CTAs of the split-TF32 kernel that the device can hold at once; 0 if it cannot launch that
 // cluster size (cached per device; -1 in the cache stands for 0).
-int tf32_resident_clusters(const cfi_layer* l, int tile_n, int split) {
-    static std::atomic<int> cache[64][3][kTfMaxSplit + 1];
+int split_resident_clusters(const cfi_layer* l, int bt, int split) {
+    static std::atomic<int> cache[kMaxDevices][4][kMaxSplit + 1];
     if (split == 1) return std::max(1, l->sm_count);
-    if (l->device < 0 || l->device >= 64) return 0;
-    std::atomic<int>& c = cache[l->device][tile_n == 128 ? 2 : tile_n == 96 ? 1 : 0][split];
+    if (l->device < 0 || l->device >= kMaxDevices) return 0;
+    std::atomic<int>& c = cache[l->device][split_bt_index(bt)][split];
     int v = c.load(std::memory_order_acquire);
     if (v == 0) {
-        v = tile_n == 128  ? tf32_query_clusters<128>(l, split)
-            : tile_n == 96 ? tf32_query_clusters<96>(l, split)
-                           : tf32_query_clusters<64>(l, split);
+        v = bt >= 128  ? split_query_clusters<128>(l, split)
+            : bt >= 64 ? split_query_clusters<64>(l, split)
+            : bt >= 32 ? split_query_clusters<32>(l, split)
+                       : split_query_clusters<16>(l, split);
         if (v <= 0) v = -1;
         c.store(v, std::memory_order_release);
     }
     return v > 0 ? v : 0;
 }
 
-struct Tf32Shape {
-    int tile_n;      // outputs per tile: 64, 96 or 128
+struct SplitShape {
+    int bt;          // batch rows per tile: 16, 32, 64 or 128 (the MMA's N is twice that)
     int split;       // CTAs per output tile (cluster size along z): 1 .. 8
     double seconds;  // modelled time of the launch
+    bool ok;
 };
 
-// Wide tiles need fewer MMA instructions per output; splitting K over a cluster fills the SMs that the tiles alone
-// would leave idle, as long as every CTA still gets a few K blocks.
-Tf32Shape tf32_shape(const cfi_layer* l, int batch) {
-    const int k_blocks = (l->d.in + kTfK - 1) / kTfK;
-    Tf32Shape best{64, 1, 0.0};
-    bool have = false;
-    for (int tile_n = 64; tile_n <= 128; tile_n += 32) {
-        const int64_t tiles = (int64_t)((batch + kTfM - 1) / kTfM) * ((l->d.out + tile_n - 1) / tile_n);
-        const double per_block = tile_n == 128  ? kDenseTf32SecondsPerBlock128
-                                 : tile_n == 96 ? kDenseTf32SecondsPerBlock96
-                                                : kDenseTf32SecondsPerBlock64;
-        const double per_wave = tile_n == 128 ? kDenseTf32Wave128 : tile_n == 96 ? kDenseTf32Wave96 : kDenseTf32Wave64;
-        for (int split = 1; split <= kTfMaxSplit; ++split) {
-            if (split > 1 && (k_blocks < 4 * split || tiles * split > 2 * (int64_t)l->sm_count)) break;
-            const int64_t resident = tf32_resident_clusters(l, tile_n, split);
+// Batch tile and K split: a narrower batch tile costs less per K block, a wider one shares each weight box among more
+// batch rows; splitting K over a cluster fills the SMs that the tiles alone would leave idle, as long as every CTA
+// still gets a few K blocks.  force_bt / force_split (0 = free) pin one or both.
+SplitShape split_shape(const cfi_layer* l, int batch, int force_bt = 0, int force_split = 0) {
+    const int k_blocks = (l->d.in + kSpK - 1) / kSpK, tiles_m = (l->d.out + kSpM - 1) / kSpM;
+    const double t_hbm = 4.0 * l->out_pad * (double)l->d.in / kSplitHbmBytesPerSecond;
+    SplitShape best{128, 1, 0.0, false};
+    for (int bt = 16; bt <= 128; bt <<= 1) {
+        if (force_bt && bt != force_bt) continue;
+        const int64_t tiles_b = (batch + bt - 1) / bt;
+        if (tiles_b > 65535) continue;
+        const int64_t tiles = tiles_m * tiles_b;
+        for (int split = 1; split <= kMaxSplit; ++split) {
+            if (force_split ? split != force_split : (split > 1 && (k_blocks < 2 * split || tiles * split > 2 * (int64_t)l->sm_count))) continue;
+            const int64_t resident = split_resident_clusters(l, bt, split);
             if (resident == 0) continue;
             const int64_t waves = (tiles + resident - 1) / resident;
-            const double t = (double)waves * (((k_blocks + split - 1) / split) * per_block + per_wave +
-                                              (split > 1 ? kDenseTf32Reduce : 0.0)) + kDenseTf32Launch;
-            if (!have || t < best.seconds) best = Tf32Shape{tile_n, split, t}, have = true;
+            const double main = (double)waves * ((k_blocks + split - 1) / split) * split_seconds_per_block(bt);
+            const double t = std::max(main, t_hbm) + (double)waves * (kSplitWave + (split > 1 ? split_seconds_reduce(bt) : 0.0)) + kSplitLaunch;
+            if (!best.ok || t < best.seconds) best = SplitShape{bt, split, t, true};
         }
     }
     return best;
 }
 
-template <int TN>
-cfi_status_t launch_dense_tf32_n(const cfi_layer* l, const CUtensorMap& map_x, const CUtensorMap& map_w, int split, void* y,
-                                 int batch, cudaStream_t st) {
-    const int grid_x = (l->d.out + TN - 1) / TN, grid_y = (batch + kTfM - 1) / kTfM;
-    if (cfi_status_t e = set_smem<cfi_dense_tf32_kernel<TN>>(tf_smem_bytes(TN), l->device)) return e;
-    return launch_pdl_cluster(cfi_dense_tf32_kernel<TN>, dim3(grid_x, grid_y, split), kTfThreads, tf_smem_bytes(TN), split, st,
-                              l->d, map_x, map_w, static_cast<float*>(y), batch);
+template <int BT>
+cfi_status_t launch_dense_split_bt(const cfi_layer* l, int split, const void* x, void* y, int batch, cudaStream_t st) {
+    const int grid_x = (l->d.out + kSpM - 1) / kSpM, grid_y = (batch + BT - 1) / BT;
+    CUtensorMap map_x;  // x in boxes of BT rows x 32 columns
+    if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 4, BT)) return CFI_ERR_SHAPE;
+    if (cfi_status_t e = set_smem<cfi_dense_split_kernel<BT>>(sp_smem_bytes(BT), l->device)) return e;
+    return launch_pdl_cluster(cfi_dense_split_kernel<BT>, dim3(grid_x, grid_y, split), kSpThreads, sp_smem_bytes(BT), split, st, l->d,
+                              l->map_w, map_x, static_cast<float*>(y), batch);
 }
 
-cfi_status_t launch_dense_tf32(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
-    if ((batch + kTfM - 1) / kTfM > 65535) return CFI_ERR_SHAPE;
-    CUtensorMap map_x;
-    if (!encode_map(&map_x, x, (uint64_t)batch, (uint64_t)l->d.in, 4, kTfM)) return CFI_ERR_SHAPE;
-    const Tf32Shape sh = tf32_shape(l, batch);
-    if (sh.tile_n == 128) return launch_dense_tf32_n<128>(l, map_x, l->map_w_wide, sh.split, y, batch, st);
-    if (sh.tile_n == 96) return launch_dense_tf32_n<96>(l, map_x, l->map_w_mid, sh.split, y, batch, st);
-    return launch_dense_tf32_n<64>(l, map_x, l->map_w, sh.split, y, batch, st);
+cfi_status_t launch_dense_split(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st, int force_bt = 0,
+                                int force_split = 0) {
+    if (force_bt && force_bt != 16 && force_bt != 32 && force_bt != 64 && force_bt != 128) return CFI_ERR_SHAPE;
+    if (force_split < 0 || force_split > kMaxSplit) return CFI_ERR_SHAPE;
+    const SplitShape sh = split_shape(l, batch, force_bt, force_split);
+    if (!sh.ok) return CFI_ERR_SHAPE;
+    switch (sh.bt) {
+        case 16: return launch_dense_split_bt<16>(l, sh.split, x, y, batch, st);
+        case 32: return launch_dense_split_bt<32>(l, sh.split, x, y, batch, st);
+        case 64: return launch_dense_split_bt<64>(l, sh.split, x, y, batch, st);
+        default: return launch_dense_split_bt<128>(l, sh.split, x, y, batch, st);
+    }
 }
 
 // bf16: with at least one 128 x 256 tile per SM the persistent kernel runs (measured: faster from about there
@@ -965,7 +973,7 @@ bool tc_bf16_persistent(const cfi_layer* l, int batch) {
 // Clusters of `split` CTAs of the one-tile bf16 kernel that the device can hold at once; 0 if it cannot launch that
 // cluster size (cached per device; -1 in the cache stands for 0).  Both activations have the same footprint.
 int tc_bf16_resident_clusters(const cfi_layer* l, int split) {
-    static std::atomic<int> cache[64][kTfMaxSplit + 1];
+    static std::atomic<int> cache[64][kMaxSplit + 1];
     if (split == 1) return std::max(1, 2 * l->sm_count);
     if (l->device < 0 || l->device >= 64) return 0;
     std::atomic<int>& c = cache[l->device][split];
@@ -998,7 +1006,7 @@ int tc_bf16_split(const cfi_layer* l, int batch, double* seconds = nullptr) {
     const int k_blocks = (l->d.in + kTcK - 1) / kTcK;
     int best = 1;
     double best_t = 0.0;
-    for (int split = 1; split <= kTfMaxSplit; ++split) {
+    for (int split = 1; split <= kMaxSplit; ++split) {
         if (split > 1 && (k_blocks < 4 * split || tiles * split > 4 * (int64_t)l->sm_count)) break;
         const int64_t resident = tc_bf16_resident_clusters(l, split);
         if (resident == 0) continue;
@@ -1010,9 +1018,14 @@ int tc_bf16_split(const cfi_layer* l, int batch, double* seconds = nullptr) {
     return best;
 }
 
-cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
+// tile / cluster: 0 = chosen here.  fp32 layers: tile = batch rows per tile (16, 32, 64, 128); bf16 layers: tile = outputs
+// per tile, 128 (one tile per CTA, K may be split over `cluster` CTAs) or 256 (persistent kernel, no split).
+cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st, int tile = 0,
+                             int cluster = 0) {
     if (!l->tc_ok) return CFI_ERR_SHAPE;
-    if (l->dtype != CFI_BF16) return launch_dense_tf32(l, x, y, batch, st);
+    if (l->dtype != CFI_BF16) return launch_dense_split(l, x, y, batch, st, tile, cluster);
+    if ((tile != 0 && tile != kTcN && tile != kTpN) || cluster < 0 || cluster > kMaxSplit || (tile == kTpN && cluster > 1))
+        return CFI_ERR_SHAPE;
     const int grid_x = (l->d.out + kTcN - 1) / kTcN, grid_y = (batch + kTcM - 1) / kTcM;
     if (grid_y > 65535) return CFI_ERR_SHAPE;
     CUtensorMap map_x;
@@ -1021,8 +1034,9 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
     // the next tile's MMAs.
     const int wide_x = (l->d.out + kTpN - 1) / kTpN;
     const int64_t n_tiles = (int64_t)wide_x * grid_y;
-    if (tc_bf16_persistent(l, batch)) {
-        const int ctas = l->sm_count;
+    if (tile == kTpN || (tile == 0 && cluster == 0 && tc_bf16_persistent(l, batch))) {
+        if (n_tiles >= (1ll << 31)) return CFI_ERR_SHAPE;
+        const int ctas = (int)std::min<int64_t>(l->sm_count, n_tiles);
         CUtensorMap map_y;  // y leaves through TMA stores of 128-row x 64-column boxes
         if (!encode_map(&map_y, y, (uint64_t)batch, (uint64_t)l->d.out, 2, kTcM)) return CFI_ERR_SHAPE;
         if (l->d.act == CFI_ACT_GELU_ERF) {
@@ -1034,7 +1048,8 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
         return launch_pdl(cfi_dense_tc_persistent_kernel<CFI_ACT_NONE>, dim3(ctas), kTpThreads, kTpSmemBytes, st, l->d, map_x,
                           l->map_w_wide, map_y, batch, wide_x, (int)n_tiles);
     }
-    const int split = tc_bf16_split(l, batch);
+    const int split = cluster ? cluster : tc_bf16_split(l, batch);
+    if (split > 1 && tc_bf16_resident_clusters(l, split) == 0) return CFI_ERR_SHAPE;
     if (l->d.act == CFI_ACT_GELU_ERF) {
         if (cfi_status_t e = set_smem<cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>>(kTcSmemBytes, l->device)) return e;
         return launch_pdl_cluster(cfi_dense_tc_kernel<CFI_ACT_GELU_ERF>, dim3(grid_x, grid_y, split), kTcThreads, kTcSmemBytes,
@@ -1069,7 +1084,7 @@ int choose_variant(const cfi_layer* l, int batch) {
             const double t_stage = (double)l->d.in * 8 * 4 / 1024.0 * 90e-9, t_fma = (double)l->d.n_active * l->d.k / 176e9;
             const double t_splitk = ((batch + 7) / 8) * (2.3e-6 + std::max(t_stage, t_fma));
             double t_dense = 0.0;
-            if (l->dtype == CFI_F32) t_dense = tf32_shape(l, batch).seconds;
+            if (l->dtype == CFI_F32) t_dense = split_shape(l, batch).seconds;
             else tc_bf16_split(l, batch, &t_dense);
             if (t_dense < t_splitk) return CFI_VARIANT_DENSE_TC;
         }
@@ -1086,7 +1101,7 @@ int choose_variant(const cfi_layer* l, int batch) {
         // of x by every row tile.  Constants fitted to measurements.
         const BatchShape bs = batch_shape(l, batch);
         if (!bs.ok) return CFI_VARIANT_DENSE_TC;
-        const double t_dense = tf32_shape(l, batch).seconds;
+        const double t_dense = split_shape(l, batch).seconds;
         const double staging = (double)bs.grid_y * kBatchTile * l->d.in * 4.0 * bs.grid_x;
         // Arithmetic and the re-staging of x overlap about half of the shorter of the two.
         const double t_fma = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12), t_stage = staging / 3.7e12;
@@ -1335,8 +1350,8 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                           seg_o.begin() + (size_t)o * (d.n_slabs + 1));
         if (st == CFI_OK) st = upload(l, seg_o, &d.seg);
 
-        // ---- dense copy for the tensor-core variant (zero rows for ablated and padding rows): bf16 for bf16 layers,
-        // fp32 for fp32 layers.  A column kept twice in one row cannot be one dense entry, so such layers go without.
+        // ---- dense copy for the tensor-core variant (zero rows for ablated and padding rows), in the layer's dtype.
+        // A column kept twice in one row cannot be one dense entry, so such layers go without.
         {
             const int eb = dtype == CFI_BF16 ? 2 : 4, tile_n = 128;
             bool usable = out_features > 0 && in_features * eb >= 16 && ((in_features * eb) & 15) == 0 &&
@@ -1365,13 +1380,11 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
                     wd_dev = p;
                 }
                 l->w_dense = wd_dev;
-                l->tc_ok = st == CFI_OK && encode_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb,
-                                                      dtype == CFI_BF16 ? kTcN : 64);
-                if (l->tc_ok)  // the same copy in the boxes of the wide tiles: 128 rows (fp32), 256 rows (bf16)
-                    l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb,
-                                          dtype == CFI_BF16 ? kTpN : 128);
-                if (l->tc_ok && dtype != CFI_BF16)
-                    l->tc_ok = encode_map(&l->map_w_mid, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb, 96);
+                // Boxes of 128 rows x 128 bytes for the one-tile kernels; for bf16 layers also 256-row boxes for the
+                // persistent kernel's wide tiles.
+                l->tc_ok = st == CFI_OK && encode_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb, kTcN);
+                if (l->tc_ok && dtype == CFI_BF16)
+                    l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, 2, kTpN);
             }
         }
 
@@ -1416,8 +1429,9 @@ extern "C" cfi_status_t cfi_dense_tile_shape(const cfi_layer_t* layer, int32_t b
         const bool persistent = tc_bf16_persistent(layer, batch);
         *tile_n = persistent ? kTpN : kTcN, *cluster = persistent ? 1 : tc_bf16_split(layer, batch);
     } else {
-        const Tf32Shape sh = tf32_shape(layer, batch);
-        *tile_n = sh.tile_n, *cluster = sh.split;
+        const SplitShape sh = split_shape(layer, batch);
+        if (!sh.ok) return CFI_ERR_SHAPE;
+        *tile_n = sh.bt, *cluster = sh.split;
     }
     return CFI_OK;
 }
@@ -1451,6 +1465,17 @@ extern "C" cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void
         }
     }
     return CFI_ERR_DTYPE;
+}
+
+extern "C" cfi_status_t cfi_forward_dense(const cfi_layer_t* layer, const void* x, void* y, int32_t batch, cfi_stream_t stream,
+                                          int32_t tile, int32_t cluster) {
+    if (!layer) return CFI_ERR_NULL;
+    if (batch < 0) return CFI_ERR_SHAPE;
+    if (batch == 0 || layer->d.out == 0) return CFI_OK;
+    if (!y || (!x && layer->d.in > 0)) return CFI_ERR_NULL;
+    if (((uintptr_t)x | (uintptr_t)y) & 15u) return CFI_ERR_ALIGNMENT;
+    DeviceGuard g(layer->device);
+    return launch_dense_tc(layer, x, y, batch, reinterpret_cast<cudaStream_t>(stream), tile, cluster);
 }
 
 extern "C" cfi_status_t cfi_forward(const cfi_layer_t* layer, const void* x, void* y, int32_t batch,

@@ -32,8 +32,9 @@ def device_layer(layer, dtype="f32", act="none"):
     return cfi.cfi_create(v, ix, rows, layer.bias, layer.in_features, layer.out_features, dtype=dtype, act=act)
 
 
-def run_device(dl, x_np, dtype="f32", variant="auto", canary=True):
-    """Forward through the library; y is allocated inside guard bands that must come back untouched."""
+def run_device(dl, x_np, dtype="f32", variant="auto", canary=True, dense_shape=None):
+    """Forward through the library; y is allocated inside guard bands that must come back untouched.
+    dense_shape = (tile, cluster) runs the tensor-core variant with that launch shape (cfi_forward_dense)."""
     import torch
     from paper_2305_02299_b200 import binding as cfi
     B = x_np.shape[0]
@@ -43,7 +44,10 @@ def run_device(dl, x_np, dtype="f32", variant="auto", canary=True):
     buf = torch.full((n + 2 * guard,), 12345.0, device="cuda", dtype=torch_dtype(dtype))
     y_d = buf[guard:guard + n]
     assert y_d.data_ptr() % 16 == 0
-    cfi.cfi_forward_variant(dl, x_d, y_d, B, variant=variant)
+    if dense_shape is not None:
+        cfi.cfi_forward_dense(dl, x_d, y_d, B, tile=dense_shape[0], cluster=dense_shape[1])
+    else:
+        cfi.cfi_forward_variant(dl, x_d, y_d, B, variant=variant)
     torch.cuda.synchronize()
     if canary:
         assert torch.all(buf[:guard] == 12345.0) and torch.all(buf[guard + n:] == 12345.0), "wrote outside y"

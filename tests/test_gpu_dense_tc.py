@@ -2,8 +2,8 @@
 
 bf16 layers: exact bf16 products, fp32 accumulation, so the bf16 tolerance of the other parity tests applies.
 fp32 layers: three TF32 products of operands split into two TF32-exact parts; what the split drops is below
-2^-19 of each term, so the fp32 tolerance (1e-5 of the sum's scale) applies unchanged.  Small-integer cases
-must agree bit for bit in both.
+3 * 2^-20 of each term, so the fp32 tolerance (1e-5 of the sum's scale) applies unchanged, down to a fan-in of one.
+Small-integer cases must agree bit for bit in both.
 """
 import numpy as np
 import pytest
@@ -31,30 +31,47 @@ def test_dense_tc_matches_oracle(in_f, out_f, k, nabl, B, act, dtype):
     assert_parity(y, y_ref, S, dtype)
 
 
-# (in, out, k, ablated, batch) chosen so that together they run all three tile widths and clusters of several sizes.
-TF32_SHAPES = [(3072, 768, 307, 77, 256), (3072, 768, 307, 77, 64), (768, 3072, 77, 0, 256), (768, 3072, 77, 0, 100),
-               (4096, 512, 205, 10, 130), (1000, 72, 100, 5, 257), (520, 640, 52, 30, 128), (768, 3072, 77, 150, 700)]
+# fp32: every batch tile (16, 32, 64, 128 rows; the MMAs are 2 x and 1 x that wide) with and without a K split over a
+# thread-block cluster, on shapes with ragged output, batch and K tails, few and many K blocks per CTA (more blocks
+# than ring stages, fewer blocks than CTAs of the cluster), ablated rows and both activations.
+SPLIT_SHAPES = [(768, 384, 77, 19, 200, "gelu"), (3072, 200, 307, 20, 70, "none"), (1000, 72, 100, 5, 257, "gelu"),
+                (520, 640, 52, 30, 129, "none"), (64, 8, 5, 1, 5, "gelu"), (40, 136, 1, 7, 33, "none")]
 
 
-def test_dense_tf32_launch_shapes_cover_wide_tiles_and_clusters():
-    """Every tile width and several cluster sizes occur among TF32_SHAPES (else the cases below prove less than
-    they seem to), and each case matches the oracle."""
+@pytest.mark.parametrize("tile", [16, 32, 64, 128])
+@pytest.mark.parametrize("cluster", [1, 2, 3, 4, 8])
+def test_dense_split_tf32_every_launch_shape(tile, cluster):
     from paper_2305_02299_b200 import binding as cfi
-    seen = set()
-    for in_f, out_f, k, nabl, B in TF32_SHAPES:
+    for in_f, out_f, k, nabl, B, act in SPLIT_SHAPES:
         L = inputs.make_layer(in_f, out_f, k, n_ablated=nabl, seed=in_f + out_f)
         x = inputs.make_x(B, in_f, seed=B)
-        y_ref, S = oracle_layer(L, x, "f32", "gelu")
-        dl = device_layer(L, "f32", "gelu")
-        shape = cfi.cfi_dense_tile_shape(dl, B)
-        seen.add(shape)
-        y = run_device(dl, x, "f32", "dense_tc")
+        y_ref, S = oracle_layer(L, x, "f32", act)
+        dl = device_layer(L, "f32", act)
+        y = run_device(dl, x, "f32", dense_shape=(tile, cluster))
+        y2 = run_device(dl, x, "f32", dense_shape=(tile, cluster))
+        assert cfi.cfi_device_status(dl) == 0
         dl.close()
-        assert scaled_error(y, y_ref, S) <= TOL["f32"], (in_f, out_f, B, shape)
-    tiles = {t for t, _ in seen}
-    clusters = {c for _, c in seen}
-    assert tiles == {64, 96, 128}, seen
-    assert 1 in clusters and len([c for c in clusters if c > 1]) >= 2, seen
+        assert scaled_error(y, y_ref, S) <= TOL["f32"], (in_f, out_f, B, tile, cluster)
+        assert np.array_equal(y, y2)                      # fixed order of additions: the same bits every time
+
+
+def test_dense_split_tf32_shape_choice_and_bad_shapes():
+    """The shape the library picks is one of the allowed ones and runs; values outside the sets are refused."""
+    from paper_2305_02299_b200 import binding as cfi
+    L = inputs.make_layer(3072, 768, 307, n_ablated=77, seed=2)
+    dl = device_layer(L, "f32")
+    seen = set()
+    for B in (9, 16, 40, 64, 100, 256, 700):
+        tile, cluster = cfi.cfi_dense_tile_shape(dl, B)
+        assert tile in (16, 32, 64, 128) and 1 <= cluster <= 8
+        seen.add((tile, cluster))
+    assert len({c for _, c in seen}) >= 2 and len({t for t, _ in seen}) >= 2, seen   # few output tiles, long K: K is split
+    x = inputs.make_x(16, 3072)
+    for tile, cluster in ((48, 1), (256, 1), (64, 9), (64, -1)):
+        with pytest.raises(cfi.CfiError) as e:
+            run_device(dl, x, "f32", dense_shape=(tile, cluster))
+        assert e.value.status == 2
+    dl.close()
 
 
 @pytest.mark.parametrize("in_f,out_f,k,nabl,B,act", [(768, 1000, 77, 50, 9601, "gelu"), (1024, 512, 102, 0, 19001, "none"),
@@ -100,7 +117,7 @@ def test_dense_tc_bf16_cluster_split_is_exercised():
     assert 1 in clusters and len([c for c in clusters if c > 1]) >= 2, seen
 
 
-def test_dense_tf32_wide_dynamic_range():
+def test_dense_split_tf32_wide_dynamic_range():
     """Inputs spread over many binades: the split must hold for every magnitude, not only for N(0,1)."""
     L = inputs.make_layer(512, 128, 51, n_ablated=7, seed=9)
     rng = np.random.default_rng(4)
