@@ -119,15 +119,17 @@ class Replicas:
     """R independent copies of (layer, x, y) so that consecutive steps touch different memory."""
 
     def __init__(self, w: inputs.Workload, cfi, torch, min_total_bytes: int, dtype: str = "f32", seed: int = 0,
-                 rank: int = 0, max_replicas: int = 64):
+                 rank: int = 0, max_replicas: int = 64, layer=None, packed=None, layouts: int = 7, streamed_bytes=None):
         self.w, self.cfi, self.torch = w, cfi, torch
         tdt = torch.float32 if dtype == "f32" else torch.bfloat16
-        base = w.layer(seed=seed, replica=0)
-        v, ix, rows = cfi.cfi_pack(base.w_dense, base.mask)
+        base = layer if layer is not None else w.layer(seed=seed, replica=0)
+        v, ix, rows = packed if packed is not None else cfi.cfi_pack(base.w_dense, base.mask)
         self.n_active = int(rows.shape[0])
         elem = 4 if dtype == "f32" else 2
         self.bytes_per_step = algorithmic_bytes(w, self.n_active, elem)
-        per = self.bytes_per_step
+        # What one call streams from memory decides how many replicas make the rotation cold: the condensed arrays
+        # and activations, or more when the kernel in use reads the dense copy.
+        per = max(self.bytes_per_step, streamed_bytes or 0)
         self.R = int(max(2, min(max_replicas, -(-min_total_bytes // per))))
         self.layers, self.x, self.y = [], [], []
         rng = np.random.default_rng(1234 + rank)
@@ -136,11 +138,12 @@ class Replicas:
             # (cheap) instead of drawing a fresh dense matrix per replica.
             p = rng.permutation(self.n_active)
             self.layers.append(cfi.cfi_create(v[p], ix[p], rows, base.bias, w.in_features, w.out_features,
-                                              dtype=dtype, act=w.act))
+                                              dtype=dtype, act=w.act, layouts=layouts))
             xr = w.x(seed=seed, replica=r + 100 * rank)
             self.x.append(torch.from_numpy(xr).to("cuda", tdt).contiguous())
             self.y.append(torch.empty((w.batch, w.out_features), device="cuda", dtype=tdt))
         self.total_bytes = self.R * per
+        self.layouts = layouts
 
     def step(self, i: int, variant: str = "auto"):
         r = i % self.R
@@ -152,8 +155,12 @@ class Replicas:
 
 
 def time_steps(rep: Replicas, torch, steps: int, warmup: int, variant: str = "auto", graph_len: int = 1000,
-               barrier=None, sampler=None):
-    """Returns (seconds for exactly `steps` steps, launches).  Warm-up covers every replica at least once."""
+               barrier=None, sampler=None, target_s: float = 0.25, max_passes: int = 5000):
+    """Times passes of exactly `steps` steps each (CUDA-graph replays between CUDA events on the launching stream)
+    and returns a dict: median and standard deviation of the per-step time over the passes, the number of passes,
+    the launches of one pass.  A short pass (few steps) is repeated until about `target_s` seconds have been timed,
+    at least five times, so that the figure is a steady-state one and the clock sampler sees the region.
+    Warm-up covers every replica at least once."""
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
         for i in range(max(warmup, 3)):
@@ -172,26 +179,45 @@ def time_steps(rep: Replicas, torch, steps: int, warmup: int, variant: str = "au
             graphs.append(g)
         main = graphs[0] if n_replay else None
         tail = graphs[-1] if rem else None
-        for g in graphs:            # one untimed replay each (graph upload)
-            g.replay()
-        stream.synchronize()
-        if barrier:
-            barrier()
-        torch.cuda.synchronize()
-        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ctx = sampler if sampler is not None else _Null()
-        with ctx:
-            start.record(stream)
+
+        def one_pass():
             for _ in range(n_replay):
                 main.replay()
             if tail is not None:
                 tail.replay()
-            end.record(stream)
-            end.synchronize()
+
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        one_pass()                  # graph upload
+        stream.synchronize()
+        a.record(stream)
+        one_pass()                  # untimed estimate of a pass
+        b.record(stream)
+        b.synchronize()
+        est = max(a.elapsed_time(b) * 1e-3, 1e-6)
+        passes = int(min(max_passes, max(5, -(-target_s // est))))
+        if barrier:
+            barrier()
+        torch.cuda.synchronize()
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(passes + 1)]
+        ctx = sampler if sampler is not None else _Null()
+        with ctx:
+            events[0].record(stream)
+            for p in range(passes):
+                one_pass()
+                events[p + 1].record(stream)
+            events[-1].synchronize()
         torch.cuda.synchronize()
         if barrier:
             barrier()
-    return start.elapsed_time(end) * 1e-3, steps
+    per_pass = [events[p].elapsed_time(events[p + 1]) * 1e-3 for p in range(passes)]
+    return {"sec_per_step": statistics.median(per_pass) / steps, "std_sec_per_step": statistics.pstdev(per_pass) / steps,
+            "passes": passes, "steps_per_pass": steps, "launches_per_pass": steps,
+            "timed_s": events[0].elapsed_time(events[-1]) * 1e-3}
+
+
+def us(t):
+    """Per-step microseconds of a time_steps result."""
+    return t["sec_per_step"] * 1e6
 
 
 class _Null:
@@ -203,14 +229,16 @@ class _Null:
 
 
 def time_e2e(rep: Replicas, torch, steps: int, warmup: int):
-    """Through cfi_forward_host: pinned host x -> device, forward, y -> pinned host, every step."""
+    """Through cfi_forward_host: pinned host x -> device, forward, y -> pinned host, every step.  The warm-up calls
+    every replica once, so each layer's staging buffers exist before the timed region starts (the entry point
+    allocates them on a layer's first call)."""
     w = rep.w
     tdt = rep.x[0].dtype
     xh = [rep.x[r].cpu().pin_memory() for r in range(min(rep.R, 8))]
     yh = torch.empty((w.batch, w.out_features), dtype=tdt).pin_memory()
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
-        for i in range(max(3, warmup)):
+        for i in range(max(3, warmup, rep.R)):
             rep.cfi.cfi_forward_host(rep.layers[i % rep.R], xh[i % len(xh)], yh, w.batch)
         torch.cuda.synchronize()
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -226,29 +254,43 @@ def time_e2e(rep: Replicas, torch, steps: int, warmup: int):
 # --------------------------------------------------------------------------------------------------
 # CPU oracle timing (reported baseline, and the --impl reference arm)
 # --------------------------------------------------------------------------------------------------
-def time_oracle(w: inputs.Workload, budget_s: float, sample_rows=None, repeats=None):
+def time_oracle(w: inputs.Workload, budget_s: float, sample_rows=None, threads=None, packed=None, layer=None):
+    """The oracle as it stands on this host, on the first `sample_rows` batch rows of the workload (all of them by
+    default, fewer if one call would take longer than the budget): median seconds per call and the flops of a call."""
     import oracle
-    L = w.layer(seed=0)
-    v, ix, rows = oracle.pack(L.w_dense, L.mask)
+    L = layer if layer is not None else w.layer(seed=0)
+    v, ix, rows = packed if packed is not None else oracle.pack(L.w_dense, L.mask)
     x = w.x(seed=0)
-    if sample_rows is None:
-        sample_rows = w.batch
-    xs = np.ascontiguousarray(x[:sample_rows])
-    call = lambda: oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, xs, act=w.act)
-    call()
-    t0 = time.perf_counter()
-    call()
-    one = time.perf_counter() - t0
-    if repeats is None:
-        repeats = int(max(5, min(2000, budget_s / max(one, 1e-6))))
-    times = []
-    for _ in range(repeats):
+    all_threads = oracle.max_threads()
+    if threads:
+        oracle.set_threads(threads)
+    try:
+        n = w.batch if sample_rows is None else min(sample_rows, w.batch)
+        t0 = time.perf_counter()
+        oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, x[:1], act=w.act)
+        per_row = max(time.perf_counter() - t0, 1e-7)
+        n = int(max(1, min(n, budget_s / 5.0 / per_row)))          # at least five calls fit the budget
+        xs = np.ascontiguousarray(x[:n])
+        call = lambda: oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, xs, act=w.act)
+        call()
         t0 = time.perf_counter()
         call()
-        times.append(time.perf_counter() - t0)
-    flops = 2 * sample_rows * rows.shape[0] * w.k
-    return {"median_s": statistics.median(times), "flops": flops, "calls": repeats, "rows": sample_rows,
-            "cores": oracle.max_threads()}
+        one = time.perf_counter() - t0
+        repeats = int(max(5, min(2000, budget_s / max(one, 1e-6))))
+        times = []
+        for _ in range(repeats):
+            t0 = time.perf_counter()
+            call()
+            times.append(time.perf_counter() - t0)
+    finally:
+        oracle.set_threads(all_threads)
+    return {"median_s": statistics.median(times), "std_s": statistics.pstdev(times), "flops": 2 * n * rows.shape[0] * w.k,
+            "calls": repeats, "rows": n, "cores": threads or all_threads}
+
+
+def config_keys(w, n_active):
+    """The keys both arms print under `config`: they name the workload and nothing else."""
+    return {"workload": w.name, "in": w.in_features, "out": w.out_features, "k": w.k, "n_active": int(n_active), "batch": w.batch}
 
 
 def run_reference(args, w):
@@ -268,18 +310,19 @@ def run_reference(args, w):
     xs = np.ascontiguousarray(x[:sample])
     for _ in range(args.warmup):
         oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, xs)
-    t0 = time.perf_counter()
+    times = []
     for _ in range(args.steps):
+        t0 = time.perf_counter()
         oracle.forward(v, ix, rows, L.bias, w.in_features, w.out_features, xs)
-    sec = time.perf_counter() - t0
+        times.append(time.perf_counter() - t0)
+    sec = sum(times)
     gflops = 2 * sample * rows.shape[0] * w.k * args.steps / sec / 1e9
     cores = oracle.max_threads()
     desc = f"{sample} of {w.batch} batch rows per step, all {w.out_features} output rows"
     line = {"impl": "reference", "metric": METRIC, "value": gflops, "unit": "GFLOP/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "in": w.in_features, "out": w.out_features, "k": w.k, "batch": w.batch,
-                       "sample": desc},
+            "config": config_keys(w, rows.shape[0]),
             "cpu_baseline": {"value": gflops, "unit": "GFLOP/s", "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": gflops, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -309,7 +352,7 @@ def main():
         args.warmup = 3 if args.warmup is None else args.warmup
         run_reference(args, w)
         return
-    args.steps = 200000 if args.steps is None else args.steps
+    args.steps = 20000 if args.steps is None else args.steps
     args.warmup = 20 if args.warmup is None else args.warmup
 
     import torch
@@ -343,67 +386,61 @@ def main():
     props = torch.cuda.get_device_properties(local)
     l2 = getattr(props, "L2_cache_size", None) or L2_BYTES_FALLBACK
     sm_count = props.multi_processor_count
+    ceil_ = Ceilings(peaks, peak_kind, sm_count)
 
     rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), rank=rank)
     sampler = ClockSampler(local)
-    sec, launches = time_steps(rep, torch, args.steps, args.warmup, args.variant, barrier=barrier, sampler=sampler)
-    sec = max_over_ranks(sec, dist, "cuda")
+    timed = time_steps(rep, torch, args.steps, args.warmup, args.variant, barrier=barrier, sampler=sampler)
+    per_call = max_over_ranks(timed["sec_per_step"], dist, "cuda")
     flops = algorithmic_flops(w, rep.n_active)
-    per_call = sec / args.steps
     value = whole_job_value(flops, world, per_call)
 
     # End to end through the host-buffer entry point (each rank on its own GPU).
-    e2e_steps = int(min(args.steps, 2000))
+    e2e_steps = int(min(max(args.steps, 200), 2000))
     e2e_sec, h2d, d2h = time_e2e(rep, torch, e2e_steps, 5)
     e2e_sec = max_over_ranks(e2e_sec, dist, "cuda")
     e2e_value = whole_job_value(flops, world, e2e_sec / e2e_steps)
 
     line = None
     if rank == 0:
-        sm_max_mhz = float(peaks.get("sm_max_mhz", 1965.0))
-        fma_peak_tflops = sm_count * FMA_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
         achieved_tflops = flops / per_call / 1e12
         hbm_gbs = rep.bytes_per_step / per_call / 1e9
         info = cfi.cfi_layer_info(rep.layers[0])
-        chosen = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
-        tile_shape = None
-        if chosen == "dense_tc" and args.variant in ("auto", "dense_tc"):
-            tn, cl = cfi.cfi_dense_tile_shape(rep.layers[0], w.batch)
-            tile_shape = {"tile": [128, tn], "cluster_k_split": cl}
+        chosen = VARIANT_NAMES[cfi.cfi_choose_variant(rep.layers[0], w.batch)] if args.variant == "auto" else args.variant
+        shape = dense_shape(cfi, rep.layers[0], w.batch) if chosen == "dense_tc" else None
         line = {
             "metric": METRIC, "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": per_call * 1e3, "us_per_call": per_call * 1e6,
+            "us_per_call_std": timed["std_sec_per_step"] * 1e6, "timed_passes": timed["passes"], "timed_s": timed["timed_s"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "in": w.in_features, "out": w.out_features, "k": w.k,
-                       "n_active": rep.n_active, "batch": w.batch, "variant": chosen if args.variant == "auto" else args.variant,
-                       "dense_tile": tile_shape,
-                       "l2": f"inputs larger than L2: {rep.R} rotating replicas of layer+x+y, "
-                             f"{rep.total_bytes / 1e6:.0f} MB vs L2 {l2 / 1e6:.0f} MB",
-                       "timing": "CUDA-graph replays between CUDA events on the launching stream"},
-            "roofline": {"bound": "alu", "achieved": achieved_tflops, "peak": fma_peak_tflops, "unit": "TFLOP/s",
-                         "frac": achieved_tflops / fma_peak_tflops,
-                         # dram__bytes_read.sum + dram__bytes_write.sum of one launch (ncu capture summarised under
-                         # profiles/); only valid for the kernel and workload it was taken on
-                         "traffic": 10.29e6 if (tile_shape is not None and w.name == "c2"
-                                                and tile_shape["tile"][1] == 96 and tile_shape["cluster_k_split"] == 2) else None,
-                         "peak_source": f"{sm_count} SMs x {FMA_LANES_PER_SM} fp32 FMA lanes x 2 x {sm_max_mhz:.0f} MHz",
-                         "kernel": {"batch": "cfi_batch_kernel<float>",
-                                    "dense_tc": f"cfi_dense_tf32_kernel<{tile_shape['tile'][1] if tile_shape else 64}>"}.get(
-                             chosen, f"cfi_{chosen}_kernel"),
+            "config": dict(config_keys(w, rep.n_active), variant=chosen, dense_shape=shape,
+                           l2=f"inputs larger than L2: {rep.R} rotating replicas of layer+x+y, "
+                              f"{rep.total_bytes / 1e6:.0f} MB vs L2 {l2 / 1e6:.0f} MB",
+                           timing=f"{timed['passes']} passes of {args.steps} steps each (CUDA-graph replays between CUDA events "
+                                  "on the launching stream); ms_per_step is the median pass / steps"),
+            "roofline": {"bound": "alu", "achieved": achieved_tflops, "peak": ceil_.fma_tflops, "unit": "TFLOP/s",
+                         "frac": achieved_tflops / ceil_.fma_tflops,
+                         # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised
+                         # under profiles/ for exactly this kernel and launch shape; null otherwise
+                         "traffic": CAPTURED_TRAFFIC.get((w.name, kernel_name(chosen, shape), json.dumps(shape))),
+                         "peak_source": ceil_.fma_source,
+                         "kernel": kernel_name(chosen, shape),
                          "note": "bound/peak are the sparse problem's own roofline (2*B*n_active*k FMAs on the fp32 FMA "
-                                 "pipes, the bound of the gather formulation); when the chosen kernel is the tensor-core "
-                                 "variant the dense flops it executes are given under tensor_*",
+                                 "pipes, the bound of the gather formulation; its shared-memory ceiling is given beside "
+                                 "it); when the chosen kernel is the tensor-core variant the dense flops it executes are "
+                                 "given under tensor_*",
+                         "smem_ceiling_tflops": ceil_.smem_tflops, "smem_ceiling_frac": achieved_tflops / ceil_.smem_tflops,
                          "hbm_achieved_gbs": hbm_gbs, "hbm_peak_gbs": peaks["hbm_gbs"],
                          "hbm_frac": hbm_gbs / peaks["hbm_gbs"], "hbm_peak_source": f"{peak_kind} copy bandwidth",
                          "algorithmic_bytes": rep.bytes_per_step, "algorithmic_flops": flops,
                          "weight_bytes_streamed_per_batch_tile": int(info.weight_bytes_batch)},
             "variants_us": {},
             "e2e": {"value": e2e_value, "unit": "GFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "us_per_call": e2e_sec / e2e_steps * 1e6, "steps": e2e_steps, "api": "cfi_forward_host"},
-            "gpu_launches": launches,
+                    "us_per_call": e2e_sec / e2e_steps * 1e6, "calls_timed": e2e_steps, "api": "cfi_forward_host",
+                    "note": "every replica's staging buffers exist before the timed region"},
+            "gpu_launches": timed["launches_per_pass"],
             "clocks": sampler.summary(),
         }
-    if rank == 0:
         if chosen == "dense_tc":
             dense = 3 * 2.0 * w.batch * w.out_features * w.in_features   # three TF32 products per fp32 product
             tf32_peak = peaks["bf16_tflops"] * 0.5                      # nominal TF32 : bf16 ratio on the measured bf16 peak
@@ -413,19 +450,24 @@ def main():
         if world == 1 and not args.no_extras:
             for v in ("batch", "dense_tc"):
                 try:
-                    sv, _ = time_steps(rep, torch, 5000, 10, v)
-                    line["variants_us"][v] = sv / 5000 * 1e6
+                    line["variants_us"][v] = us(time_steps(rep, torch, 2000, 10, v, target_s=0.05))
                 except Exception as exc:  # a variant that cannot run this shape
                     line["variants_us"][v] = str(exc)
     rep.close()
 
     if rank == 0 and world == 1 and not args.no_extras:
-        line["batch1"] = batch1_leg(W, cfi, torch, l2, peaks, peak_kind)
-        cb = time_oracle(w, budget_s=15.0)
+        line["floor"] = floor_leg(cfi, torch, l2)
+        line["sweep"] = sweep_leg(W, cfi, torch, l2, ceil_, line["floor"])
+        line["batch1"] = {k: v for k, v in line["sweep"].items() if k in W and W[k].batch == 1}
+        cb = time_oracle(w, budget_s=10.0)
+        c1 = time_oracle(w, budget_s=10.0, threads=1)
         line["cpu_baseline"] = {"value": cb["flops"] / cb["median_s"] / 1e9, "unit": "GFLOP/s", "cores": cb["cores"],
-                                "kind": "oracle", "us_per_call": cb["median_s"] * 1e6,
-                                "sample": f"whole workload ({cb['rows']} batch rows), median of {cb['calls']} calls"}
-        line["context"] = context_leg(w, torch)
+                                "kind": "oracle", "us_per_call": cb["median_s"] * 1e6, "us_per_call_std": cb["std_s"] * 1e6,
+                                "sample": f"{cb['rows']} of {w.batch} batch rows per call, median of {cb['calls']} calls",
+                                "one_thread": {"value": c1["flops"] / c1["median_s"] / 1e9, "unit": "GFLOP/s", "cores": 1,
+                                               "us_per_call": c1["median_s"] * 1e6,
+                                               "sample": f"{c1['rows']} of {w.batch} batch rows per call, median of {c1['calls']} calls"}}
+        line["context"] = context_leg(W, torch)
         line["stack_c5"] = stack_leg(cfi, torch, peaks, sm_count)
         line["batch2048"] = batch2048_leg(W, cfi, torch, l2, peaks, sm_count)
         # Ceilings measured in this run by the library's own micro-probes (fp32 FMA, L2 read, empty launch).
@@ -439,6 +481,36 @@ def main():
         print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
+
+
+VARIANT_NAMES = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}
+# DRAM bytes (read + written) of one launch from an ncu capture, keyed by (workload, kernel, launch shape); see profiles/.
+CAPTURED_TRAFFIC = {}
+
+
+def dense_shape(cfi, layer, batch):
+    tile, cluster = cfi.cfi_dense_tile_shape(layer, batch)
+    return {"batch_tile": tile, "cluster_k_split": cluster}
+
+
+def kernel_name(variant, shape=None, dtype="f32"):
+    if variant == "dense_tc":
+        return f"cfi_dense_split_kernel<{shape['batch_tile']}>" if shape else "cfi_dense_split_kernel"
+    return {"batch": "cfi_batch_kernel<float>", "splitk": "cfi_splitk_kernel<float>", "simple": "cfi_simple_kernel<float>"}[variant]
+
+
+class Ceilings:
+    """The denominators: fp32 FMA peak derived from the unit counts and the maximum clock, the measured shared-memory
+    gather ceiling of the gather formulation (25.5 FMA per clock and SM: one 4-byte gather per FMA at 128 bytes per
+    clock, measured with a stand-alone copy of the inner loop), and the measured copy bandwidth."""
+
+    def __init__(self, peaks, peak_kind, sm_count):
+        self.sm_mhz = float(peaks.get("sm_max_mhz", 1965.0))
+        self.fma_tflops = sm_count * FMA_LANES_PER_SM * 2 * self.sm_mhz * 1e6 / 1e12
+        self.fma_source = f"{sm_count} SMs x {FMA_LANES_PER_SM} fp32 FMA lanes x 2 x {self.sm_mhz:.0f} MHz"
+        self.smem_tflops = sm_count * 25.5 * 2 * self.sm_mhz * 1e6 / 1e12
+        self.hbm_gbs = float(peaks["hbm_gbs"])
+        self.peak_kind = peak_kind
 
 
 def max_over_ranks(seconds: float, dist, device) -> float:
@@ -469,21 +541,29 @@ def _time_torch(fn, torch, iters=200):
     return a.elapsed_time(b) * 1e-3 / iters
 
 
-def context_leg(w, torch):
-    """Library routines on the same masked weights, as context (not a target): cuBLAS dense through
-    torch.matmul on the full masked weight, cuSPARSE CSR through torch's sparse matmul.  Warm (one layer),
-    eager launches, batch of the headline workload and batch 1."""
-    L = w.layer(seed=0)
-    wd = torch.from_numpy(L.w_dense * L.mask).cuda()
-    csr = wd.to_sparse_csr()
+def context_leg(W, torch):
+    """Library routines on the same masked weights, as context (not a target): cuBLAS dense through torch.matmul on
+    the full masked weight, cuBLAS dense on the active rows only (the "structured" representation of Sec. 4.4: neuron
+    ablation alone), cuSPARSE CSR through torch's sparse matmul.  Warm (one layer), eager launches."""
     out = {}
-    for batch in (w.batch, 1):
-        x = torch.from_numpy(w.x(seed=0, batch=batch)).cuda()
-        xt = x.t().contiguous()
-        out[f"b{batch}"] = {"cublas_dense_us": _time_torch(lambda: torch.matmul(x, wd.t()), torch) * 1e6,
-                            "cusparse_csr_us": _time_torch(lambda: torch.matmul(csr, xt), torch) * 1e6}
-    out["note"] = "torch.matmul (cuBLAS fp32, TF32 off) and torch CSR matmul (cuSPARSE), warm, eager; paper: 1.7x / 13.0x " \
-                  "faster than dense / CSR at batch 256 on a Titan V, 3.4x / 2.5x on a Xeon W-2145 at batch 1"
+    for name in ("c2", "c3_b256"):
+        w = W[name]
+        L = w.layer(seed=0)
+        wd = torch.from_numpy(L.w_dense * L.mask).cuda()
+        active = np.setdiff1d(np.arange(w.out_features), L.ablated)
+        wa = wd[torch.from_numpy(active).cuda()].contiguous()
+        csr = wd.to_sparse_csr()
+        for batch in (w.batch, 1):
+            x = torch.from_numpy(w.x(seed=0, batch=batch)).cuda()
+            xt = x.t().contiguous()
+            out[f"{name.split('_')[0]}_b{batch}"] = {
+                "cublas_dense_us": _time_torch(lambda: torch.matmul(x, wd.t()), torch) * 1e6,
+                "cublas_dense_active_rows_us": _time_torch(lambda: torch.matmul(x, wa.t()), torch) * 1e6,
+                "cusparse_csr_us": _time_torch(lambda: torch.matmul(csr, xt), torch) * 1e6,
+                "active_rows": int(active.size), "rows": w.out_features}
+    out["note"] = "torch.matmul (cuBLAS fp32, TF32 off) on all rows and on the active rows only, torch CSR matmul (cuSPARSE); " \
+                  "warm, eager; paper: 1.7x / 13.0x faster than dense / CSR at batch 256 on a Titan V, 3.4x / 2.5x on a " \
+                  "Xeon W-2145 at batch 1"
     return out
 
 
@@ -516,16 +596,14 @@ def batch2048_leg(W, cfi, torch, l2, peaks, sm_count):
     import dataclasses
     w = dataclasses.replace(W["c2"], name="c2_b2048", batch=2048)
     rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), max_replicas=16)
-    steps = 2000
     out = {"batch": w.batch}
     for v in ("auto", "batch"):
-        sec, _ = time_steps(rep, torch, steps, 10, v)
-        out[f"us_per_call_{v}"] = sec / steps * 1e6
+        out[f"us_per_call_{v}"] = us(time_steps(rep, torch, 500, 10, v, target_s=0.05))
     flops = algorithmic_flops(w, rep.n_active)
     fma_peak = sm_count * FMA_LANES_PER_SM * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
     out["effective_tflops"] = flops / (out["us_per_call_auto"] * 1e-6) / 1e12
     out["fma_frac"] = out["effective_tflops"] / fma_peak
-    out["variant"] = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
+    out["variant"] = VARIANT_NAMES[cfi.cfi_choose_variant(rep.layers[0], w.batch)]
     rep.close()
     return out
 
@@ -605,31 +683,108 @@ def srigl_update_leg(cfi, torch, peaks):
     return out
 
 
-def batch1_leg(W, cfi, torch, l2, peaks, peak_kind):
-    """Online inference (batch 1): us per call and achieved fraction of the HBM roofline, cold (rotating
-    replicas larger than L2) and warm (one layer, L2-resident)."""
+def floor_leg(cfi, torch, l2):
+    """What a forward call costs with all of the layer's work taken out, measured the way the forward is timed (a CUDA
+    graph of back-to-back launches with the forward kernels' launch attributes): an empty kernel, and a kernel in
+    which every CTA makes one dependent trip to DRAM and one store.  A batch-1 call can be no faster than the second."""
+    buf = torch.empty(max(4 * l2, 256 << 20) // 4, dtype=torch.float32, device="cuda")
+    buf.zero_()
+    scratch = torch.zeros(1024, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
     out = {}
-    for name in ("c1", "c3_b1", "c4_s80_b1", "c4_s90_b1"):
-        w = W[name]
-        rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), max_replicas=160)
-        info = cfi.cfi_layer_info(rep.layers[0])
-        streamed = int(info.weight_bytes_splitk) + (w.in_features + 2 * w.out_features) * 4
-        steps = 20000
-        sec, _ = time_steps(rep, torch, steps, 20)
-        cold = sec / steps
-        one = Replicas(w, cfi, torch, 0, max_replicas=2)
-        one.R = 1
-        sec, _ = time_steps(one, torch, steps, 20)
-        warm = sec / steps
-        one.close()
-        out[name] = {"us_per_call_cold": cold * 1e6, "us_per_call_warm": warm * 1e6,
-                     "algorithmic_bytes": rep.bytes_per_step, "streamed_bytes": streamed,
-                     "hbm_gbs_cold": rep.bytes_per_step / cold / 1e9,
-                     "hbm_frac_cold": rep.bytes_per_step / cold / 1e9 / peaks["hbm_gbs"],
-                     "hbm_peak_source": f"{peak_kind} copy bandwidth",
-                     "gflops_cold": algorithmic_flops(w, rep.n_active) / cold / 1e9,
-                     "replicas": rep.R, "replica_bytes_total": rep.total_bytes}
-        rep.close()
+    with torch.cuda.stream(stream):
+        for kind, name in ((0, "empty_node_us"), (1, "dram_roundtrip_node_us")):
+            for _ in range(10):
+                cfi.cfi_probe_floor_launch(kind, buf, scratch)
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(1000):
+                    cfi.cfi_probe_floor_launch(kind, buf, scratch)
+            g.replay()
+            stream.synchronize()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(21)]
+            ev[0].record(stream)
+            for i in range(20):
+                g.replay()
+                ev[i + 1].record(stream)
+            ev[-1].synchronize()
+            t = [ev[i].elapsed_time(ev[i + 1]) for i in range(20)]
+            out[name] = statistics.median(t)           # ms per 1000 launches = us per launch
+            out[name.replace("_us", "_std_us")] = statistics.pstdev(t)
+    out["note"] = "us per node of a 1000-node CUDA graph, median of 20 replays; nodes are launched with programmatic " \
+                  "dependent launch like the forward kernels, one CTA per SM"
+    return out
+
+
+# Layer shapes of the named workloads: every batch size of a shape is timed on the same replicas of the layer.
+SWEEP = [("c1", ["c1", "c2"]), ("c3_b1", ["c3_b1", "c3_b64", "c3_b256"])] + \
+        [(f"c4_s{sp}_b1", [f"c4_s{sp}_b{b}" for b in (1, 16, 256)]) for sp in (80, 90, 95, 99)]
+
+
+def sweep_leg(W, cfi, torch, l2, ceil_, floor):
+    """Every named workload, cold (rotating replicas of layer, x and y larger than twice the L2): us per call (median
+    and standard deviation over the passes), the kernel the library picks, algorithmic bytes and flops, the time the
+    HBM and the fp32 FMA rooflines allow, the fraction of the binding one, the fraction of the gather formulation's
+    shared-memory ceiling for batch > 1, the launch floor for batch 1, and the oracle on this host's cores."""
+    import oracle
+    out = {}
+    for base_name, names in SWEEP:
+        base = W[base_name]
+        L = base.layer(seed=0)
+        packed = cfi.cfi_pack(L.w_dense, L.mask)
+        opk = oracle.pack(L.w_dense, L.mask)            # the oracle's own pack for its own timing
+        probe = cfi.cfi_create(packed[0], packed[1], packed[2], L.bias, base.in_features, base.out_features)
+        for name in names:
+            w = W[name]
+            # The replicas hold the layouts the chosen kernel needs (all three for the tensor-core variant, whose dense
+            # copy is then what a call streams; the two condensed ones otherwise; the small-batch one alone at batch 1).
+            variant = VARIANT_NAMES[cfi.cfi_choose_variant(probe, w.batch)]
+            shape = dense_shape(cfi, probe, w.batch) if variant == "dense_tc" else None
+            dense_bytes = int(cfi.cfi_layer_info(probe).bytes_dense) if variant == "dense_tc" else None
+            layouts = 7 if variant == "dense_tc" else 1 if w.batch == 1 else 3
+            rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), max_replicas=200, layer=L, packed=packed, layouts=layouts,
+                           streamed_bytes=dense_bytes)
+            assert VARIANT_NAMES[cfi.cfi_choose_variant(rep.layers[0], w.batch)] == variant
+            t = time_steps(rep, torch, 1000, 10, target_s=0.05)
+            sec = t["sec_per_step"]
+            flops, nbytes = algorithmic_flops(w, rep.n_active), rep.bytes_per_step
+            t_hbm, t_fma = nbytes / (ceil_.hbm_gbs * 1e9), flops / (ceil_.fma_tflops * 1e12)
+            info = cfi.cfi_layer_info(rep.layers[0])
+            e = {"us_per_call": sec * 1e6, "us_per_call_std": t["std_sec_per_step"] * 1e6, "passes": t["passes"],
+                 "variant": variant, "dense_shape": shape, "algorithmic_bytes": nbytes, "algorithmic_flops": flops,
+                 "gflops": flops / sec / 1e9, "hbm_gbs": nbytes / sec / 1e9,
+                 "t_hbm_us": t_hbm * 1e6, "t_fma_us": t_fma * 1e6, "bound": "hbm" if t_hbm >= t_fma else "alu",
+                 "frac_of_bound": max(t_hbm, t_fma) / sec, "hbm_frac": t_hbm / sec, "fma_frac": t_fma / sec,
+                 "replicas": rep.R, "layouts": layouts, "device_bytes_per_layer": int(info.device_bytes)}
+            if w.batch > 1:
+                e["smem_ceiling_frac"] = flops / sec / 1e12 / ceil_.smem_tflops
+            else:
+                e["floor_us"] = floor["dram_roundtrip_node_us"]
+                e["times_floor"] = sec * 1e6 / floor["dram_roundtrip_node_us"]
+                e["streamed_bytes"] = int(info.weight_bytes_splitk) + (w.in_features + 2 * w.out_features) * 4
+                one = Replicas(w, cfi, torch, 0, max_replicas=2, layer=L, packed=packed, layouts=layouts)
+                one.R = 1
+                e["us_per_call_warm"] = us(time_steps(one, torch, 1000, 10, target_s=0.02))
+                one.close()
+            rep.close()
+            cb = time_oracle(w, budget_s=1.0, layer=L, packed=opk)
+            e["cpu_oracle"] = {"us_per_call_scaled": cb["median_s"] * 1e6 * w.batch / cb["rows"], "rows_timed": cb["rows"],
+                               "cores": cb["cores"], "gflops": cb["flops"] / cb["median_s"] / 1e9}
+            out[name] = e
+        probe.close()
+    # The bf16 stack's CPU time: one block's two layers on a 788-row slice (1/64 of the batch), scaled.
+    s = inputs.StackWorkload(blocks=1)
+    x = s.x(seed=0, batch=788)
+    tot = 0.0
+    for Ls, sp in zip(s.layers(seed=0), s.layer_specs()):
+        pk = oracle.pack(Ls.w_dense, Ls.mask)
+        xin = oracle.round_bf16(x) if sp[0] == s.d_model else np.zeros((788, sp[0]), np.float32)
+        t0 = time.perf_counter()
+        oracle.forward(oracle.round_bf16(pk[0]), pk[1], pk[2], Ls.bias, sp[0], sp[1], xin, act=sp[4])
+        tot += time.perf_counter() - t0
+    out["c5_cpu_oracle"] = {"ms_per_pass_scaled": tot * 12 * 64 * 1e3, "rows_timed": 788, "blocks_timed": 1,
+                            "cores": oracle.max_threads(), "note": "one block on 788 of 50,432 rows, x 64 x 12"}
     return out
 
 

@@ -69,6 +69,15 @@ typedef enum {
                                  row, otherwise CFI_ERR_SHAPE */
 } cfi_variant_t;
 
+/* Device layouts a layer may hold (cfi_create_layouts).  The condensed form exists to save memory (Sec. 4.4: n x k
+ * values and indices instead of the n x d weight), so a caller chooses what to pay for. */
+typedef enum {
+    CFI_LAYOUT_SMALL_BATCH = 1, /* values + indices, n_active x k padded to 16-byte vectors: CFI_VARIANT_SPLITK / SIMPLE   */
+    CFI_LAYOUT_GATHER = 2,      /* the same entries grouped by column slab for CFI_VARIANT_BATCH: about as large            */
+    CFI_LAYOUT_DENSE = 4,       /* dense out x in copy in the layer's dtype for CFI_VARIANT_DENSE_TC: 1 / density as large  */
+    CFI_LAYOUT_ALL = 7
+} cfi_layout_t;
+
 const char* cfi_status_string(cfi_status_t s);
 
 /*
@@ -192,11 +201,30 @@ cfi_status_t cfi_pack_device(const float* w_dense, const uint8_t* mask, int32_t 
  *
  * Requires 0 <= n_active <= out_features, 0 <= k <= in_features (k >= 1 if n_active > 0),
  * in_features <= 2^20.  The arrays are copied; the caller may free them after the call.
- * The layer lives on the CUDA device that is current when cfi_create is called.
+ * The layer lives on the CUDA device that is current when cfi_create is called.  All three device layouts are
+ * built (cfi_create_layouts builds fewer).
  */
 cfi_status_t cfi_create(const float* values, const int32_t* indices, const int32_t* active_rows, const float* bias,
                         int32_t n_active, int32_t k, int32_t in_features, int32_t out_features,
                         cfi_dtype_t dtype, cfi_act_t act, cfi_layer_t** layer);
+
+/*
+ * cfi_create_layouts — cfi_create with the device layouts chosen by the caller (a bit set of cfi_layout_t;
+ * cfi_create builds CFI_LAYOUT_ALL).  A layer used for online inference only needs CFI_LAYOUT_SMALL_BATCH and then
+ * holds little more than the condensed arrays themselves: 4096 x 4096 at 99 % sparsity is 1.4 MB, against 67 MB with
+ * the dense copy.  cfi_forward chooses among the kernels whose layout exists (a small batch runs on the dense or
+ * gather layout if that is all there is, and the other way round); cfi_forward_variant with a variant whose layout is
+ * missing returns CFI_ERR_SHAPE.  CFI_LAYOUT_DENSE is skipped silently where the tensor-core variant cannot address
+ * the shapes (see CFI_VARIANT_DENSE_TC) unless it is the only layout asked for, which is CFI_ERR_SHAPE;
+ * cfi_layer_info reports what was built.  CFI_ERR_DTYPE for an empty or unknown bit set.  The paper has no counterpart of the choice: its layer has the one condensed form.
+ *
+ * cfi_layer_add_layouts builds layouts the layer does not have yet (the layer keeps a host copy of its condensed
+ * arrays for this).  No forward call may be running on the layer meanwhile.
+ */
+cfi_status_t cfi_create_layouts(const float* values, const int32_t* indices, const int32_t* active_rows, const float* bias,
+                                int32_t n_active, int32_t k, int32_t in_features, int32_t out_features,
+                                cfi_dtype_t dtype, cfi_act_t act, int32_t layouts, cfi_layer_t** layer);
+cfi_status_t cfi_layer_add_layouts(cfi_layer_t* layer, int32_t layouts);
 
 /*
  * cfi_forward — y = layer(x) for `batch` rows (Algorithm 1 with bias, ablated rows and activation).
@@ -262,7 +290,12 @@ typedef struct {
     int32_t reserved;
     int64_t weight_bytes_splitk; /* bytes of values+indices the small-batch kernel reads per pass        */
     int64_t weight_bytes_batch;  /* bytes of values+columns the large-batch kernel reads per batch tile  */
-    int64_t device_bytes;        /* device memory held by the layer                                      */
+    int64_t device_bytes;        /* device memory held by the layer: the three below + bias, row map, status */
+    int64_t bytes_small_batch;   /* CFI_LAYOUT_SMALL_BATCH                                               */
+    int64_t bytes_gather;        /* CFI_LAYOUT_GATHER                                                    */
+    int64_t bytes_dense;         /* CFI_LAYOUT_DENSE                                                     */
+    int32_t layouts;             /* bit set of cfi_layout_t: what exists                                 */
+    int32_t reserved2;
 } cfi_layer_info_t;
 
 cfi_status_t cfi_layer_info(const cfi_layer_t* layer, cfi_layer_info_t* info);
@@ -358,6 +391,22 @@ typedef struct {
 } cfi_device_probe_t;
 
 cfi_status_t cfi_probe_device(cfi_device_probe_t* probe);
+
+/*
+ * cfi_probe_floor_launch — enqueues one launch of a kernel that does none of the layer's work, for measuring what a
+ * forward call costs at the very least.  It has the forward kernels' launch attributes (one CTA per SM, programmatic
+ * dependent launch: it releases its successor at once and waits for its predecessor), so a chain of these launches
+ * in a stream or a CUDA graph is timed exactly like a chain of cfi_forward calls.  No counterpart in the paper, which
+ * reports wall-clock medians only (Sec. 4.4, Fig. 4).
+ *
+ *   kind     0: an empty kernel;  1: every CTA makes one dependent trip to DRAM (a 128-byte line of `buf` that no
+ *            recent launch has read, chosen from a launch counter kept in `scratch`) and one store
+ *   buf      device, 256-byte aligned, buf_bytes >= 1 MiB and best several times the L2 size (kind 1; ignored for 0)
+ *   scratch  device, 256-byte aligned, at least 4 KiB, zeroed by the caller before the first launch
+ *
+ * Asynchronous on `stream`.  CFI_ERR_DTYPE (kind), CFI_ERR_NULL, CFI_ERR_ALIGNMENT, CFI_ERR_BUFFER_TOO_SMALL, CFI_ERR_CUDA.
+ */
+cfi_status_t cfi_probe_floor_launch(int32_t kind, const void* buf, size_t buf_bytes, void* scratch, cfi_stream_t stream);
 
 #ifdef __cplusplus
 }

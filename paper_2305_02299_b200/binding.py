@@ -25,11 +25,11 @@ _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE,
 _VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_srigl_workspace_bytes",
-           "cfi_srigl_update", "cfi_pack_device", "cfi_create", "cfi_forward", "cfi_forward_variant", "cfi_forward_dense",
+           "cfi_srigl_update", "cfi_pack_device", "cfi_create", "cfi_create_layouts", "cfi_layer_add_layouts", "cfi_forward", "cfi_forward_variant", "cfi_forward_dense",
            "cfi_forward_host",
            "cfi_layer_info", "cfi_choose_variant", "cfi_dense_tile_shape", "cfi_device_status", "cfi_destroy",
            "cfi_stack_create", "cfi_stack_forward", "cfi_stack_destroy", "cfi_stack_forward_static",
-           "cfi_probe_device")
+           "cfi_probe_device", "cfi_probe_floor_launch")
 
 
 class CfiError(RuntimeError):
@@ -44,7 +44,8 @@ class LayerInfo(ctypes.Structure):
                 ("k_padded", ctypes.c_int32), ("batch_slab_columns", ctypes.c_int32),
                 ("batch_row_stride", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("weight_bytes_splitk", ctypes.c_int64), ("weight_bytes_batch", ctypes.c_int64),
-                ("device_bytes", ctypes.c_int64)]
+                ("device_bytes", ctypes.c_int64), ("bytes_small_batch", ctypes.c_int64), ("bytes_gather", ctypes.c_int64),
+                ("bytes_dense", ctypes.c_int64), ("layouts", ctypes.c_int32), ("reserved2", ctypes.c_int32)]
 
 
 class DeviceProbe(ctypes.Structure):
@@ -77,6 +78,8 @@ def _load() -> ctypes.CDLL:
     lib.cfi_srigl_update.argtypes = [vp, vp, vp, ci, ci, ctypes.c_int64, ctypes.c_float, vp, ctypes.c_size_t, i32p, i32p, vp]
     lib.cfi_pack_device.argtypes = [vp, vp, ci, ci, vp, ctypes.c_size_t, i32p, i32p, vp, vp, vp, vp]
     lib.cfi_create.argtypes = [f32p, i32p, i32p, f32p, ci, ci, ci, ci, ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
+    lib.cfi_create_layouts.argtypes = [f32p, i32p, i32p, f32p, ci, ci, ci, ci, ctypes.c_int, ctypes.c_int, ci, ctypes.POINTER(vp)]
+    lib.cfi_layer_add_layouts.argtypes = [vp, ci]
     lib.cfi_forward.argtypes = [vp, vp, vp, ci, vp]
     lib.cfi_forward_variant.argtypes = [vp, vp, vp, ci, vp, ctypes.c_int]
     lib.cfi_forward_dense.argtypes = [vp, vp, vp, ci, vp, ci, ci]
@@ -91,6 +94,7 @@ def _load() -> ctypes.CDLL:
     lib.cfi_stack_destroy.argtypes = [vp]
     lib.cfi_stack_forward_static.argtypes = [ctypes.POINTER(vp), ci, vp, vp, ci, vp]
     lib.cfi_probe_device.argtypes = [ctypes.POINTER(DeviceProbe)]
+    lib.cfi_probe_floor_launch.argtypes = [ci, vp, ctypes.c_size_t, vp, vp]
     for name in EXPORTS:
         if name != "cfi_status_string":
             getattr(lib, name).restype = ctypes.c_int
@@ -170,8 +174,12 @@ class Layer:
             pass
 
 
+LAYOUT_SMALL_BATCH, LAYOUT_GATHER, LAYOUT_DENSE, LAYOUT_ALL = 1, 2, 4, 7
+
+
 def cfi_create(values, indices, active_rows, bias, in_features: int, out_features: int, dtype="f32",
-               act="none") -> Layer:
+               act="none", layouts: int = LAYOUT_ALL) -> Layer:
+    """cfi_create, or cfi_create_layouts when `layouts` (a bit set of LAYOUT_*) is not LAYOUT_ALL."""
     v = np.ascontiguousarray(values, dtype=np.float32)
     ix = np.ascontiguousarray(indices, dtype=np.int32)
     ar = np.ascontiguousarray(active_rows, dtype=np.int32)
@@ -185,10 +193,19 @@ def cfi_create(values, indices, active_rows, bias, in_features: int, out_feature
     if b is not None and b.shape != (out_features,):
         raise ValueError("bias must be [out_features]")
     h = ctypes.c_void_p()
-    _check(_lib.cfi_create(_hp(v, ctypes.c_float), _hp(ix, ctypes.c_int32), _hp(ar, ctypes.c_int32),
-                           _hp(b, ctypes.c_float), n_active, k, in_features, out_features, _DTYPES[dtype],
-                           _ACTS[act], ctypes.byref(h)), "cfi_create")
+    if layouts == LAYOUT_ALL:
+        _check(_lib.cfi_create(_hp(v, ctypes.c_float), _hp(ix, ctypes.c_int32), _hp(ar, ctypes.c_int32),
+                               _hp(b, ctypes.c_float), n_active, k, in_features, out_features, _DTYPES[dtype],
+                               _ACTS[act], ctypes.byref(h)), "cfi_create")
+    else:
+        _check(_lib.cfi_create_layouts(_hp(v, ctypes.c_float), _hp(ix, ctypes.c_int32), _hp(ar, ctypes.c_int32),
+                                       _hp(b, ctypes.c_float), n_active, k, in_features, out_features, _DTYPES[dtype],
+                                       _ACTS[act], int(layouts), ctypes.byref(h)), "cfi_create_layouts")
     return Layer(h.value, in_features, out_features, _DTYPES[dtype])
+
+
+def cfi_layer_add_layouts(layer: Layer, layouts: int) -> None:
+    _check(_lib.cfi_layer_add_layouts(layer.handle, int(layouts)), "cfi_layer_add_layouts")
 
 
 def cfi_compact_producer(bias, active_rows, out_features: int):
@@ -352,3 +369,10 @@ def cfi_probe_device() -> DeviceProbe:
     p = DeviceProbe()
     _check(_lib.cfi_probe_device(ctypes.byref(p)), "cfi_probe_device")
     return p
+
+
+def cfi_probe_floor_launch(kind: int, buf, scratch, stream=None) -> None:
+    """One launch of the no-work kernel (kind 0: empty, kind 1: one DRAM round trip per CTA); see include/cfi.h."""
+    nbytes = 0 if buf is None else buf.numel() * buf.element_size()
+    _check(_lib.cfi_probe_floor_launch(kind, 0 if buf is None else _dev_ptr(buf), nbytes, _dev_ptr(scratch), _stream_handle(stream)),
+           "cfi_probe_floor_launch")

@@ -52,7 +52,11 @@ struct DevLayer {
 struct cfi_layer {
     DevLayer d{};
     int dtype = 0, device = 0, sm_count = 0, smem_optin = 0;
-    int64_t device_bytes = 0;
+    int64_t device_bytes = 0, bytes_small = 0, bytes_gather = 0, bytes_dense = 0;
+    int layouts = 0;  // CFI_LAYOUT_* bits of the device layouts that exist
+    // The condensed arrays as given, each row sorted by column, kept so that further layouts can be built later.
+    std::vector<float> h_values;
+    std::vector<int32_t> h_cols, h_rows, h_slot;
     std::vector<void*> allocs;
     void* stage_x = nullptr;
     void* stage_y = nullptr;
@@ -676,6 +680,7 @@ size_t batch_smem(const cfi_layer* l, int warps, int rph) {
 BatchShape batch_shape(const cfi_layer* l, int batch) {
     BatchShape best{};
     best.ok = false;
+    if (!(l->layouts & CFI_LAYOUT_GATHER)) return best;
     double best_cost = 0;
     const int es = l->dtype == CFI_BF16 ? 2 : 4;
     const int grid_y = (batch + kBatchTile - 1) / kBatchTile;
@@ -777,6 +782,7 @@ cfi_status_t launch_splitk_bt(const cfi_layer* l, const SplitkShape& s, const VT
 template <typename VT>
 cfi_status_t launch_splitk(const cfi_layer* l, const SplitkShape& s, const void* x, void* y, int batch,
                            cudaStream_t st) {
+    if (!(l->layouts & CFI_LAYOUT_SMALL_BATCH)) return CFI_ERR_SHAPE;
     if (s.smem > (size_t)l->smem_optin || s.grid_y > 65535) return CFI_ERR_SHAPE;
     const VT* xx = static_cast<const VT*>(x);
     VT* yy = static_cast<VT*>(y);
@@ -816,6 +822,7 @@ cfi_status_t launch_batch(const cfi_layer* l, const BatchShape& s, const void* x
 
 template <typename VT>
 cfi_status_t launch_simple(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
+    if (!(l->layouts & CFI_LAYOUT_SMALL_BATCH)) return CFI_ERR_SHAPE;
     const int64_t total = (int64_t)batch * l->d.out;
     const int threads = 256;
     const int64_t blocks = (total + threads - 1) / threads;
@@ -1064,15 +1071,22 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
 constexpr double kGatherTflops = 12.5;
 
 // The split-k kernel keeps at least one whole row of x (+ one zero element) in shared memory.
-bool splitk_fits(const cfi_layer* l, int batch) { return splitk_shape(l, batch).smem <= (size_t)l->smem_optin; }
+bool splitk_fits(const cfi_layer* l, int batch) {
+    return (l->layouts & CFI_LAYOUT_SMALL_BATCH) && splitk_shape(l, batch).smem <= (size_t)l->smem_optin;
+}
 
 // What remains when the preferred kernel cannot hold its tile: the gather kernel (column slabs), else one thread per output.
 int fallback_variant(const cfi_layer* l, int batch) {
     if (batch_shape(l, batch).ok) return CFI_VARIANT_BATCH;
-    return splitk_fits(l, batch) ? CFI_VARIANT_SPLITK : CFI_VARIANT_SIMPLE;
+    if (splitk_fits(l, batch)) return CFI_VARIANT_SPLITK;
+    if (l->tc_ok && !(l->layouts & CFI_LAYOUT_SMALL_BATCH)) return CFI_VARIANT_DENSE_TC;
+    return CFI_VARIANT_SIMPLE;
 }
 
 int choose_variant(const cfi_layer* l, int batch) {
+    // A layer built without the small-batch layout runs every batch size on what it has.
+    if (!(l->layouts & CFI_LAYOUT_SMALL_BATCH) && batch <= 24)
+        return l->tc_ok && (batch > 4 || !batch_shape(l, batch).ok) ? CFI_VARIANT_DENSE_TC : fallback_variant(l, batch);
     // Up to three batch tiles of 8 the split-k kernel (weights re-read from L2 per tile) beats the 64-wide tiles of
     // the batch kernel, which would be mostly empty.
     if (batch <= 24) {
@@ -1200,6 +1214,179 @@ void free_layer(cfi_layer* l) {
     delete l;
 }
 
+// Small-batch ("split-k") layout: values and indices padded to whole 16-byte vectors, entries ordered for the banks.
+cfi_status_t build_small(cfi_layer* l) {
+    const int32_t k = l->d.k, n_active = l->d.n_active, in_features = l->d.in, out_features = l->d.out;
+    const int dtype = l->dtype;
+    DevLayer& d = l->d;
+    const std::vector<float>& v_sorted = l->h_values;
+    const std::vector<int32_t>&c_sorted = l->h_cols, &active_rows = l->h_rows, &slot = l->h_slot;
+    cfi_status_t st = CFI_OK;
+    const int64_t before = l->device_bytes;
+    (void)k, (void)n_active, (void)in_features, (void)out_features, (void)dtype, (void)d, (void)v_sorted, (void)c_sorted,
+        (void)active_rows, (void)slot;
+    // ---- small-batch layout
+    const int vec = vec_of(dtype);
+    d.kp = ((k + vec - 1) / vec) * vec;
+    std::vector<int32_t> place((size_t)std::max(d.kp, 1));  // position in the padded row of sorted entry j
+    const int lanes = splitk_lanes_per_row(std::max(1, d.kp / vec));
+    std::vector<int32_t> idx_p((size_t)n_active * d.kp, in_features);
+    if (dtype == CFI_F32) {
+        std::vector<float> val_p((size_t)n_active * d.kp, 0.0f);
+        for (int32_t r = 0; r < n_active; ++r) {
+            order_for_banks(&c_sorted[(size_t)r * k], k, d.kp, vec, lanes, place.data());
+            for (int32_t j = 0; j < k; ++j) {
+                val_p[(size_t)r * d.kp + place[j]] = v_sorted[(size_t)r * k + j];
+                idx_p[(size_t)r * d.kp + place[j]] = c_sorted[(size_t)r * k + j];
+            }
+        }
+        const float* p = nullptr;
+        st = upload(l, val_p, &p);
+        d.values = p;
+    } else {
+        std::vector<uint16_t> val_p((size_t)n_active * d.kp, (uint16_t)0);
+        for (int32_t r = 0; r < n_active; ++r) {
+            order_for_banks(&c_sorted[(size_t)r * k], k, d.kp, vec, lanes, place.data());
+            for (int32_t j = 0; j < k; ++j) {
+                val_p[(size_t)r * d.kp + place[j]] = bf16_bits_rne(v_sorted[(size_t)r * k + j]);
+                idx_p[(size_t)r * d.kp + place[j]] = c_sorted[(size_t)r * k + j];
+            }
+        }
+        const uint16_t* p = nullptr;
+        st = upload(l, val_p, &p);
+        d.values = p;
+    }
+    if (st == CFI_OK) st = upload(l, idx_p, &d.indices);
+
+    if (st == CFI_OK) l->layouts |= CFI_LAYOUT_SMALL_BATCH;
+    l->bytes_small += l->device_bytes - before;
+    return st;
+}
+
+// Large-batch gather layout: column slabs, 32-byte quads, per-row slab offsets.
+cfi_status_t build_gather(cfi_layer* l) {
+    const int32_t k = l->d.k, n_active = l->d.n_active, in_features = l->d.in, out_features = l->d.out;
+    const int dtype = l->dtype;
+    DevLayer& d = l->d;
+    const std::vector<float>& v_sorted = l->h_values;
+    const std::vector<int32_t>&c_sorted = l->h_cols, &active_rows = l->h_rows, &slot = l->h_slot;
+    cfi_status_t st = CFI_OK;
+    const int64_t before = l->device_bytes;
+    (void)k, (void)n_active, (void)in_features, (void)out_features, (void)dtype, (void)d, (void)v_sorted, (void)c_sorted,
+        (void)active_rows, (void)slot;
+    // ---- large-batch layout: the fewest slabs (at least two when there is enough to pipeline) for which
+    // two x buffers, the tile metadata and the per-warp weight buffers of the largest tile fit.
+    const int es = dtype == CFI_BF16 ? 2 : 4;
+    std::vector<int32_t> seg;
+    for (int n_slabs = in_features >= 128 ? 2 : 1;; ++n_slabs) {
+        d.cs = std::max(8, (((in_features + n_slabs - 1) / n_slabs) + 7) & ~7);
+        d.n_slabs = std::max(1, (in_features + d.cs - 1) / d.cs);
+        seg.assign((size_t)n_active * (d.n_slabs + 1), 0);
+        int max_row_quads = 1, maxq = 1;
+        for (int32_t r = 0; r < n_active; ++r) {
+            int q = 0, j = 0;
+            for (int s = 0; s < d.n_slabs; ++s) {
+                seg[(size_t)r * (d.n_slabs + 1) + s] = q;
+                int cnt = 0;
+                while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) ++j, ++cnt;
+                q += (cnt + 3) / 4;
+                maxq = std::max(maxq, (cnt + 3) / 4);
+            }
+            seg[(size_t)r * (d.n_slabs + 1) + d.n_slabs] = q;
+            max_row_quads = std::max(max_row_quads, q);
+        }
+        d.stride_q = max_row_quads;
+        d.maxq = maxq;
+        const BatchSmem m = batch_smem_layout(d.cs, d.n_slabs, d.maxq, es, kBatchTile, 128, 8);
+        if (m.total <= (size_t)kBatchSmemBudget || d.cs <= 8) break;
+    }
+    struct Quad { float w[4]; int32_t c[4]; };
+    std::vector<Quad> quads((size_t)n_active * d.stride_q);
+    for (auto& q : quads)
+        for (int e = 0; e < 4; ++e) q.w[e] = 0.0f, q.c[e] = d.cs * kBatchTile * es;
+    for (int32_t r = 0; r < n_active; ++r) {
+        int j = 0;
+        for (int s = 0; s < d.n_slabs; ++s) {
+            size_t w = (size_t)seg[(size_t)r * (d.n_slabs + 1) + s] * 4;
+            while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) {
+                Quad& q = quads[(size_t)r * d.stride_q + w / 4];
+                q.w[w % 4] = v_sorted[(size_t)r * k + j];
+                const int col = c_sorted[(size_t)r * k + j] - s * d.cs;
+                q.c[w % 4] = col * kBatchTile * es + ((col >> 2) & (kBatchTile / 4 - 1)) * 4 * es;
+                ++w, ++j;
+            }
+        }
+    }
+    const Quad* quads_dev = nullptr;
+    if (st == CFI_OK) st = upload(l, quads, &quads_dev);
+    d.wq_b = quads_dev;
+    // The kernel looks the quad offsets up by output row: ablated rows get an all-zero line.
+    std::vector<int32_t> seg_o((size_t)out_features * (d.n_slabs + 1), 0);
+    for (int32_t o = 0; o < out_features; ++o)
+        if (slot[o] >= 0)
+            std::copy(seg.begin() + (size_t)slot[o] * (d.n_slabs + 1), seg.begin() + (size_t)(slot[o] + 1) * (d.n_slabs + 1),
+                      seg_o.begin() + (size_t)o * (d.n_slabs + 1));
+    if (st == CFI_OK) st = upload(l, seg_o, &d.seg);
+
+    if (st == CFI_OK) l->layouts |= CFI_LAYOUT_GATHER;
+    l->bytes_gather += l->device_bytes - before;
+    return st;
+}
+
+// Dense copy for the tensor-core variant; leaves tc_ok false where the shapes cannot be addressed.
+cfi_status_t build_dense(cfi_layer* l) {
+    const int32_t k = l->d.k, n_active = l->d.n_active, in_features = l->d.in, out_features = l->d.out;
+    const int dtype = l->dtype;
+    DevLayer& d = l->d;
+    const std::vector<float>& v_sorted = l->h_values;
+    const std::vector<int32_t>&c_sorted = l->h_cols, &active_rows = l->h_rows, &slot = l->h_slot;
+    cfi_status_t st = CFI_OK;
+    const int64_t before = l->device_bytes;
+    (void)k, (void)n_active, (void)in_features, (void)out_features, (void)dtype, (void)d, (void)v_sorted, (void)c_sorted,
+        (void)active_rows, (void)slot;
+    // ---- dense copy for the tensor-core variant (zero rows for ablated and padding rows), in the layer's dtype.
+    // A column kept twice in one row cannot be one dense entry, so such layers go without.
+    {
+        const int eb = dtype == CFI_BF16 ? 2 : 4, tile_n = 128;
+        bool usable = out_features > 0 && in_features * eb >= 16 && ((in_features * eb) & 15) == 0 &&
+                      ((out_features * eb) & 15) == 0 && (size_t)out_features * in_features * eb <= ((size_t)1 << 30);
+        for (int32_t r = 0; usable && r < n_active; ++r)
+            for (int32_t j = 1; j < k; ++j) usable = usable && c_sorted[(size_t)r * k + j] != c_sorted[(size_t)r * k + j - 1];
+        if (usable) {
+            l->out_pad = ((out_features + tile_n - 1) / tile_n) * tile_n;
+            const void* wd_dev = nullptr;
+            if (dtype == CFI_BF16) {
+                std::vector<uint16_t> wd((size_t)l->out_pad * in_features, (uint16_t)0);
+                for (int32_t r = 0; r < n_active; ++r)
+                    for (int32_t j = 0; j < k; ++j)
+                        wd[(size_t)active_rows[r] * in_features + c_sorted[(size_t)r * k + j]] =
+                            bf16_bits_rne(v_sorted[(size_t)r * k + j]);
+                const uint16_t* p = nullptr;
+                if (st == CFI_OK) st = upload(l, wd, &p);
+                wd_dev = p;
+            } else {
+                std::vector<float> wd((size_t)l->out_pad * in_features, 0.0f);
+                for (int32_t r = 0; r < n_active; ++r)
+                    for (int32_t j = 0; j < k; ++j)
+                        wd[(size_t)active_rows[r] * in_features + c_sorted[(size_t)r * k + j]] = v_sorted[(size_t)r * k + j];
+                const float* p = nullptr;
+                if (st == CFI_OK) st = upload(l, wd, &p);
+                wd_dev = p;
+            }
+            l->w_dense = wd_dev;
+            // Boxes of 128 rows x 128 bytes for the one-tile kernels; for bf16 layers also 256-row boxes for the
+            // persistent kernel's wide tiles.
+            l->tc_ok = st == CFI_OK && encode_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb, kTcN);
+            if (l->tc_ok && dtype == CFI_BF16)
+                l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, 2, kTpN);
+        }
+    }
+
+    if (st == CFI_OK && l->tc_ok) l->layouts |= CFI_LAYOUT_DENSE;
+    l->bytes_dense += l->device_bytes - before;
+    return st;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
@@ -1208,8 +1395,17 @@ void free_layer(cfi_layer* l) {
 extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, const int32_t* active_rows,
                                    const float* bias, int32_t n_active, int32_t k, int32_t in_features,
                                    int32_t out_features, cfi_dtype_t dtype, cfi_act_t act, cfi_layer_t** layer) {
+    return cfi_create_layouts(values, indices, active_rows, bias, n_active, k, in_features, out_features, dtype, act,
+                              CFI_LAYOUT_ALL, layer);
+}
+
+extern "C" cfi_status_t cfi_create_layouts(const float* values, const int32_t* indices, const int32_t* active_rows,
+                                           const float* bias, int32_t n_active, int32_t k, int32_t in_features,
+                                           int32_t out_features, cfi_dtype_t dtype, cfi_act_t act, int32_t layouts,
+                                           cfi_layer_t** layer) {
     if (!layer) return CFI_ERR_NULL;
     *layer = nullptr;
+    if (layouts <= 0 || (layouts & ~CFI_LAYOUT_ALL)) return CFI_ERR_DTYPE;
     if (dtype != CFI_F32 && dtype != CFI_BF16) return CFI_ERR_DTYPE;
     if (act != CFI_ACT_NONE && act != CFI_ACT_GELU_ERF) return CFI_ERR_DTYPE;
     if (n_active < 0 || k < 0 || in_features < 0 || out_features < 0) return CFI_ERR_SHAPE;
@@ -1247,8 +1443,10 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
     try {
         // Each row sorted by column (stable, so repeated columns keep the caller's order).
         std::vector<int32_t> order((size_t)std::max(k, 1));
-        std::vector<float> v_sorted(nnz);
-        std::vector<int32_t> c_sorted(nnz);
+        l->h_values.resize(nnz);
+        l->h_cols.resize(nnz);
+        l->h_rows.assign(active_rows, active_rows + n_active);
+        l->h_slot = slot;
         for (int32_t r = 0; r < n_active; ++r) {
             const size_t off = (size_t)r * k;
             std::iota(order.begin(), order.begin() + k, 0);
@@ -1257,137 +1455,17 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
             for (int32_t j = 0; j < k; ++j) {
                 float w = values[off + order[j]];
                 if (dtype == CFI_BF16) w = bf16_widen(bf16_bits_rne(w));
-                v_sorted[off + j] = w;
-                c_sorted[off + j] = indices[off + order[j]];
+                l->h_values[off + j] = w;
+                l->h_cols[off + j] = indices[off + order[j]];
             }
         }
-
-        // ---- small-batch layout
         const int vec = vec_of(dtype);
         d.kp = ((k + vec - 1) / vec) * vec;
-        std::vector<int32_t> place((size_t)std::max(d.kp, 1));  // position in the padded row of sorted entry j
-        const int lanes = splitk_lanes_per_row(std::max(1, d.kp / vec));
-        std::vector<int32_t> idx_p((size_t)n_active * d.kp, in_features);
         cfi_status_t st = CFI_OK;
-        if (dtype == CFI_F32) {
-            std::vector<float> val_p((size_t)n_active * d.kp, 0.0f);
-            for (int32_t r = 0; r < n_active; ++r) {
-                order_for_banks(&c_sorted[(size_t)r * k], k, d.kp, vec, lanes, place.data());
-                for (int32_t j = 0; j < k; ++j) {
-                    val_p[(size_t)r * d.kp + place[j]] = v_sorted[(size_t)r * k + j];
-                    idx_p[(size_t)r * d.kp + place[j]] = c_sorted[(size_t)r * k + j];
-                }
-            }
-            const float* p = nullptr;
-            st = upload(l, val_p, &p);
-            d.values = p;
-        } else {
-            std::vector<uint16_t> val_p((size_t)n_active * d.kp, (uint16_t)0);
-            for (int32_t r = 0; r < n_active; ++r) {
-                order_for_banks(&c_sorted[(size_t)r * k], k, d.kp, vec, lanes, place.data());
-                for (int32_t j = 0; j < k; ++j) {
-                    val_p[(size_t)r * d.kp + place[j]] = bf16_bits_rne(v_sorted[(size_t)r * k + j]);
-                    idx_p[(size_t)r * d.kp + place[j]] = c_sorted[(size_t)r * k + j];
-                }
-            }
-            const uint16_t* p = nullptr;
-            st = upload(l, val_p, &p);
-            d.values = p;
-        }
-        if (st == CFI_OK) st = upload(l, idx_p, &d.indices);
-
-        // ---- large-batch layout: the fewest slabs (at least two when there is enough to pipeline) for which
-        // two x buffers, the tile metadata and the per-warp weight buffers of the largest tile fit.
-        const int es = dtype == CFI_BF16 ? 2 : 4;
-        std::vector<int32_t> seg;
-        for (int n_slabs = in_features >= 128 ? 2 : 1;; ++n_slabs) {
-            d.cs = std::max(8, (((in_features + n_slabs - 1) / n_slabs) + 7) & ~7);
-            d.n_slabs = std::max(1, (in_features + d.cs - 1) / d.cs);
-            seg.assign((size_t)n_active * (d.n_slabs + 1), 0);
-            int max_row_quads = 1, maxq = 1;
-            for (int32_t r = 0; r < n_active; ++r) {
-                int q = 0, j = 0;
-                for (int s = 0; s < d.n_slabs; ++s) {
-                    seg[(size_t)r * (d.n_slabs + 1) + s] = q;
-                    int cnt = 0;
-                    while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) ++j, ++cnt;
-                    q += (cnt + 3) / 4;
-                    maxq = std::max(maxq, (cnt + 3) / 4);
-                }
-                seg[(size_t)r * (d.n_slabs + 1) + d.n_slabs] = q;
-                max_row_quads = std::max(max_row_quads, q);
-            }
-            d.stride_q = max_row_quads;
-            d.maxq = maxq;
-            const BatchSmem m = batch_smem_layout(d.cs, d.n_slabs, d.maxq, es, kBatchTile, 128, 8);
-            if (m.total <= (size_t)kBatchSmemBudget || d.cs <= 8) break;
-        }
-        struct Quad { float w[4]; int32_t c[4]; };
-        std::vector<Quad> quads((size_t)n_active * d.stride_q);
-        for (auto& q : quads)
-            for (int e = 0; e < 4; ++e) q.w[e] = 0.0f, q.c[e] = d.cs * kBatchTile * es;
-        for (int32_t r = 0; r < n_active; ++r) {
-            int j = 0;
-            for (int s = 0; s < d.n_slabs; ++s) {
-                size_t w = (size_t)seg[(size_t)r * (d.n_slabs + 1) + s] * 4;
-                while (j < k && c_sorted[(size_t)r * k + j] < (s + 1) * d.cs) {
-                    Quad& q = quads[(size_t)r * d.stride_q + w / 4];
-                    q.w[w % 4] = v_sorted[(size_t)r * k + j];
-                    const int col = c_sorted[(size_t)r * k + j] - s * d.cs;
-                    q.c[w % 4] = col * kBatchTile * es + ((col >> 2) & (kBatchTile / 4 - 1)) * 4 * es;
-                    ++w, ++j;
-                }
-            }
-        }
-        const Quad* quads_dev = nullptr;
-        if (st == CFI_OK) st = upload(l, quads, &quads_dev);
-        d.wq_b = quads_dev;
-        // The kernel looks the quad offsets up by output row: ablated rows get an all-zero line.
-        std::vector<int32_t> seg_o((size_t)out_features * (d.n_slabs + 1), 0);
-        for (int32_t o = 0; o < out_features; ++o)
-            if (slot[o] >= 0)
-                std::copy(seg.begin() + (size_t)slot[o] * (d.n_slabs + 1), seg.begin() + (size_t)(slot[o] + 1) * (d.n_slabs + 1),
-                          seg_o.begin() + (size_t)o * (d.n_slabs + 1));
-        if (st == CFI_OK) st = upload(l, seg_o, &d.seg);
-
-        // ---- dense copy for the tensor-core variant (zero rows for ablated and padding rows), in the layer's dtype.
-        // A column kept twice in one row cannot be one dense entry, so such layers go without.
-        {
-            const int eb = dtype == CFI_BF16 ? 2 : 4, tile_n = 128;
-            bool usable = out_features > 0 && in_features * eb >= 16 && ((in_features * eb) & 15) == 0 &&
-                          ((out_features * eb) & 15) == 0 && (size_t)out_features * in_features * eb <= ((size_t)1 << 30);
-            for (int32_t r = 0; usable && r < n_active; ++r)
-                for (int32_t j = 1; j < k; ++j) usable = usable && c_sorted[(size_t)r * k + j] != c_sorted[(size_t)r * k + j - 1];
-            if (usable) {
-                l->out_pad = ((out_features + tile_n - 1) / tile_n) * tile_n;
-                const void* wd_dev = nullptr;
-                if (dtype == CFI_BF16) {
-                    std::vector<uint16_t> wd((size_t)l->out_pad * in_features, (uint16_t)0);
-                    for (int32_t r = 0; r < n_active; ++r)
-                        for (int32_t j = 0; j < k; ++j)
-                            wd[(size_t)active_rows[r] * in_features + c_sorted[(size_t)r * k + j]] =
-                                bf16_bits_rne(v_sorted[(size_t)r * k + j]);
-                    const uint16_t* p = nullptr;
-                    if (st == CFI_OK) st = upload(l, wd, &p);
-                    wd_dev = p;
-                } else {
-                    std::vector<float> wd((size_t)l->out_pad * in_features, 0.0f);
-                    for (int32_t r = 0; r < n_active; ++r)
-                        for (int32_t j = 0; j < k; ++j)
-                            wd[(size_t)active_rows[r] * in_features + c_sorted[(size_t)r * k + j]] = v_sorted[(size_t)r * k + j];
-                    const float* p = nullptr;
-                    if (st == CFI_OK) st = upload(l, wd, &p);
-                    wd_dev = p;
-                }
-                l->w_dense = wd_dev;
-                // Boxes of 128 rows x 128 bytes for the one-tile kernels; for bf16 layers also 256-row boxes for the
-                // persistent kernel's wide tiles.
-                l->tc_ok = st == CFI_OK && encode_map(&l->map_w, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, eb, kTcN);
-                if (l->tc_ok && dtype == CFI_BF16)
-                    l->tc_ok = encode_map(&l->map_w_wide, wd_dev, (uint64_t)l->out_pad, (uint64_t)in_features, 2, kTpN);
-            }
-        }
-
+        if (st == CFI_OK && (layouts & CFI_LAYOUT_SMALL_BATCH)) st = build_small(l);
+        if (st == CFI_OK && (layouts & CFI_LAYOUT_GATHER)) st = build_gather(l);
+        if (st == CFI_OK && (layouts & CFI_LAYOUT_DENSE)) st = build_dense(l);
+        if (st == CFI_OK && l->layouts == 0) st = CFI_ERR_SHAPE;  // only the dense layout was asked for and it cannot be built
         std::vector<float> bias_h((size_t)out_features, 0.0f);
         if (bias) std::copy(bias, bias + out_features, bias_h.begin());
         if (st == CFI_OK) st = upload(l, bias_h, &d.bias);
@@ -1406,6 +1484,22 @@ extern "C" cfi_status_t cfi_create(const float* values, const int32_t* indices, 
     }
     *layer = l;
     return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_layer_add_layouts(cfi_layer_t* layer, int32_t layouts) {
+    if (!layer) return CFI_ERR_NULL;
+    if (layouts <= 0 || (layouts & ~CFI_LAYOUT_ALL)) return CFI_ERR_DTYPE;
+    DeviceGuard g(layer->device);
+    const int missing = layouts & ~layer->layouts;
+    cfi_status_t st = CFI_OK;
+    try {
+        if (st == CFI_OK && (missing & CFI_LAYOUT_SMALL_BATCH)) st = build_small(layer);
+        if (st == CFI_OK && (missing & CFI_LAYOUT_GATHER)) st = build_gather(layer);
+        if (st == CFI_OK && (missing & CFI_LAYOUT_DENSE) && !layer->w_dense) st = build_dense(layer);
+    } catch (const std::bad_alloc&) {
+        return CFI_ERR_ALLOC;
+    }
+    return st;
 }
 
 extern "C" cfi_status_t cfi_destroy(cfi_layer_t* layer) {
@@ -1525,6 +1619,11 @@ extern "C" cfi_status_t cfi_layer_info(const cfi_layer_t* layer, cfi_layer_info_
     info->weight_bytes_splitk = (int64_t)d.n_active * d.kp * (vs + 4);
     info->weight_bytes_batch = (int64_t)d.n_active * d.stride_q * 32;
     info->device_bytes = layer->device_bytes;
+    info->bytes_small_batch = layer->bytes_small;
+    info->bytes_gather = layer->bytes_gather;
+    info->bytes_dense = layer->bytes_dense;
+    info->layouts = layer->layouts;
+    info->reserved2 = 0;
     return CFI_OK;
 }
 

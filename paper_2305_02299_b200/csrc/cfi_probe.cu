@@ -65,6 +65,28 @@ __global__ void probe_l2_kernel(const float4* __restrict__ buf, size_t n4, int p
 
 __global__ void probe_empty_kernel() {}
 
+// The two kernels of cfi_probe_floor_launch.  Both start and finish the way the forward kernels do (they let the next
+// kernel in the stream start early and wait for the one before them), so a chain of them in a stream or graph costs
+// what a chain of forward launches would cost with all of their work taken out.
+__global__ void probe_floor_empty_kernel(float* out) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (out == nullptr) return;  // never: keeps the argument alive
+}
+// One dependent trip to DRAM per CTA and one store: thread 0 reads the launch counter (on chip), then a line of
+// `buf` that no recent launch has touched, and writes what it read to out[cta]; CTA 0 then advances the counter.
+__global__ void probe_floor_roundtrip_kernel(const float* __restrict__ buf, unsigned long long lines, unsigned long long* counter,
+                                             float* out) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (threadIdx.x == 0) {
+        const unsigned long long c = *reinterpret_cast<volatile unsigned long long*>(counter);
+        const unsigned long long line = ((c * gridDim.x + blockIdx.x) * 4099ull) % lines;
+        out[blockIdx.x] = __ldcg(buf + line * 32ull);
+        if (blockIdx.x == 0) atomicAdd(counter, 1ull);
+    }
+}
+
 float elapsed_ms(cudaEvent_t a, cudaEvent_t b) {
     float ms = 0.f;
     cudaEventElapsedTime(&ms, a, b);
@@ -153,6 +175,38 @@ extern "C" cfi_status_t cfi_probe_device(cfi_device_probe_t* p) {
     cudaFree(out);
     const cudaError_t err = cudaDeviceSynchronize();
     if (err != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
+    return CFI_OK;
+}
+
+extern "C" cfi_status_t cfi_probe_floor_launch(int32_t kind, const void* buf, size_t buf_bytes, void* scratch, cfi_stream_t stream) {
+    if (kind != 0 && kind != 1) return CFI_ERR_DTYPE;
+    if (!scratch || (kind == 1 && !buf)) return CFI_ERR_NULL;
+    if (((uintptr_t)buf | (uintptr_t)scratch) & 255u) return CFI_ERR_ALIGNMENT;
+    if (kind == 1 && buf_bytes < (1u << 20)) return CFI_ERR_BUFFER_TOO_SMALL;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)sms);
+    cfg.blockDim = dim3(128);
+    cfg.stream = reinterpret_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    unsigned long long* counter = static_cast<unsigned long long*>(scratch);
+    float* out = reinterpret_cast<float*>(counter + 32);
+    cudaError_t e;
+    if (kind == 0) e = cudaLaunchKernelEx(&cfg, probe_floor_empty_kernel, out);
+    else e = cudaLaunchKernelEx(&cfg, probe_floor_roundtrip_kernel, static_cast<const float*>(buf), (unsigned long long)(buf_bytes / 128),
+                                counter, out);
+    if (e != cudaSuccess) {
         cudaGetLastError();
         return CFI_ERR_CUDA;
     }

@@ -113,6 +113,12 @@ def test_create_rejects_bad_arguments_before_touching_cuda():
     assert lib.cfi_create(None, None, None, None, 2, 2, 4, 3, 0, 0, ctypes.byref(h)) == 1   # NULL arrays
     assert lib.cfi_forward(None, None, None, 1, None) == 1
     assert lib.cfi_destroy(None) == 0 and lib.cfi_stack_destroy(None) == 0
+    for layouts in (0, 8, -1):                                                          # empty or unknown layout set
+        with bad() as e:
+            cfi.cfi_create(v, np.zeros((2, 2), np.int32), rows, None, 4, 3, layouts=layouts)
+        assert e.value.status == 6
+    assert lib.cfi_layer_add_layouts(None, 1) == 1 and lib.cfi_forward_dense(None, None, None, 1, None, 0, 0) == 1
+    assert lib.cfi_probe_floor_launch(2, None, 0, None, None) == 6 and lib.cfi_probe_floor_launch(0, None, 0, None, None) == 1
 
 
 def test_no_cpu_fallback():
