@@ -341,6 +341,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
     ap.add_argument("--stack-only", type=int, default=0, metavar="ROWS",
                     help="run only the bf16 MLP stack leg on ROWS batch rows (for profiling) and print its JSON")
+    ap.add_argument("--sweep-only", default=None, metavar="NAMES",
+                    help="run only the floor probe and the sweep over these named workloads (comma separated; 'all') and print its JSON")
     ap.add_argument("--srigl-only", action="store_true",
                     help="run only the SRigL mask-update leg (for profiling) and print its JSON")
     args = ap.parse_args()
@@ -362,6 +364,16 @@ def main():
         torch.cuda.set_device(0)
         peaks, _ = measured_peaks()
         print(json.dumps(srigl_update_leg(cfi, torch, peaks)))
+        return
+    if args.sweep_only:
+        torch.cuda.set_device(0)
+        peaks, kind = measured_peaks()
+        props = torch.cuda.get_device_properties(0)
+        l2 = getattr(props, "L2_cache_size", None) or L2_BYTES_FALLBACK
+        only = None if args.sweep_only == "all" else set(args.sweep_only.split(","))
+        floor = floor_leg(cfi, torch, l2)
+        print(json.dumps({"floor": floor, "sweep": sweep_leg(W, cfi, torch, l2, Ceilings(peaks, kind, props.multi_processor_count),
+                                                               floor, only=only, cpu=False)}))
         return
     if args.stack_only:
         torch.cuda.set_device(0)
@@ -722,7 +734,7 @@ SWEEP = [("c1", ["c1", "c2"]), ("c3_b1", ["c3_b1", "c3_b64", "c3_b256"])] + \
         [(f"c4_s{sp}_b1", [f"c4_s{sp}_b{b}" for b in (1, 16, 256)]) for sp in (80, 90, 95, 99)]
 
 
-def sweep_leg(W, cfi, torch, l2, ceil_, floor):
+def sweep_leg(W, cfi, torch, l2, ceil_, floor, only=None, cpu=True):
     """Every named workload, cold (rotating replicas of layer, x and y larger than twice the L2): us per call (median
     and standard deviation over the passes), the kernel the library picks, algorithmic bytes and flops, the time the
     HBM and the fp32 FMA rooflines allow, the fraction of the binding one, the fraction of the gather formulation's
@@ -730,10 +742,13 @@ def sweep_leg(W, cfi, torch, l2, ceil_, floor):
     import oracle
     out = {}
     for base_name, names in SWEEP:
+        names = [n for n in names if only is None or n in only]
+        if not names:
+            continue
         base = W[base_name]
         L = base.layer(seed=0)
         packed = cfi.cfi_pack(L.w_dense, L.mask)
-        opk = oracle.pack(L.w_dense, L.mask)            # the oracle's own pack for its own timing
+        opk = oracle.pack(L.w_dense, L.mask) if cpu else None   # the oracle's own pack for its own timing
         probe = cfi.cfi_create(packed[0], packed[1], packed[2], L.bias, base.in_features, base.out_features)
         for name in names:
             w = W[name]
@@ -768,11 +783,16 @@ def sweep_leg(W, cfi, torch, l2, ceil_, floor):
                 e["us_per_call_warm"] = us(time_steps(one, torch, 1000, 10, target_s=0.02))
                 one.close()
             rep.close()
+            out[name] = e
+            if not cpu:
+                continue
             cb = time_oracle(w, budget_s=1.0, layer=L, packed=opk)
             e["cpu_oracle"] = {"us_per_call_scaled": cb["median_s"] * 1e6 * w.batch / cb["rows"], "rows_timed": cb["rows"],
                                "cores": cb["cores"], "gflops": cb["flops"] / cb["median_s"] / 1e9}
             out[name] = e
         probe.close()
+    if not cpu:
+        return out
     # The bf16 stack's CPU time: one block's two layers on a 788-row slice (1/64 of the batch), scaled.
     s = inputs.StackWorkload(blocks=1)
     x = s.x(seed=0, batch=788)

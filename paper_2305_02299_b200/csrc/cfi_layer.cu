@@ -3,7 +3,8 @@
 // Two device layouts are built from the caller's condensed arrays (values / column indices, both
 // n_active x k, as in the paper's appendix "Condensed matrix multiplication"):
 //
-//   small-batch ("split-k") layout: rows padded to a multiple of 4 (fp32) or 8 (bf16) entries so that
+//   small-batch ("split-k") layout: columns stored in 16 bits for long index streams of layers narrower than 65,536
+//     inputs, else in 32; rows padded to a multiple of 8 entries (4 for fp32 values with 32-bit columns) so that
 //     every lane reads whole 16-byte vectors; a pad entry has weight 0 and points at one extra zero
 //     element behind the staged x, so it contributes exactly 0 even when x holds inf or NaN.
 //
@@ -34,7 +35,7 @@ constexpr int kBatchSmemBudget = 216 * 1024;  // what the large-batch kernel may
 
 struct DevLayer {
     const void* values;      // [n_active][kp]  fp32 or bf16
-    const int32_t* indices;  // [n_active][kp]
+    const void* indices;     // [n_active][kp] uint16 when in_features < 65536 (idx16), else int32
     const void* wq_b;        // [n_active][stride_q] quads: 4 fp32 weights, then 4 int32 gather offsets: the byte
                              //   offset of the slab-relative column in the staged slab with the bank permutation
                              //   key folded in (a pad entry has weight 0 and points at column cs, all zero)
@@ -44,6 +45,7 @@ struct DevLayer {
     int32_t* status;
     int in, out, n_active, k, kp, act;
     int cs, n_slabs, stride_q, maxq;  // slab width, slabs, quads per row, most quads of a row in one slab
+    int idx16;                        // 1 if `indices` holds 16-bit columns
     int identity_rows;                // 1 if output row o is condensed row o for every o (no ablated row, rows in order)
 };
 
@@ -105,10 +107,10 @@ __global__ void cfi_simple_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
     float s = 0.0f;
     if (r >= 0) {
         const VT* w = reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp;
-        const int32_t* ix = L.indices + (size_t)r * L.kp;
+        const size_t ix0 = (size_t)r * L.kp;
         const VT* xr = x + (size_t)b * L.in;
         for (int j = 0; j < L.kp; ++j) {  // pad entries (column == in) may sit anywhere in the row
-            const int c = ix[j];
+            const int c = L.idx16 ? (int)static_cast<const uint16_t*>(L.indices)[ix0 + j] : static_cast<const int32_t*>(L.indices)[ix0 + j];
             if (c < L.in) s = fmaf(to_f32(w[j]), to_f32(xr[c]), s);
         }
     }
@@ -119,17 +121,23 @@ __global__ void cfi_simple_kernel(DevLayer L, const VT* __restrict__ x, VT* __re
 // CFI_VARIANT_SPLITK: small batch.  G lanes share one output row and split its k terms; the CTA's
 // x rows sit in shared memory as xs[column][BT] (+ one zero column for pad entries).
 // ------------------------------------------------------------------------------------------------
-template <typename VT> struct Chunk;
+// Units a lane of the split-k kernel keeps in flight: 4, or 2 of the 48-byte units of fp32 values with 16-bit columns
+// (the same lanes per row, and so the same launch shapes, as 4 units of 4 entries would give).
+__host__ __device__ constexpr int splitk_units_in_flight(bool fp32_values, bool idx16) { return fp32_values && idx16 ? 2 : 4; }
 
-template <> struct Chunk<float> {  // 4 weights + 4 columns
+// One lane's unit of the weight stream: VEC weights and their VEC columns, read with 16-byte loads.  With 16-bit
+// columns (every layer narrower than 65,536 inputs) a unit is 8 entries for both storage types: the index stream is
+// then 2 bytes per entry instead of 4, a quarter (fp32) to a third (bf16) fewer bytes from HBM per call.
+template <typename VT, bool I16> struct Chunk;
+
+template <> struct Chunk<float, false> {  // 4 weights + 4 int32 columns
     static constexpr int VEC = 4;
     float4 w;
     int4 c;
-    __device__ __forceinline__ void load(const void* values, const int32_t* indices, size_t row_off, int v, bool pred,
-                                         int pad_col) {
+    __device__ __forceinline__ void load(const void* values, const void* indices, size_t row_off, int v, bool pred, int pad_col) {
         if (pred) {
             w = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(values) + row_off) + v);
-            c = __ldg(reinterpret_cast<const int4*>(indices + row_off) + v);
+            c = __ldg(reinterpret_cast<const int4*>(reinterpret_cast<const int32_t*>(indices) + row_off) + v);
         } else {
             w = make_float4(0.f, 0.f, 0.f, 0.f);
             c = make_int4(pad_col, pad_col, pad_col, pad_col);
@@ -139,16 +147,15 @@ template <> struct Chunk<float> {  // 4 weights + 4 columns
     __device__ __forceinline__ int col(int e) const { return e == 0 ? c.x : e == 1 ? c.y : e == 2 ? c.z : c.w; }
 };
 
-template <> struct Chunk<__nv_bfloat16> {  // 8 weights + 8 columns
+template <> struct Chunk<__nv_bfloat16, false> {  // 8 weights + 8 int32 columns
     static constexpr int VEC = 8;
     uint4 w;
     int4 c0, c1;
-    __device__ __forceinline__ void load(const void* values, const int32_t* indices, size_t row_off, int v, bool pred,
-                                         int pad_col) {
+    __device__ __forceinline__ void load(const void* values, const void* indices, size_t row_off, int v, bool pred, int pad_col) {
         if (pred) {
             w = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(values) + row_off) + v);
-            c0 = __ldg(reinterpret_cast<const int4*>(indices + row_off) + 2 * v);
-            c1 = __ldg(reinterpret_cast<const int4*>(indices + row_off) + 2 * v + 1);
+            c0 = __ldg(reinterpret_cast<const int4*>(reinterpret_cast<const int32_t*>(indices) + row_off) + 2 * v);
+            c1 = __ldg(reinterpret_cast<const int4*>(reinterpret_cast<const int32_t*>(indices) + row_off) + 2 * v + 1);
         } else {
             w = make_uint4(0u, 0u, 0u, 0u);
             c0 = c1 = make_int4(pad_col, pad_col, pad_col, pad_col);
@@ -163,6 +170,54 @@ template <> struct Chunk<__nv_bfloat16> {  // 8 weights + 8 columns
         const int f = e & 3;
         return f == 0 ? q.x : f == 1 ? q.y : f == 2 ? q.z : q.w;
     }
+};
+
+__device__ __forceinline__ int col16(const uint4& c, int e) {
+    const uint32_t u = (e >> 1) == 0 ? c.x : (e >> 1) == 1 ? c.y : (e >> 1) == 2 ? c.z : c.w;
+    return (int)((e & 1) ? (u >> 16) : (u & 0xFFFFu));
+}
+
+template <> struct Chunk<float, true> {  // 8 weights + 8 uint16 columns
+    static constexpr int VEC = 8;
+    float4 w0, w1;
+    uint4 c;
+    __device__ __forceinline__ void load(const void* values, const void* indices, size_t row_off, int v, bool pred, int pad_col) {
+        if (pred) {
+            w0 = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(values) + row_off) + 2 * v);
+            w1 = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(values) + row_off) + 2 * v + 1);
+            c = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(indices) + row_off) + v);
+        } else {
+            w0 = w1 = make_float4(0.f, 0.f, 0.f, 0.f);
+            const uint32_t p = (uint32_t)pad_col | ((uint32_t)pad_col << 16);
+            c = make_uint4(p, p, p, p);
+        }
+    }
+    __device__ __forceinline__ float weight(int e) const {
+        const float4& q = e < 4 ? w0 : w1;
+        const int f = e & 3;
+        return f == 0 ? q.x : f == 1 ? q.y : f == 2 ? q.z : q.w;
+    }
+    __device__ __forceinline__ int col(int e) const { return col16(c, e); }
+};
+
+template <> struct Chunk<__nv_bfloat16, true> {  // 8 weights + 8 uint16 columns
+    static constexpr int VEC = 8;
+    uint4 w, c;
+    __device__ __forceinline__ void load(const void* values, const void* indices, size_t row_off, int v, bool pred, int pad_col) {
+        if (pred) {
+            w = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(values) + row_off) + v);
+            c = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(indices) + row_off) + v);
+        } else {
+            w = make_uint4(0u, 0u, 0u, 0u);
+            const uint32_t p = (uint32_t)pad_col | ((uint32_t)pad_col << 16);
+            c = make_uint4(p, p, p, p);
+        }
+    }
+    __device__ __forceinline__ float weight(int e) const {
+        const uint32_t u = (e >> 1) == 0 ? w.x : (e >> 1) == 1 ? w.y : (e >> 1) == 2 ? w.z : w.w;
+        return (e & 1) ? bf16_hi(u) : bf16_lo(u);
+    }
+    __device__ __forceinline__ int col(int e) const { return col16(c, e); }
 };
 
 template <int BT>
@@ -199,15 +254,16 @@ __device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
-// A lane keeps U = 4 16-byte vector pairs (weights + indices) in flight in registers; the rest of the row is
+// A lane keeps U units (16-byte vectors of weights with their indices) in flight in registers; the rest of the row is
 // on its way into L2.  XS = loads of x in flight per thread while staging (8 where few threads stage a long x).
-template <typename VT, int BT, int G, int XS>
+template <typename VT, bool I16, int BT, int G, int XS>
 __global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int batch,
                                   int rows_per_group) {
     extern __shared__ __align__(16) float xs_f32[];  // [(in + 1)][BT]
     float* xs = xs_f32;
-    using CK = Chunk<VT>;
-    constexpr int U = 4;
+    using CK = Chunk<VT, I16>;
+    constexpr uint32_t kIdxBytes = I16 ? 2 : 4;
+    constexpr int U = splitk_units_in_flight(sizeof(VT) == 4, I16);
     pdl_launch_dependents();
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int b0 = blockIdx.y * BT;
@@ -223,7 +279,7 @@ __global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* _
     // so the weight stream is in flight while x is awaited and staged.
     if (lg == 0 && r >= 0) {
         prefetch_l2(reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp, (uint32_t)(L.kp * sizeof(VT)));
-        prefetch_l2(L.indices + (size_t)r * L.kp, (uint32_t)(L.kp * 4));
+        prefetch_l2(static_cast<const unsigned char*>(L.indices) + (size_t)r * L.kp * kIdxBytes, (uint32_t)L.kp * kIdxBytes);
     }
     CK ck[U];
 #pragma unroll
@@ -310,7 +366,7 @@ __global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* _
             r = o < L.out ? (dense_rows ? o : L.slot[o]) : -1;
             if (lg == 0 && r >= 0) {
                 prefetch_l2(reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp, (uint32_t)(L.kp * sizeof(VT)));
-                prefetch_l2(L.indices + (size_t)r * L.kp, (uint32_t)(L.kp * 4));
+                prefetch_l2(static_cast<const unsigned char*>(L.indices) + (size_t)r * L.kp * kIdxBytes, (uint32_t)L.kp * kIdxBytes);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -629,13 +685,19 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 struct SplitkShape { int bt, g, xs, threads, rows_per_group, grid_x, grid_y; size_t smem; };
 struct BatchShape { int warps, rph, threads, rt, grid_x, grid_y; size_t smem; bool ok; };
 
-int vec_of(int dtype) { return dtype == CFI_BF16 ? 8 : 4; }
+// Entries per 16-byte unit of the small-batch layout: 8 for bf16 values and wherever the columns are 16-bit, else 4.
+// 16-bit columns: possible when the pad column `in` is representable, worth it when the index stream is long.  They
+// save 2 bytes per entry from HBM and cost a few instructions per unit on the critical path of a row; measured at
+// batch 1, layers below about a million entries run at the launch floor either way and were 0.2-0.3 us slower with
+// them, 4096 x 4096 at 80 % (3.4 M entries) went from 5.6 to 4.9 us.
+bool use_idx16(int in_features, int64_t nnz) { return in_features < 65536 && nnz >= 1500000; }
+int vec_of(int dtype, bool idx16) { return (dtype == CFI_BF16 || idx16) ? 8 : 4; }
 
-// Lanes that share a row in the split-k kernel: the smallest power of two for which 4 vectors per lane cover
-// the row, at most a warp.  The small-batch layout orders a row's entries for this number (order_for_banks).
-int splitk_lanes_per_row(int nvec) {
+// Lanes that share a row in the split-k kernel: the smallest power of two for which the units a lane keeps in flight
+// cover the row, at most a warp.  The small-batch layout orders a row's entries for this number (order_for_banks).
+int splitk_lanes_per_row(int nvec, int units) {
     int g = 4;
-    while (g < 32 && g * 4 < nvec) g <<= 1;
+    while (g < 32 && g * units < nvec) g <<= 1;
     return g;
 }
 
@@ -643,8 +705,8 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     SplitkShape s{};
     s.bt = batch >= 8 ? 8 : batch >= 3 ? 4 : batch == 2 ? 2 : 1;
     while (s.bt > 1 && (size_t)(l->d.in + 1) * s.bt * 4 > (size_t)l->smem_optin) s.bt >>= 1;
-    const int nvec = l->d.kp / vec_of(l->dtype);
-    s.g = splitk_lanes_per_row(nvec);
+    const int nvec = l->d.kp / vec_of(l->dtype, l->d.idx16 != 0);
+    s.g = splitk_lanes_per_row(nvec, splitk_units_in_flight(l->dtype == CFI_F32, l->d.idx16 != 0));
     // Every CTA stages x for itself (from L2), so larger CTAs spend less of the L2 bandwidth on x.  The staged x
     // also limits how many CTAs fit an SM; the grid is sized to one wave of what fits (at most eight CTAs per
     // SM), with several rows per group when needed (rows of a group run one after the other).
@@ -754,29 +816,34 @@ cfi_status_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int threads, size_t
     return launch_pdl_cluster(kernel, grid, threads, smem, 1, st, args...);
 }
 
-template <typename VT, int BT, int G>
+template <typename VT, bool I16, int BT, int G>
 cfi_status_t launch_splitk_g(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
                              cudaStream_t st) {
     if (s.xs == 8) {
-        if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, BT, G, 8>>(s.smem, l->device)) return e;
-        return launch_pdl(cfi_splitk_kernel<VT, BT, G, 8>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch,
+        if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, I16, BT, G, 8>>(s.smem, l->device)) return e;
+        return launch_pdl(cfi_splitk_kernel<VT, I16, BT, G, 8>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch,
                           s.rows_per_group);
     }
-    if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, BT, G, 4>>(s.smem, l->device)) return e;
-    return launch_pdl(cfi_splitk_kernel<VT, BT, G, 4>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch,
+    if (cfi_status_t e = set_smem<cfi_splitk_kernel<VT, I16, BT, G, 4>>(s.smem, l->device)) return e;
+    return launch_pdl(cfi_splitk_kernel<VT, I16, BT, G, 4>, dim3(s.grid_x, s.grid_y), s.threads, s.smem, st, l->d, x, y, batch,
                       s.rows_per_group);
+}
+
+template <typename VT, bool I16, int BT>
+cfi_status_t launch_splitk_i(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch, cudaStream_t st) {
+    switch (s.g) {
+        case 4: return launch_splitk_g<VT, I16, BT, 4>(l, s, x, y, batch, st);
+        case 8: return launch_splitk_g<VT, I16, BT, 8>(l, s, x, y, batch, st);
+        case 16: return launch_splitk_g<VT, I16, BT, 16>(l, s, x, y, batch, st);
+        case 32: return launch_splitk_g<VT, I16, BT, 32>(l, s, x, y, batch, st);
+    }
+    return CFI_ERR_SHAPE;
 }
 
 template <typename VT, int BT>
 cfi_status_t launch_splitk_bt(const cfi_layer* l, const SplitkShape& s, const VT* x, VT* y, int batch,
                               cudaStream_t st) {
-    switch (s.g) {
-        case 4: return launch_splitk_g<VT, BT, 4>(l, s, x, y, batch, st);
-        case 8: return launch_splitk_g<VT, BT, 8>(l, s, x, y, batch, st);
-        case 16: return launch_splitk_g<VT, BT, 16>(l, s, x, y, batch, st);
-        case 32: return launch_splitk_g<VT, BT, 32>(l, s, x, y, batch, st);
-    }
-    return CFI_ERR_SHAPE;
+    return l->d.idx16 ? launch_splitk_i<VT, true, BT>(l, s, x, y, batch, st) : launch_splitk_i<VT, false, BT>(l, s, x, y, batch, st);
 }
 
 template <typename VT>
@@ -1226,10 +1293,10 @@ cfi_status_t build_small(cfi_layer* l) {
     (void)k, (void)n_active, (void)in_features, (void)out_features, (void)dtype, (void)d, (void)v_sorted, (void)c_sorted,
         (void)active_rows, (void)slot;
     // ---- small-batch layout
-    const int vec = vec_of(dtype);
+    const int vec = vec_of(dtype, d.idx16 != 0);
     d.kp = ((k + vec - 1) / vec) * vec;
     std::vector<int32_t> place((size_t)std::max(d.kp, 1));  // position in the padded row of sorted entry j
-    const int lanes = splitk_lanes_per_row(std::max(1, d.kp / vec));
+    const int lanes = splitk_lanes_per_row(std::max(1, d.kp / vec), splitk_units_in_flight(dtype == CFI_F32, d.idx16 != 0));
     std::vector<int32_t> idx_p((size_t)n_active * d.kp, in_features);
     if (dtype == CFI_F32) {
         std::vector<float> val_p((size_t)n_active * d.kp, 0.0f);
@@ -1256,7 +1323,18 @@ cfi_status_t build_small(cfi_layer* l) {
         st = upload(l, val_p, &p);
         d.values = p;
     }
-    if (st == CFI_OK) st = upload(l, idx_p, &d.indices);
+    if (st == CFI_OK) {
+        if (d.idx16) {
+            std::vector<uint16_t> idx16(idx_p.begin(), idx_p.end());
+            const uint16_t* p = nullptr;
+            st = upload(l, idx16, &p);
+            d.indices = p;
+        } else {
+            const int32_t* p = nullptr;
+            st = upload(l, idx_p, &p);
+            d.indices = p;
+        }
+    }
 
     if (st == CFI_OK) l->layouts |= CFI_LAYOUT_SMALL_BATCH;
     l->bytes_small += l->device_bytes - before;
@@ -1459,7 +1537,8 @@ extern "C" cfi_status_t cfi_create_layouts(const float* values, const int32_t* i
                 l->h_cols[off + j] = indices[off + order[j]];
             }
         }
-        const int vec = vec_of(dtype);
+        d.idx16 = use_idx16(in_features, (int64_t)nnz) ? 1 : 0;
+        const int vec = vec_of(dtype, d.idx16 != 0);
         d.kp = ((k + vec - 1) / vec) * vec;
         cfi_status_t st = CFI_OK;
         if (st == CFI_OK && (layouts & CFI_LAYOUT_SMALL_BATCH)) st = build_small(l);
@@ -1616,7 +1695,7 @@ extern "C" cfi_status_t cfi_layer_info(const cfi_layer_t* layer, cfi_layer_info_
     info->batch_slab_columns = d.cs;
     info->batch_row_stride = d.stride_q * 4;
     info->reserved = 0;
-    info->weight_bytes_splitk = (int64_t)d.n_active * d.kp * (vs + 4);
+    info->weight_bytes_splitk = (int64_t)d.n_active * d.kp * (vs + (d.idx16 ? 2 : 4));
     info->weight_bytes_batch = (int64_t)d.n_active * d.stride_q * 32;
     info->device_bytes = layer->device_bytes;
     info->bytes_small_batch = layer->bytes_small;

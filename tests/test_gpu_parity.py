@@ -284,3 +284,28 @@ def test_wide_layer_small_batch_falls_back_to_a_kernel_that_fits():
     with pytest.raises(cfi.CfiError):
         run_device(dl, inputs.make_x(1, in_f), "f32", "splitk")
     dl.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_long_index_stream_with_16_bit_columns(dtype):
+    """Above 1.5 M entries (and below 65,536 inputs) the small-batch layout stores its columns in 16 bits: the stream
+    is 2 bytes per entry shorter (checked through cfi_layer_info) and every batch tile of the small-batch kernels
+    still matches the oracle, ablated rows, odd fan-in and the pad column included."""
+    from paper_2305_02299_b200 import binding as cfi
+    in_f, out_f, k = 2052, 1100, 1501                                  # 1.6 M entries, k not a multiple of 8
+    L = inputs.make_layer(in_f, out_f, k, n_ablated=31, seed=5)
+    dl = device_layer(L, dtype, "gelu")
+    info = cfi.cfi_layer_info(dl)
+    assert info.k_padded == 1504
+    assert info.weight_bytes_splitk == info.n_active * info.k_padded * ((4 if dtype == "f32" else 2) + 2)
+    packed = oracle.pack(L.w_dense, L.mask)
+    for B in (1, 2, 3, 5, 8, 17):
+        x = inputs.make_x(B, in_f, seed=B)
+        y_ref, S = oracle_layer(L, x, dtype, "gelu", packed=packed)
+        for v in ("splitk", "simple", "auto"):
+            assert_parity(run_device(dl, x, dtype, v), y_ref, S, dtype, f"{v} B={B}")
+    dl.close()
+    small = device_layer(inputs.make_layer(64, 40, 7, seed=1), dtype)  # a short stream keeps 32-bit columns
+    i2 = cfi.cfi_layer_info(small)
+    assert i2.weight_bytes_splitk == i2.n_active * i2.k_padded * ((4 if dtype == "f32" else 2) + 4)
+    small.close()
