@@ -495,7 +495,7 @@ def main():
         dist.destroy_process_group()
 
 
-VARIANT_NAMES = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}
+VARIANT_NAMES = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc", 5: "slab"}
 # DRAM bytes (read + written) of one launch from an ncu capture, keyed by (workload, kernel, launch shape); see profiles/.
 CAPTURED_TRAFFIC = {}
 
@@ -508,7 +508,8 @@ def dense_shape(cfi, layer, batch):
 def kernel_name(variant, shape=None, dtype="f32"):
     if variant == "dense_tc":
         return f"cfi_dense_split_kernel<{shape['batch_tile']}>" if shape else "cfi_dense_split_kernel"
-    return {"batch": "cfi_batch_kernel<float>", "splitk": "cfi_splitk_kernel<float>", "simple": "cfi_simple_kernel<float>"}[variant]
+    return {"batch": "cfi_batch_kernel<float>", "splitk": "cfi_splitk_kernel<float>", "simple": "cfi_simple_kernel<float>",
+            "slab": "cfi_slab_kernel<float>"}[variant]
 
 
 class Ceilings:

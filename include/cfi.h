@@ -62,6 +62,8 @@ typedef enum {
     CFI_VARIANT_SIMPLE = 1,   /* one thread per output element, no staging: a cross-check, not fast      */
     CFI_VARIANT_SPLITK = 2,   /* small batch: lanes split a row's k terms, x staged in shared memory     */
     CFI_VARIANT_BATCH = 3,    /* large batch: lanes own batch columns, x tile transposed in shared memory */
+    CFI_VARIANT_SLAB = 5,     /* a few tens of batch rows (tiles of 16) on a very sparse layer: the columns of x are
+                                 divided over a thread-block cluster that shares a group of output rows           */
     CFI_VARIANT_DENSE_TC = 4  /* batch above a handful of rows: dense copy of the weight on the tensor cores (tcgen05):
                                  bf16 layers directly, fp32 layers as three TF32 products of operands split into two
                                  TF32-exact parts each (K may be split over a thread-block cluster); needs row pitches
@@ -73,7 +75,7 @@ typedef enum {
  * values and indices instead of the n x d weight), so a caller chooses what to pay for. */
 typedef enum {
     CFI_LAYOUT_SMALL_BATCH = 1, /* values + indices, n_active x k padded to 16-byte vectors: CFI_VARIANT_SPLITK / SIMPLE   */
-    CFI_LAYOUT_GATHER = 2,      /* the same entries grouped by column slab for CFI_VARIANT_BATCH: about as large            */
+    CFI_LAYOUT_GATHER = 2,      /* the same entries grouped by column slab for CFI_VARIANT_BATCH / SLAB: about as large     */
     CFI_LAYOUT_DENSE = 4,       /* dense out x in copy in the layer's dtype for CFI_VARIANT_DENSE_TC: 1 / density as large  */
     CFI_LAYOUT_ALL = 7
 } cfi_layout_t;

@@ -19,10 +19,10 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 ACT_NONE, ACT_GELU = 0, 1
-VARIANT_AUTO, VARIANT_SIMPLE, VARIANT_SPLITK, VARIANT_BATCH, VARIANT_DENSE_TC = 0, 1, 2, 3, 4
+VARIANT_AUTO, VARIANT_SIMPLE, VARIANT_SPLITK, VARIANT_BATCH, VARIANT_DENSE_TC, VARIANT_SLAB = 0, 1, 2, 3, 4, 5
 _DTYPES = {"f32": F32, "fp32": F32, "float32": F32, "bf16": BF16, "bfloat16": BF16, F32: F32, BF16: BF16}
 _ACTS = {"none": ACT_NONE, None: ACT_NONE, "gelu": ACT_GELU, ACT_NONE: ACT_NONE, ACT_GELU: ACT_GELU}
-_VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4}
+_VARIANTS = {"auto": 0, "simple": 1, "splitk": 2, "batch": 3, "dense_tc": 4, "slab": 5, 0: 0, 1: 1, 2: 2, 3: 3, 4: 4, 5: 5}
 
 EXPORTS = ("cfi_status_string", "cfi_pack", "cfi_compact_producer", "cfi_compact_consumer", "cfi_srigl_workspace_bytes",
            "cfi_srigl_update", "cfi_pack_device", "cfi_create", "cfi_create_layouts", "cfi_layer_add_layouts", "cfi_forward", "cfi_forward_variant", "cfi_forward_dense",

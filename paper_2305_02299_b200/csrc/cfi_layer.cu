@@ -676,6 +676,7 @@ cfi_batch_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int b
 }
 
 #include "cfi_dense_tc.cuh"
+#include "cfi_slab.cuh"
 #include "cfi_dense_split.cuh"
 #include "cfi_dense_tc_persistent.cuh"
 
@@ -938,7 +939,7 @@ constexpr int kMaxSplit = kMaxClusterSplit;
 // wave pays it again), the cluster reduction when K is split, and the launch itself.  The dense weight pieces
 // (4 bytes per dense entry) have to come from HBM at least once per call.
 constexpr double kSplitLaunch = 0.7e-6, kSplitWave = 4.2e-6, kSplitHbmBytesPerSecond = 5.5e12;
-double split_seconds_per_block(int bt) { return bt >= 128 ? 0.51e-6 : 0.49e-6; }  // bound by the issue of 4 + 4 MMAs and a commit
+double split_seconds_per_block(int bt) { return bt >= 128 ? 0.51e-6 : bt >= 64 ? 0.42e-6 : 0.31e-6; }  // the issue of 4 + 4 MMAs and a commit
 double split_seconds_reduce(int bt) { return 0.5e-6 + 0.95e-6 * bt / 128.0; }
 int split_bt_index(int bt) { return bt >= 128 ? 3 : bt >= 64 ? 2 : bt >= 32 ? 1 : 0; }
 
@@ -1134,6 +1135,101 @@ cfi_status_t launch_dense_tc(const cfi_layer* l, const void* x, void* y, int bat
                               l->d, map_x, l->map_w, static_cast<__nv_bfloat16*>(y), batch);
 }
 
+// Clusters of `split` CTAs of the slab kernel with `smem` bytes of shared memory each that the device holds at once
+// (cached per device, storage type, cluster size and 8 KB step of shared memory; 0 if unknown).
+int slab_resident_clusters(const cfi_layer* l, int split, size_t smem) {
+    static std::atomic<int> cache[kMaxDevices][2][4][32];
+    const int bf = l->dtype == CFI_BF16 ? 1 : 0, ls = split >= 8 ? 3 : split >= 4 ? 2 : split >= 2 ? 1 : 0;
+    const int step = (int)std::min<size_t>(31, smem >> 13);
+    if (l->device < 0 || l->device >= kMaxDevices) return 0;
+    std::atomic<int>& c = cache[l->device][bf][ls][step];
+    int v = c.load(std::memory_order_acquire);
+    if (v == 0) {
+        v = -1;
+        const size_t bytes = ((size_t)step + 1) << 13;  // the step's upper end
+        const bool set = bf ? set_smem<cfi_slab_kernel<__nv_bfloat16>>(bytes, l->device) == CFI_OK
+                            : set_smem<cfi_slab_kernel<float>>(bytes, l->device) == CFI_OK;
+        if (set) {
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)split, 1, 1);
+            cfg.blockDim = dim3(kSlabThreads);
+            cfg.dynamicSmemBytes = bytes;
+            cudaLaunchAttribute attr{};
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = (unsigned)split, attr.val.clusterDim.y = 1, attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            const cudaError_t e = bf ? cudaOccupancyMaxActiveClusters(&n, cfi_slab_kernel<__nv_bfloat16>, &cfg)
+                                     : cudaOccupancyMaxActiveClusters(&n, cfi_slab_kernel<float>, &cfg);
+            if (e == cudaSuccess && n > 0) v = n;
+            else cudaGetLastError();
+        }
+        c.store(v, std::memory_order_release);
+    }
+    return v > 0 ? v : 0;
+}
+
+// Launch shape of the slab kernel: S CTAs of a cluster share a group of rows and divide the column slabs (the fewest
+// for which a CTA's columns of a 16-row batch tile take at most 96 KB, so that two CTAs fit an SM), and the rows are
+// divided into as many groups as the device holds clusters at once: one wave.
+struct SlabShape { int split, groups, rows_pc, tiles, ncols_max; size_t smem; bool ok; };
+
+SlabShape slab_shape(const cfi_layer* l, int batch) {
+    SlabShape s{};
+    s.ok = false;
+    if (!(l->layouts & CFI_LAYOUT_GATHER) || l->d.out < 1 || batch < 1) return s;
+    s.tiles = (batch + kSlabBT - 1) / kSlabBT;
+    if (s.tiles > 65535) return s;
+    for (int split = 1; split <= kMaxClusterSplit; split <<= 1) {
+        const int nsl_max = (l->d.n_slabs + split - 1) / split, ncols_max = nsl_max * l->d.cs;
+        const size_t xbytes = (size_t)(ncols_max + 1) * kSlabBT * 4;
+        if (xbytes > 96 * 1024 && split < kMaxClusterSplit) continue;
+        s.split = split, s.ncols_max = ncols_max;
+        auto with_groups = [&](int64_t want) {
+            const int groups = (int)std::max<int64_t>(1, std::min<int64_t>(want, (l->d.out + kSlabWarps - 1) / kSlabWarps));
+            s.rows_pc = (l->d.out + groups - 1) / groups;
+            s.groups = (l->d.out + s.rows_pc - 1) / s.rows_pc;
+            s.smem = xbytes + (size_t)s.rows_pc * kSlabBT * 4 + (size_t)s.rows_pc * (nsl_max + 2) * 4;
+        };
+        with_groups((2 * (int64_t)l->sm_count) / ((int64_t)split * s.tiles));
+        if (s.smem <= (size_t)l->smem_optin) {
+            const int resident = slab_resident_clusters(l, split, s.smem);
+            if (resident > 0 && (int64_t)s.groups * s.tiles > resident) with_groups(resident / s.tiles);
+        }
+        s.ok = s.smem <= (size_t)l->smem_optin && s.groups <= 65535;
+        return s;
+    }
+    return s;
+}
+
+template <typename VT>
+cfi_status_t launch_slab(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st) {
+    const SlabShape s = slab_shape(l, batch);
+    if (!s.ok) return CFI_ERR_SHAPE;
+    if (cfi_status_t e = set_smem<cfi_slab_kernel<VT>>(s.smem, l->device)) return e;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)s.split, (unsigned)s.groups, (unsigned)s.tiles);
+    cfg.blockDim = dim3(kSlabThreads);
+    cfg.dynamicSmemBytes = s.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2]{};
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)s.split;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = s.split > 1 ? 2 : 1;
+    if (cudaLaunchKernelEx(&cfg, cfi_slab_kernel<VT>, l->d, static_cast<const VT*>(x), static_cast<VT*>(y), batch, s.rows_pc,
+                           s.ncols_max) != cudaSuccess) {
+        cudaGetLastError();
+        return CFI_ERR_CUDA;
+    }
+    return CFI_OK;
+}
+
 // Rate of the gather kernel's arithmetic, used to choose between it and the split-TF32 dense kernel (measured).
 constexpr double kGatherTflops = 12.5;
 
@@ -1148,6 +1244,12 @@ int fallback_variant(const cfi_layer* l, int batch) {
     if (splitk_fits(l, batch)) return CFI_VARIANT_SPLITK;
     if (l->tc_ok && !(l->layouts & CFI_LAYOUT_SMALL_BATCH)) return CFI_VARIANT_DENSE_TC;
     return CFI_VARIANT_SIMPLE;
+}
+
+// Time model of the slab kernel (measured, fp32): a fixed part (cluster launch, row table, staging of x, cluster
+// reduction) and the entries of all batch tiles at the rate the gathers sustain.
+double slab_seconds(const cfi_layer* l, int batch) {
+    return 10.8e-6 + 4.4e-12 * (double)l->d.n_active * l->d.k * ((batch + kSlabBT - 1) / kSlabBT);
 }
 
 int choose_variant(const cfi_layer* l, int batch) {
@@ -1167,6 +1269,10 @@ int choose_variant(const cfi_layer* l, int batch) {
             double t_dense = 0.0;
             if (l->dtype == CFI_F32) t_dense = split_shape(l, batch).seconds;
             else tc_bf16_split(l, batch, &t_dense);
+            // Very sparse fp32 layers: the condensed arrays are far smaller than the dense copy, and the slab kernel
+            // reads only them.
+            if (l->dtype == CFI_F32 && slab_seconds(l, batch) < std::min(t_dense, t_splitk) && slab_shape(l, batch).ok)
+                return CFI_VARIANT_SLAB;
             if (t_dense < t_splitk) return CFI_VARIANT_DENSE_TC;
         }
         return splitk_fits(l, batch) ? CFI_VARIANT_SPLITK : fallback_variant(l, batch);
@@ -1187,6 +1293,7 @@ int choose_variant(const cfi_layer* l, int batch) {
         // Arithmetic and the re-staging of x overlap about half of the shorter of the two.
         const double t_fma = 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12), t_stage = staging / 3.7e12;
         const double t_gather = t_fma + t_stage - 0.5 * std::min(t_fma, t_stage) + 5e-6;
+        if (batch <= 64 && slab_seconds(l, batch) < std::min(t_dense, t_gather) && slab_shape(l, batch).ok) return CFI_VARIANT_SLAB;
         if (t_dense < t_gather) return CFI_VARIANT_DENSE_TC;
     }
     return fallback_variant(l, batch);
@@ -1631,6 +1738,8 @@ extern "C" cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void
         }
         case CFI_VARIANT_DENSE_TC:
             return launch_dense_tc(layer, x, y, batch, st);
+        case CFI_VARIANT_SLAB:
+            return bf ? launch_slab<__nv_bfloat16>(layer, x, y, batch, st) : launch_slab<float>(layer, x, y, batch, st);
         case CFI_VARIANT_BATCH: {
             const BatchShape s = batch_shape(layer, batch);
             return bf ? launch_batch<__nv_bfloat16>(layer, s, x, y, batch, st)

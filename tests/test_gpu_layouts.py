@@ -10,7 +10,7 @@ from parity import TOL, assert_parity, oracle_layer, run_device
 
 pytestmark = pytest.mark.gpu
 SMALL, GATHER, DENSE = 1, 2, 4
-NEEDS = {"simple": SMALL, "splitk": SMALL, "batch": GATHER, "dense_tc": DENSE}
+NEEDS = {"simple": SMALL, "splitk": SMALL, "batch": GATHER, "dense_tc": DENSE, "slab": GATHER}
 
 
 @pytest.mark.parametrize("layouts", [1, 2, 3, 4, 5, 6, 7])
@@ -29,7 +29,7 @@ def test_every_layout_subset_runs_every_batch(layouts, dtype):
     for B in (1, 3, 8, 17, 40, 130, 300):
         x = inputs.make_x(B, 256, seed=B)
         y_ref, S = oracle_layer(L, x, dtype, "gelu")
-        assert NEEDS[{1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc"}[cfi.cfi_choose_variant(dl, B)]] & layouts
+        assert NEEDS[{1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc", 5: "slab"}[cfi.cfi_choose_variant(dl, B)]] & layouts
         assert_parity(run_device(dl, x, dtype, "auto"), y_ref, S, dtype, f"layouts {layouts} B {B}")
     x = inputs.make_x(5, 256)
     for variant, need in NEEDS.items():
@@ -60,7 +60,7 @@ def test_small_batch_only_layer_is_small_and_can_grow():
     cfi.cfi_layer_add_layouts(dl, DENSE | GATHER)
     info = cfi.cfi_layer_info(dl)
     assert info.layouts == 7 and info.bytes_dense >= 4096 * 4096 * 4
-    assert cfi.cfi_choose_variant(dl, 300) in (3, 4)
+    assert cfi.cfi_choose_variant(dl, 300) in (3, 4, 5)
     assert_parity(run_device(dl, x300, "f32", "auto"), y_ref, S, "f32")
     cfi.cfi_layer_add_layouts(dl, 7)                                  # nothing missing: no-op
     assert cfi.cfi_layer_info(dl).device_bytes == info.device_bytes

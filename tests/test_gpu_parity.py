@@ -12,7 +12,7 @@ from paper_2305_02299_b200 import inputs
 from parity import TOL, assert_parity, check_layer, device_layer, oracle_layer, run_device, scaled_error, to_device, torch_dtype
 
 pytestmark = pytest.mark.gpu
-ALL = ("simple", "splitk", "batch", "auto")
+ALL = ("simple", "splitk", "batch", "slab", "auto")
 
 
 @pytest.mark.parametrize("k", [1, 2, 3, 4, 5, 31, 32, 33, 77])
@@ -309,3 +309,48 @@ def test_long_index_stream_with_16_bit_columns(dtype):
     i2 = cfi.cfi_layer_info(small)
     assert i2.weight_bytes_splitk == i2.n_active * i2.k_padded * ((4 if dtype == "f32" else 2) + 4)
     small.close()
+
+
+@pytest.mark.parametrize("in_f,out_f,k,nabl", [(4096, 300, 41, 9), (3072, 768, 307, 77), (700, 40, 100, 3), (6000, 64, 13, 0), (20000, 24, 6, 2)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_slab_kernel_cluster_shapes(in_f, out_f, k, nabl, dtype):
+    """The slab kernel with its column slabs on one CTA and divided over clusters of 2, 4 and 8 (by layer width), ragged
+    last slab, ragged batch tile, more than one batch tile, ablated rows, bit-identical on a second run."""
+    L = inputs.make_layer(in_f, out_f, k, n_ablated=nabl, seed=in_f)
+    dl = device_layer(L, dtype, "gelu")
+    packed = oracle.pack(L.w_dense, L.mask)
+    for B in (9, 16, 37, 64):
+        x = inputs.make_x(B, in_f, seed=B)
+        y_ref, S = oracle_layer(L, x, dtype, "gelu", packed=packed)
+        y = run_device(dl, x, dtype, "slab")
+        assert_parity(y, y_ref, S, dtype, f"B={B}")
+        assert np.array_equal(y, run_device(dl, x, dtype, "slab"))
+    dl.close()
+
+
+def test_slab_kernel_refuses_a_layer_too_wide_for_a_cluster():
+    from paper_2305_02299_b200 import binding as cfi
+    dl = device_layer(inputs.make_layer(40000, 24, 6, seed=1))      # an eighth of x for 16 batch rows exceeds shared memory
+    with pytest.raises(cfi.CfiError) as e:
+        run_device(dl, inputs.make_x(16, 40000), "f32", "slab")
+    assert e.value.status == 2
+    assert cfi.cfi_choose_variant(dl, 16) != 5
+    dl.close()
+
+
+def test_slab_kernel_exact_integers_and_unused_inf():
+    L = inputs.make_layer(1024, 150, 24, n_ablated=11, seed=7, integer_valued=True)
+    x = inputs.make_x(40, 1024, seed=7, integer_valued=True)
+    y_ref, _ = oracle_layer(L, x, "f32")
+    dl = device_layer(L, "f32")
+    assert np.array_equal(run_device(dl, x, "f32", "slab"), y_ref)
+    dl.close()
+    L = inputs.make_layer(900, 20, 3, seed=3)                      # most columns unused; pad entries in every quad
+    unused = np.nonzero(L.mask.sum(axis=0) == 0)[0]
+    x = inputs.make_x(20, 900, seed=3)
+    x[:, unused] = np.inf
+    y_ref, S = oracle_layer(L, x)
+    dl = device_layer(L)
+    y = run_device(dl, x, "f32", "slab")
+    assert np.all(np.isfinite(y)) and scaled_error(y, y_ref, S) <= 1e-5
+    dl.close()
