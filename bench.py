@@ -339,6 +339,8 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--variant", default="auto")
     ap.add_argument("--no-extras", action="store_true", help="skip the batch-1 and CPU-baseline legs")
+    ap.add_argument("--target-s", type=float, default=0.25,
+                    help="seconds of timed passes to aim for (at least five passes are always timed); small values for profiler runs")
     ap.add_argument("--stack-only", type=int, default=0, metavar="ROWS",
                     help="run only the bf16 MLP stack leg on ROWS batch rows (for profiling) and print its JSON")
     ap.add_argument("--sweep-only", default=None, metavar="NAMES",
@@ -402,13 +404,13 @@ def main():
 
     rep = Replicas(w, cfi, torch, 2 * l2 + (32 << 20), rank=rank)
     sampler = ClockSampler(local)
-    timed = time_steps(rep, torch, args.steps, args.warmup, args.variant, barrier=barrier, sampler=sampler)
+    timed = time_steps(rep, torch, args.steps, args.warmup, args.variant, barrier=barrier, sampler=sampler, target_s=args.target_s)
     per_call = max_over_ranks(timed["sec_per_step"], dist, "cuda")
     flops = algorithmic_flops(w, rep.n_active)
     value = whole_job_value(flops, world, per_call)
 
     # End to end through the host-buffer entry point (each rank on its own GPU).
-    e2e_steps = int(min(max(args.steps, 200), 2000))
+    e2e_steps = int(min(max(args.steps, 200), 2000)) if args.target_s >= 0.25 else 8
     e2e_sec, h2d, d2h = time_e2e(rep, torch, e2e_steps, 5)
     e2e_sec = max_over_ranks(e2e_sec, dist, "cuda")
     e2e_value = whole_job_value(flops, world, e2e_sec / e2e_steps)
@@ -497,7 +499,10 @@ def main():
 
 VARIANT_NAMES = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc", 5: "slab"}
 # DRAM bytes (read + written) of one launch from an ncu capture, keyed by (workload, kernel, launch shape); see profiles/.
-CAPTURED_TRAFFIC = {}
+CAPTURED_TRAFFIC = {
+    # profiles/cfi_dense_split_kernel_c2_768x3072_k77_b256.md: 10.285 MB read (dense copy + x), 0 written (y still in L2)
+    ("c2", "cfi_dense_split_kernel<128>", json.dumps({"batch_tile": 128, "cluster_k_split": 2})): 10.285e6,
+}
 
 
 def dense_shape(cfi, layer, batch):

@@ -1263,12 +1263,13 @@ int choose_variant(const cfi_layer* l, int batch) {
         // variant does for any batch up to 128 (measured 4096 x 4096 at 80 %, batch 16: 31 against 25 us; 3072 -> 768:
         // 22 against 11 us).  A pass of eight batch rows costs about 2.3 us plus the larger of staging x (90 ns per KB
         // of the 8-row tile, every CTA stages all of it) and the weights (176 G entries per second).
-        if (batch > 8 && l->tc_ok) {
+        if (batch > 8) {
+            constexpr double kNever = 1e30;
             const double t_stage = (double)l->d.in * 8 * 4 / 1024.0 * 90e-9, t_fma = (double)l->d.n_active * l->d.k / 176e9;
-            const double t_splitk = ((batch + 7) / 8) * (2.3e-6 + std::max(t_stage, t_fma));
-            double t_dense = 0.0;
-            if (l->dtype == CFI_F32) t_dense = split_shape(l, batch).seconds;
-            else tc_bf16_split(l, batch, &t_dense);
+            const double t_splitk = splitk_fits(l, batch) ? ((batch + 7) / 8) * (2.3e-6 + std::max(t_stage, t_fma)) : kNever;
+            double t_dense = kNever;
+            if (l->tc_ok && l->dtype == CFI_F32) t_dense = split_shape(l, batch).seconds;
+            else if (l->tc_ok) tc_bf16_split(l, batch, &t_dense);
             // Very sparse fp32 layers: the condensed arrays are far smaller than the dense copy, and the slab kernel
             // reads only them.
             if (l->dtype == CFI_F32 && slab_seconds(l, batch) < std::min(t_dense, t_splitk) && slab_shape(l, batch).ok)
@@ -1295,6 +1296,12 @@ int choose_variant(const cfi_layer* l, int batch) {
         const double t_gather = t_fma + t_stage - 0.5 * std::min(t_fma, t_stage) + 5e-6;
         if (batch <= 64 && slab_seconds(l, batch) < std::min(t_dense, t_gather) && slab_shape(l, batch).ok) return CFI_VARIANT_SLAB;
         if (t_dense < t_gather) return CFI_VARIANT_DENSE_TC;
+    }
+    if (batch <= 64 && l->dtype == CFI_F32 && !l->tc_ok && slab_shape(l, batch).ok) {
+        // Without a dense copy: the slab kernel against the gather kernel's 64-wide, partly empty batch tiles.
+        const BatchShape bs = batch_shape(l, batch);
+        if (!bs.ok || slab_seconds(l, batch) < 2.0 * batch * (double)l->d.n_active * l->d.k / (kGatherTflops * 1e12) * (64.0 / std::min(batch, 64)) + 8e-6)
+            return CFI_VARIANT_SLAB;
     }
     return fallback_variant(l, batch);
 }
