@@ -121,7 +121,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "memory");
 }
 
-// Thread-block cluster helpers (K split over a cluster, see below and cfi_dense_tf32.cuh).
+// Thread-block cluster helpers (K split over a cluster, see below, cfi_dense_split.cuh and cfi_slab.cuh).
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));

@@ -1,9 +1,9 @@
 // CFI_VARIANT_DENSE_TC for bf16 layers at very large batch: a persistent kernel with 128 x 256 tiles.
 //
-// Included by cfi_layer.cu after cfi_dense_tc.cuh and cfi_dense_tf32.cuh (same operands and helpers).
+// Included by cfi_layer.cu after cfi_dense_tc.cuh (same operands and helpers).
 //
-// Two things hold the one-tile kernel (128 x 128 tiles, two CTAs per SM) back at 50,432 rows.  An MMA instruction has
-// a cost that grows slowly with its N (measured on the TF32 kernel: about 50 cycles + 0.43 per column), so N = 128
+// Two things hold the one-tile kernel (128 x 128 tiles, two CTAs per SM) back at 50,432 rows.  One thread gets an
+// MMA instruction accepted only about every 150 cycles whatever its N (measured with a stand-alone loop), so N = 128
 // leaves tensor throughput on the table that N = 256 gets.  And the epilogue of one tile overlaps the main loop of
 // another only by chance: CTAs that start together stay in step, contend for the tensor pipe during their main
 // loops and for the ALUs during their epilogues; for the 768 -> 3072 layer with GELU the epilogue costs about as

@@ -1,7 +1,8 @@
 // Device side of the library: layer construction, the forward kernels and their launch logic.
 //
-// Two device layouts are built from the caller's condensed arrays (values / column indices, both
-// n_active x k, as in the paper's appendix "Condensed matrix multiplication"):
+// Up to three device layouts are built from the caller's condensed arrays (values / column indices, both
+// n_active x k, as in the paper's appendix "Condensed matrix multiplication"); the dense copy for the tensor-core
+// variants is the third (see cfi_dense_tc.cuh and cfi_dense_split.cuh):
 //
 //   small-batch ("split-k") layout: columns stored in 16 bits for long index streams of layers narrower than 65,536
 //     inputs, else in 32; rows padded to a multiple of 8 entries (4 for fp32 values with 32-bit columns) so that
