@@ -257,7 +257,7 @@ cfi_status_t cfi_forward_variant(const cfi_layer_t* layer, const void* x, void* 
  * cfi_forward_dense — CFI_VARIANT_DENSE_TC with the launch shape chosen by the caller (tests and sweeps; the paper
  * has no counterpart).  0 leaves a value to the library.
  *
- *   fp32 layers   tile = batch rows per tile: 16, 32, 64 or 128;  cluster = CTAs that share one tile by splitting K
+ *   fp32 layers   tile = batch rows per tile: 16, 32, 48, 64, 96 or 128;  cluster = CTAs that share one tile by splitting K
  *                 over a thread-block cluster, 1 .. 8
  *   bf16 layers   tile = outputs per tile: 128 (one tile per CTA; cluster 1 .. 8 as above) or 256 (persistent kernel;
  *                 cluster must be 0 or 1)
@@ -307,7 +307,7 @@ cfi_status_t cfi_choose_variant(const cfi_layer_t* layer, int32_t batch, int32_t
 
 /*
  * Launch shape CFI_VARIANT_DENSE_TC would use for this batch size, in the terms of cfi_forward_dense: *tile_n = batch
- * rows per tile (16, 32, 64 or 128) for fp32 layers, outputs per tile (128, or 256 for the persistent kernel) for bf16
+ * rows per tile (16, 32, 48, 64, 96 or 128) for fp32 layers, outputs per tile (128, or 256 for the persistent kernel) for bf16
  * layers; *cluster = the number of CTAs that share one tile by splitting K over a thread-block cluster (1 .. 8).
  * An introspection call for tests and benchmarks; the paper has no counterpart.
  * CFI_ERR_SHAPE if the layer has no dense copy (see CFI_VARIANT_DENSE_TC), CFI_ERR_NULL on a NULL argument.

@@ -45,12 +45,19 @@
 // the K blocks, leaves its partial tile [BT][128] in its shared memory, and after the hardware cluster barrier sums its
 // share of the batch rows over all CTAs in rank order through distributed shared memory.  No flags, no workspace, a
 // fixed order of additions, and the layer stays read-only.
-// Every mbarrier wait is bounded (status code 2); tensor memory is freed on every path.
+// Every mbarrier wait is bounded (status code 2).  After a wait that gave up the CTA still waits, bounded again, for the
+// boxes it has requested and for the MMAs it has issued before it frees its tensor memory and ends.
 
 constexpr int kSpM = 128, kSpK = 32;
 constexpr int kSpTeamWarps = 8, kSpTeams = 2, kSpWorkerWarps = kSpTeams * kSpTeamWarps, kSpFirstWorker = 3;
 constexpr int kSpThreads = 32 * (kSpFirstWorker + kSpWorkerWarps);
-__host__ __device__ constexpr int sp_stages(int bt) { return bt >= 128 ? 4 : bt >= 64 ? 6 : 8; }  // ring depth
+// Batch tiles of the kernel (the MMA's N is BT and 2 BT, multiples of 16 up to 256) and the ring depth each one affords
+// in shared memory (16 KB + 256 BT bytes per stage) and tensor memory (3 BT accumulator columns + 32 per stage).
+constexpr int kSpTiles[] = {16, 32, 48, 64, 96, 128};
+constexpr int kSpNumTiles = sizeof(kSpTiles) / sizeof(kSpTiles[0]);
+// The depth is a multiple of the number of worker teams, so that a ring slot always belongs to the same team: a team
+// that met only every other phase of a slot's barrier could not tell a phase from the one two before it by parity.
+__host__ __device__ constexpr int sp_stages(int bt) { return bt >= 96 ? 4 : bt >= 48 ? 6 : 8; }
 constexpr int kMaxClusterSplit = 8;  // largest portable thread-block cluster
 constexpr uint32_t kSpWBytes = kSpM * kSpK * 4;  // one weight box: 16 KB
 constexpr uint32_t kSpTmemCols = 512;            // 3 BT accumulator columns ... one 32-column w_lo stage per ring slot at the top
@@ -92,6 +99,51 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 // What the hi part (v itself, of which the tensor core reads the upper 19 bits) leaves over: exact in fp32.
 __device__ __forceinline__ float tf32_lo(float v) { return v - __uint_as_float(__float_as_uint(v) & 0xFFFFE000u); }
 
+// The cluster reduction of a K split, for a cluster of NS CTAs: batch rows [split * rows_per, (split + 1) * rows_per)
+// of the tile are summed over the CTAs' partial tiles in rank order, then bias, activation, store.  32 threads per
+// batch row (4 outputs each), 16 rows per pass, 512-byte runs of y.  The loads of kRows rows (NS each; the CTA's own tile
+// is read as ordinary shared memory) are all issued before the first sum needs one, so that the latency of distributed
+// shared memory is paid once per kRows rows.
+template <int BT, int NS>
+__device__ __forceinline__ void sp_reduce(const DevLayer& L, float* __restrict__ y, int batch, int n0, int b0, uint32_t base, int split,
+                                          int wt) {
+    constexpr int kRows = NS <= 2 ? 4 : NS <= 4 ? 2 : 1;
+    const int ch = wt & 31, rows_per = (BT + NS - 1) / NS, o = n0 + 4 * ch;
+    if (o >= L.out) return;
+    const float4 bv = __ldg(reinterpret_cast<const float4*>(L.bias + o));
+    const bool gelu = L.act == CFI_ACT_GELU_ERF;
+    for (int rr0 = wt >> 5; rr0 < rows_per; rr0 += kSpWorkerWarps * kRows) {
+        float4 t[kRows][NS];
+#pragma unroll
+        for (int j = 0; j < kRows; ++j) {
+            const int b = split * rows_per + rr0 + j * kSpWorkerWarps;
+            if (rr0 + j * kSpWorkerWarps < rows_per && b < BT && b0 + b < batch) {
+                const uint32_t off = base + (uint32_t)b * 512u + (uint32_t)ch * 16u;
+#pragma unroll
+                for (int p = 0; p < NS; ++p)
+                    t[j][p] = p == split ? *reinterpret_cast<const float4*>(smem_at(off)) : ld_cluster_f4(smem_u32(off), (uint32_t)p);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kRows; ++j) {
+            const int b = split * rows_per + rr0 + j * kSpWorkerWarps;
+            if (rr0 + j * kSpWorkerWarps < rows_per && b < BT && b0 + b < batch) {
+                float4 a = t[j][0];
+#pragma unroll
+                for (int p = 1; p < NS; ++p) a.x += t[j][p].x, a.y += t[j][p].y, a.z += t[j][p].z, a.w += t[j][p].w;
+                a.x += bv.x, a.y += bv.y, a.z += bv.z, a.w += bv.w;
+                if (gelu) {
+                    a.x = activate(a.x, CFI_ACT_GELU_ERF);
+                    a.y = activate(a.y, CFI_ACT_GELU_ERF);
+                    a.z = activate(a.z, CFI_ACT_GELU_ERF);
+                    a.w = activate(a.w, CFI_ACT_GELU_ERF);
+                }
+                *reinterpret_cast<float4*>(y + (size_t)(b0 + b) * L.out + o) = a;
+            }
+        }
+    }
+}
+
 // Shared memory from the first 1024-byte boundary: kSpStages stages of [Wd box | x box | x_lo]; after the main loop the
 // start of it holds the partial tile when K is split.  Then
 //   +0 full[8] (TMA bytes), +64 ready[8] (x_lo and w_lo written), +128 empty[8] (both issuers done), +192 accumulator
@@ -100,11 +152,12 @@ template <int BT>
 __global__ void __launch_bounds__(kSpThreads, 1)
 cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                        float* __restrict__ y, int batch) {
-    static_assert(BT == 16 || BT == 32 || BT == 64 || BT == 128, "batch tile");
+    static_assert(BT % 16 == 0 && BT >= 16 && BT <= 128, "batch tile");
     constexpr int kSpStages = sp_stages(BT);
     constexpr uint32_t kXBytes = sp_x_bytes(BT), kStageBytes = sp_stage_bytes(BT);
     constexpr uint32_t kABase = kSpTmemCols - 32 * kSpStages;  // accumulators in columns 0 .. 3BT-1, w_lo stages at the top
     static_assert(3 * BT <= kABase, "tensor memory: accumulators + w_lo stages");
+    static_assert(kSpStages % kSpTeams == 0 && kSpStages <= 8, "a ring slot belongs to one team; eight barriers of each kind");
     constexpr int kTeam = 32 * kSpTeamWarps;                    // threads that prepare one block
     constexpr int kVec = (BT * (kSpK / 4) + kTeam - 1) / kTeam; // 16-byte pieces of the x box per worker and block
     pdl_launch_dependents();
@@ -129,8 +182,16 @@ cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, co
         }
         mbar_init(accum, 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // The weight belongs to no earlier kernel: its boxes of the first ring round are requested at once, before the
+        // rest of the set-up and before the wait for the kernel ahead (each stage's barrier already expects the x box
+        // as well).
+        for (int i = 0; i < n_local && i < kSpStages; ++i) {
+            mbar_expect_tx(full0 + 8 * i, kSpWBytes + kXBytes);
+            tma_load_2d(smem_u32(ring + i * kStageBytes), &map_w, full0 + 8 * i, (kb0 + i) * kSpK, n0);
+        }
     }
-    if (warp == 0) {
+    if (warp == 1) {  // meanwhile another warp allocates the tensor memory
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(ctl + 200)), "r"(kSpTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -140,15 +201,10 @@ cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, co
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     bool ok = true;
+    int issued = 0;  // thread 0: K blocks whose boxes it has requested
 
     if (warp == 0 && lane == 0) {
-        // ---------------------------------------------------------------- TMA producer.  The weight belongs to no
-        // earlier kernel: its boxes of the first ring round are requested before the wait for the kernel ahead (each
-        // stage's barrier already expects the x box as well).
-        for (int i = 0; i < n_local && i < kSpStages; ++i) {
-            mbar_expect_tx(full0 + 8 * i, kSpWBytes + kXBytes);
-            tma_load_2d(smem_u32(ring + i * kStageBytes), &map_w, full0 + 8 * i, (kb0 + i) * kSpK, n0);
-        }
+        // ---------------------------------------------------------------- TMA producer.
         // x may belong to the kernel ahead and must not be read before that kernel is done; asking for its first boxes
         // to be brought into L2 reads nothing (L2 is where that kernel's writes land, so nothing stale can be kept),
         // and a cold x is then on chip when the wait returns.  The same for the weight boxes of the second round.
@@ -167,6 +223,7 @@ cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, co
                 tma_load_2d(dst, &map_w, full0 + 8 * s, (kb0 + i) * kSpK, n0);
             }
             tma_load_2d(dst + kSpWBytes, &map_x, full0 + 8 * s, (kb0 + i) * kSpK, b0);
+            issued = i + 1;  // (the first ring round has no wait that could fail, so no stage is left with only its weight box)
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- first MMA issuer: Wd x [x; x_lo], N = 2 BT.
@@ -187,7 +244,7 @@ cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, co
             umma_tf32_ss(tmem_base, dw + 6u, dx + 6u, idesc, 1u);
             umma_commit(empty0 + 8 * s);
         }
-        if (ok) umma_commit(accum);
+        umma_commit(accum);  // also after a failed wait: the arrival then tells when the MMAs issued so far are done
     } else if (warp == 2 && lane == 0) {
         // ---------------------------------------------------------------- second MMA issuer: w_lo x x, N = BT
         constexpr uint32_t idesc = sp_instr_desc(BT);
@@ -205,7 +262,7 @@ cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, co
             umma_tf32_ts(acc, a_lo + 24u, dx + 6u, idesc, 1u);
             umma_commit(empty0 + 8 * s);
         }
-        if (ok) umma_commit(accum);
+        umma_commit(accum);
     } else if (warp >= kSpFirstWorker) {
         // ---------------------------------------------------------------- lo parts, then the epilogue
         const int team = (warp - kSpFirstWorker) / kSpTeamWarps;
@@ -254,13 +311,13 @@ cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, co
         ok = __all_sync(0xffffffffu, ok);
         if (ok) ok = mbar_wait(accum, 0u, kTcSpinLimit);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        constexpr int kColsPerPart = BT >= 64 ? BT / 4 : 16;  // four warps share a lane quarter; narrow tiles use fewer of them
-        if (ok && part * kColsPerPart < BT) {
+        // The four warps of a lane quarter take the 16-column chunks of the tile in turn.
+        if (ok && 16 * part < BT) {
             const int o = n0 + row;
             auto drain = [&](auto gelu_tag) {
                 constexpr bool kGelu = decltype(gelu_tag)::value;
 #pragma unroll 1
-                for (int c0 = part * kColsPerPart; c0 < (part + 1) * kColsPerPart; c0 += 16) {
+                for (int c0 = 16 * part; c0 < BT; c0 += 64) {
                     uint32_t a[3][16];
                     const uint32_t t = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)c0;
 #pragma unroll
@@ -290,44 +347,33 @@ cfi_dense_split_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_w, co
         // Every thread of every CTA of the cluster passes both barriers, whatever `ok` says.
         cluster_sync_all();  // the partial tiles are complete
         if (warp >= kSpFirstWorker && ok) {
-            // Batch rows [split * rows_per, (split + 1) * rows_per) of the tile: sum over the cluster in rank order, bias,
-            // activation, store.  32 threads per batch row (4 outputs each), 16 rows per pass, 512-byte runs of y.
-            const int wt = tid - 32 * kSpFirstWorker, ch = wt & 31, rows_per = (BT + n_split - 1) / n_split, o = n0 + 4 * ch;
-            const float4 bv = o < L.out ? __ldg(reinterpret_cast<const float4*>(L.bias + o)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            const bool gelu = L.act == CFI_ACT_GELU_ERF;
-            for (int rr = wt >> 5; rr < rows_per; rr += kSpWorkerWarps) {
-                const int b = split * rows_per + rr;
-                if (b < BT && b0 + b < batch && o < L.out) {
-                    // All loads of the row are issued before the first sum needs one, so the latency of distributed
-                    // shared memory is paid once per row; the CTA's own tile is read as ordinary shared memory.
-                    const uint32_t off = smem_u32(base + (uint32_t)b * 512u + (uint32_t)ch * 16u);
-                    float4 t[kMaxClusterSplit];
-#pragma unroll
-                    for (int p = 0; p < kMaxClusterSplit; ++p)
-                        if (p < n_split)
-                            t[p] = p == split ? *reinterpret_cast<const float4*>(smem_at(base + (uint32_t)b * 512u + (uint32_t)ch * 16u))
-                                              : ld_cluster_f4(off, (uint32_t)p);
-                    float4 a = t[0];
-#pragma unroll
-                    for (int p = 1; p < kMaxClusterSplit; ++p)
-                        if (p < n_split) a.x += t[p].x, a.y += t[p].y, a.z += t[p].z, a.w += t[p].w;
-                    a.x += bv.x, a.y += bv.y, a.z += bv.z, a.w += bv.w;
-                    if (gelu) {
-                        a.x = activate(a.x, CFI_ACT_GELU_ERF);
-                        a.y = activate(a.y, CFI_ACT_GELU_ERF);
-                        a.z = activate(a.z, CFI_ACT_GELU_ERF);
-                        a.w = activate(a.w, CFI_ACT_GELU_ERF);
-                    }
-                    *reinterpret_cast<float4*>(y + (size_t)(b0 + b) * L.out + o) = a;
-                }
+            const int wt = tid - 32 * kSpFirstWorker;
+            switch (n_split) {
+                case 2: sp_reduce<BT, 2>(L, y, batch, n0, b0, base, split, wt); break;
+                case 3: sp_reduce<BT, 3>(L, y, batch, n0, b0, base, split, wt); break;
+                case 4: sp_reduce<BT, 4>(L, y, batch, n0, b0, base, split, wt); break;
+                case 5: sp_reduce<BT, 5>(L, y, batch, n0, b0, base, split, wt); break;
+                case 6: sp_reduce<BT, 6>(L, y, batch, n0, b0, base, split, wt); break;
+                case 7: sp_reduce<BT, 7>(L, y, batch, n0, b0, base, split, wt); break;
+                default: sp_reduce<BT, 8>(L, y, batch, n0, b0, base, split, wt); break;
             }
         }
         cluster_sync_all_relaxed();  // no CTA leaves while another may still read its tile
     }
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp == 0) {
+    if (__syncthreads_or(!ok)) {
+        // A wait gave up somewhere in this CTA.  It must not end while a box is still on its way into its shared memory
+        // (the copy would land in, and signal a barrier of, whichever CTA gets that memory next) or while an MMA still
+        // works on its tensor memory: wait, again bounded, for the boxes requested and for both issuers' last commit.
+        if (tid == 0) {
+            for (int j = issued > kSpStages ? issued - kSpStages : 0; j < issued; ++j)
+                mbar_wait(full0 + 8 * (j % kSpStages), (uint32_t)(j / kSpStages) & 1u, kTcSpinLimit);
+            mbar_wait(accum, 0u, kTcSpinLimit);
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kSpTmemCols) : "memory");
     }

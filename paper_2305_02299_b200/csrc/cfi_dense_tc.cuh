@@ -28,8 +28,8 @@
 // epilogue overlaps the other's main loop.
 //
 // Every mbarrier wait is bounded.  If one expires the thread records code 2 in the layer's status word and
-// leaves its role's loop; all roles still meet at the final barrier, tensor memory is freed and the kernel
-// returns.
+// leaves its role's loop; all roles still meet at the final barrier, where the CTA waits (bounded) for the boxes
+// still on their way into its shared memory and for its last MMA, then frees tensor memory and returns.
 //
 // With few tiles and a long K the launch may give each tile to a thread-block cluster of up to 8 CTAs (cluster
 // dimension z): CTA r contracts the r-th share of the K blocks and leaves its fp32 partial tile (no bias) in its
@@ -294,6 +294,7 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
     }
     pdl_wait();  // x and y may belong to the kernel before this one
     bool ok = true;
+    int issued = 0;  // thread 0: K blocks whose boxes it has requested
 
     if (warp == 0 && lane == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -305,6 +306,7 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
             if (kb >= kTcStages) mbar_expect_tx(full0 + 8 * s, kTcStageBytes);
             tma_load_2d(a_dst, &map_x, full0 + 8 * s, (kb0 + kb) * kTcK, m0);
             if (kb >= kTcStages) tma_load_2d(b_dst, &map_w, full0 + 8 * s, (kb0 + kb) * kTcK, n0);
+            issued = kb + 1;  // (the first ring round has no wait that could fail, so no stage is left with only its weight box)
         }
     } else if (warp == 1 && lane == 0) {
         // ---------------------------------------------------------------- MMA issuer
@@ -320,7 +322,7 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
                 umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), (kb | k) != 0 ? 1u : 0u);
             umma_commit(empty0 + 8 * s);  // the slot is free once these MMAs have read it
         }
-        if (ok) umma_commit(accum);  // the accumulator is complete once every MMA issued so far has finished
+        umma_commit(accum);  // the accumulator is complete once every MMA issued so far has finished (also after a failed wait)
     } else if (warp >= 2) {
         // ---------------------------------------------------------------- epilogue
         ok = mbar_wait(accum, 0u, kTcSpinLimit);
@@ -410,7 +412,17 @@ cfi_dense_tc_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const
     }
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    if (__syncthreads_or(!ok)) {
+        // A wait gave up somewhere in this CTA.  It must not end while a box is still on its way into its shared memory
+        // (the copy would land in, and signal a barrier of, whichever CTA gets that memory next) or while an MMA still
+        // works on its tensor memory: wait, again bounded, for the boxes requested and for the issuer's last commit.
+        if (tid == 0) {
+            for (int j = issued > kTcStages ? issued - kTcStages : 0; j < issued; ++j)
+                mbar_wait(full0 + 8 * (j % kTcStages), (uint32_t)(j / kTcStages) & 1u, kTcSpinLimit);
+            mbar_wait(accum, 0u, kTcSpinLimit);
+        }
+        __syncthreads();
+    }
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(128u) : "memory");

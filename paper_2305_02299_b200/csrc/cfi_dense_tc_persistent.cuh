@@ -28,7 +28,8 @@
 // Barriers: full/empty per ring slot as in the one-tile kernel, with the phase taken from a running count of K
 // blocks; acc_full[b] (tcgen05.commit after a tile's last MMA) and acc_empty[b] (one arrival per epilogue warp once
 // its tcgen05.ld of the tile have completed).  Every wait is bounded (status code 2); a role that gives up leaves
-// its loop, the roles waiting on it give up in turn, and all meet at the final barrier where tensor memory is freed.
+// its loop, the roles waiting on it give up in turn, and all meet at the final barrier; there the CTA waits (bounded) for
+// the boxes still on their way into its shared memory and for its last MMA, then frees tensor memory and ends.
 
 constexpr int kTpN = 256, kTpStages = 4, kTpEpilogueWarps = 16, kTpThreads = 64 + 32 * kTpEpilogueWarps;
 constexpr uint32_t kTpABytes = kTcM * kTcK * 2, kTpBBytes = kTpN * kTcK * 2, kTpStageBytes = kTpABytes + kTpBBytes;  // 16 + 32 KB
@@ -47,7 +48,7 @@ __device__ __forceinline__ void umma_bf16_n256(uint32_t tmem_d, uint64_t desc_a,
 }
 
 // Shared memory from the first 1024-byte boundary: ring (4 x 48 KB) | two store boxes (2 x 16 KB) | control:
-//   +0 full[4], +32 empty[4], +64 acc_full[2], +80 acc_empty[2], +96 tensor-memory base.
+//   +0 full[4], +32 empty[4], +64 acc_full[2], +80 acc_empty[2], +96 tensor-memory base, +104 the issuer's last commit.
 template <int ACT>
 __global__ void __launch_bounds__(kTpThreads, 1)
 cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
@@ -59,6 +60,7 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
     const uint32_t full0 = smem_u32(ctl), empty0 = smem_u32(ctl + 32), acc_full0 = smem_u32(ctl + 64),
                    acc_empty0 = smem_u32(ctl + 80);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_at(ctl + 96));
+    const uint32_t mma_done = smem_u32(ctl + 104);  // the issuer's last commit: every MMA of this CTA has finished
     const int k_blocks = (L.in + kTcK - 1) / kTcK;
     const int first = blockIdx.x, stride = gridDim.x;
 
@@ -74,6 +76,7 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
             mbar_init(acc_full0 + 8 * b, 1);
             mbar_init(acc_empty0 + 8 * b, kTpEpilogueWarps);
         }
+        mbar_init(mma_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -87,6 +90,7 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();  // x and y may belong to the kernel before this one
     bool ok = true;
+    uint32_t issued = 0;  // thread 0: K blocks whose boxes it has requested
 
     if (warp == 0 && lane == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -101,6 +105,7 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
                 mbar_expect_tx(full0 + 8 * s, kTpStageBytes);
                 tma_load_2d(a_dst, &map_x, full0 + 8 * s, kb * kTcK, m0);
                 tma_load_2d(b_dst, &map_w, full0 + 8 * s, kb * kTcK, n0);
+                issued = g + 1;
             }
         }
     } else if (warp == 1 && lane == 0) {
@@ -126,6 +131,7 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
             }
             if (ok) umma_commit(acc_full0 + 8 * b);  // tile i is complete once every MMA issued so far has finished
         }
+        umma_commit(mma_done);
     } else if (warp >= 2) {
         // ---------------------------------------------------------------- epilogue
         const int et = tid - 64;
@@ -187,7 +193,17 @@ cfi_dense_tc_persistent_kernel(DevLayer L, const __grid_constant__ CUtensorMap m
     }
     if (!ok) atomicExch(L.status, 2);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    if (__syncthreads_or(!ok)) {
+        // A wait gave up somewhere in this CTA.  It must not end while a box is still on its way into its shared memory
+        // (the copy would land in, and signal a barrier of, whichever CTA gets that memory next) or while an MMA still
+        // works on its tensor memory: wait, again bounded, for the boxes requested and for the issuer's last commit.
+        if (tid == 0) {
+            for (uint32_t j = issued > (uint32_t)kTpStages ? issued - kTpStages : 0u; j < issued; ++j)
+                mbar_wait(full0 + 8 * (j % kTpStages), (j / kTpStages) & 1u, kTcSpinLimit);
+            mbar_wait(mma_done, 0u, kTcSpinLimit);
+        }
+        __syncthreads();
+    }
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTpTmemCols) : "memory");

@@ -278,7 +278,8 @@ __global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* _
     // The first row's weights and indices depend neither on x nor on the kernel before this one.  The whole row
     // is asked into L2 by one lane, and its first vectors are requested into registers, before anything else,
     // so the weight stream is in flight while x is awaited and staged.
-    if (lg == 0 && r >= 0) {
+    const bool long_row = nvec > G * U;  // else the first units of the lanes are the whole row: nothing left to ask for
+    if (lg == 0 && r >= 0 && long_row) {
         prefetch_l2(reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp, (uint32_t)(L.kp * sizeof(VT)));
         prefetch_l2(static_cast<const unsigned char*>(L.indices) + (size_t)r * L.kp * kIdxBytes, (uint32_t)L.kp * kIdxBytes);
     }
@@ -365,7 +366,7 @@ __global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* _
         if (more) {
             o += groups;
             r = o < L.out ? (dense_rows ? o : L.slot[o]) : -1;
-            if (lg == 0 && r >= 0) {
+            if (lg == 0 && r >= 0 && long_row) {
                 prefetch_l2(reinterpret_cast<const VT*>(L.values) + (size_t)r * L.kp, (uint32_t)(L.kp * sizeof(VT)));
                 prefetch_l2(static_cast<const unsigned char*>(L.indices) + (size_t)r * L.kp * kIdxBytes, (uint32_t)L.kp * kIdxBytes);
             }
@@ -940,9 +941,13 @@ constexpr int kMaxSplit = kMaxClusterSplit;
 // wave pays it again), the cluster reduction when K is split, and the launch itself.  The dense weight pieces
 // (4 bytes per dense entry) have to come from HBM at least once per call.
 constexpr double kSplitLaunch = 0.7e-6, kSplitWave = 4.2e-6, kSplitHbmBytesPerSecond = 5.5e12;
-double split_seconds_per_block(int bt) { return bt >= 128 ? 0.51e-6 : bt >= 64 ? 0.42e-6 : 0.31e-6; }  // the issue of 4 + 4 MMAs and a commit
+double split_seconds_per_block(int bt) { return bt >= 128 ? 0.51e-6 : bt >= 96 ? 0.40e-6 : 0.31e-6; }  // the issue of 4 + 4 MMAs and a commit
 double split_seconds_reduce(int bt) { return 0.5e-6 + 0.95e-6 * bt / 128.0; }
-int split_bt_index(int bt) { return bt >= 128 ? 3 : bt >= 64 ? 2 : bt >= 32 ? 1 : 0; }
+int split_bt_index(int bt) {
+    for (int i = 0; i < kSpNumTiles; ++i)
+        if (kSpTiles[i] == bt) return i;
+    return -1;
+}
 
 template <int BT>
 int split_query_clusters(const cfi_layer* l, int split) {
@@ -967,16 +972,21 @@ int split_query_clusters(const cfi_layer* l, int split) {
 // Clusters of `split` CTAs of the split-TF32 kernel that the device can hold at once; 0 if it cannot launch that
 // cluster size (cached per device; -1 in the cache stands for 0).
 int split_resident_clusters(const cfi_layer* l, int bt, int split) {
-    static std::atomic<int> cache[kMaxDevices][4][kMaxSplit + 1];
+    static std::atomic<int> cache[kMaxDevices][kSpNumTiles][kMaxSplit + 1];
     if (split == 1) return std::max(1, l->sm_count);
-    if (l->device < 0 || l->device >= kMaxDevices) return 0;
-    std::atomic<int>& c = cache[l->device][split_bt_index(bt)][split];
+    const int ti = split_bt_index(bt);
+    if (l->device < 0 || l->device >= kMaxDevices || ti < 0) return 0;
+    std::atomic<int>& c = cache[l->device][ti][split];
     int v = c.load(std::memory_order_acquire);
     if (v == 0) {
-        v = bt >= 128  ? split_query_clusters<128>(l, split)
-            : bt >= 64 ? split_query_clusters<64>(l, split)
-            : bt >= 32 ? split_query_clusters<32>(l, split)
-                       : split_query_clusters<16>(l, split);
+        switch (bt) {
+            case 16: v = split_query_clusters<16>(l, split); break;
+            case 32: v = split_query_clusters<32>(l, split); break;
+            case 48: v = split_query_clusters<48>(l, split); break;
+            case 64: v = split_query_clusters<64>(l, split); break;
+            case 96: v = split_query_clusters<96>(l, split); break;
+            default: v = split_query_clusters<128>(l, split); break;
+        }
         if (v <= 0) v = -1;
         c.store(v, std::memory_order_release);
     }
@@ -984,7 +994,7 @@ int split_resident_clusters(const cfi_layer* l, int bt, int split) {
 }
 
 struct SplitShape {
-    int bt;          // batch rows per tile: 16, 32, 64 or 128 (the MMA's N is twice that)
+    int bt;          // batch rows per tile: one of kSpTiles (the MMA's N is twice that)
     int split;       // CTAs per output tile (cluster size along z): 1 .. 8
     double seconds;  // modelled time of the launch
     bool ok;
@@ -997,7 +1007,7 @@ SplitShape split_shape(const cfi_layer* l, int batch, int force_bt = 0, int forc
     const int k_blocks = (l->d.in + kSpK - 1) / kSpK, tiles_m = (l->d.out + kSpM - 1) / kSpM;
     const double t_hbm = 4.0 * l->out_pad * (double)l->d.in / kSplitHbmBytesPerSecond;
     SplitShape best{128, 1, 0.0, false};
-    for (int bt = 16; bt <= 128; bt <<= 1) {
+    for (int bt : kSpTiles) {
         if (force_bt && bt != force_bt) continue;
         const int64_t tiles_b = (batch + bt - 1) / bt;
         if (tiles_b > 65535) continue;
@@ -1027,14 +1037,16 @@ cfi_status_t launch_dense_split_bt(const cfi_layer* l, int split, const void* x,
 
 cfi_status_t launch_dense_split(const cfi_layer* l, const void* x, void* y, int batch, cudaStream_t st, int force_bt = 0,
                                 int force_split = 0) {
-    if (force_bt && force_bt != 16 && force_bt != 32 && force_bt != 64 && force_bt != 128) return CFI_ERR_SHAPE;
+    if (force_bt && split_bt_index(force_bt) < 0) return CFI_ERR_SHAPE;
     if (force_split < 0 || force_split > kMaxSplit) return CFI_ERR_SHAPE;
     const SplitShape sh = split_shape(l, batch, force_bt, force_split);
     if (!sh.ok) return CFI_ERR_SHAPE;
     switch (sh.bt) {
         case 16: return launch_dense_split_bt<16>(l, sh.split, x, y, batch, st);
         case 32: return launch_dense_split_bt<32>(l, sh.split, x, y, batch, st);
+        case 48: return launch_dense_split_bt<48>(l, sh.split, x, y, batch, st);
         case 64: return launch_dense_split_bt<64>(l, sh.split, x, y, batch, st);
+        case 96: return launch_dense_split_bt<96>(l, sh.split, x, y, batch, st);
         default: return launch_dense_split_bt<128>(l, sh.split, x, y, batch, st);
     }
 }

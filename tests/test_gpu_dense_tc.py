@@ -31,14 +31,14 @@ def test_dense_tc_matches_oracle(in_f, out_f, k, nabl, B, act, dtype):
     assert_parity(y, y_ref, S, dtype)
 
 
-# fp32: every batch tile (16, 32, 64, 128 rows; the MMAs are 2 x and 1 x that wide) with and without a K split over a
+# fp32: every batch tile (16, 32, 48, 64, 96, 128 rows; the MMAs are 2 x and 1 x that wide) with and without a K split over a
 # thread-block cluster, on shapes with ragged output, batch and K tails, few and many K blocks per CTA (more blocks
 # than ring stages, fewer blocks than CTAs of the cluster), ablated rows and both activations.
 SPLIT_SHAPES = [(768, 384, 77, 19, 200, "gelu"), (3072, 200, 307, 20, 70, "none"), (1000, 72, 100, 5, 257, "gelu"),
                 (520, 640, 52, 30, 129, "none"), (64, 8, 5, 1, 5, "gelu"), (40, 136, 1, 7, 33, "none")]
 
 
-@pytest.mark.parametrize("tile", [16, 32, 64, 128])
+@pytest.mark.parametrize("tile", [16, 32, 48, 64, 96, 128])
 @pytest.mark.parametrize("cluster", [1, 2, 3, 4, 8])
 def test_dense_split_tf32_every_launch_shape(tile, cluster):
     from paper_2305_02299_b200 import binding as cfi
@@ -63,11 +63,11 @@ def test_dense_split_tf32_shape_choice_and_bad_shapes():
     seen = set()
     for B in (9, 16, 40, 64, 100, 256, 700):
         tile, cluster = cfi.cfi_dense_tile_shape(dl, B)
-        assert tile in (16, 32, 64, 128) and 1 <= cluster <= 8
+        assert tile in (16, 32, 48, 64, 96, 128) and 1 <= cluster <= 8
         seen.add((tile, cluster))
     assert len({c for _, c in seen}) >= 2 and len({t for t, _ in seen}) >= 2, seen   # few output tiles, long K: K is split
     x = inputs.make_x(16, 3072)
-    for tile, cluster in ((48, 1), (256, 1), (64, 9), (64, -1)):
+    for tile, cluster in ((40, 1), (256, 1), (64, 9), (64, -1)):
         with pytest.raises(cfi.CfiError) as e:
             run_device(dl, x, "f32", dense_shape=(tile, cluster))
         assert e.value.status == 2
