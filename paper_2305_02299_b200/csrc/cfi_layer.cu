@@ -290,6 +290,14 @@ __global__ void __launch_bounds__(512) cfi_splitk_kernel(DevLayer L, const VT* _
         ck[u].load(L.values, L.indices, (size_t)max(r, 0) * L.kp, v, r >= 0 && v < nvec, L.in);
     }
     float bias = o < L.out ? L.bias[o] : 0.0f;
+    // x may belong to the kernel ahead and must not be read before that kernel is done; asking for it to be brought
+    // into L2 reads nothing (L2 is where that kernel's writes land, so nothing stale can be kept), and a cold x is
+    // then on chip when the wait returns.  The first CTAs of a batch tile ask, 16 KB per thread.
+    if (blockIdx.x < 2 && ((size_t)L.in * sizeof(VT)) % 16 == 0) {
+        const size_t bytes = (size_t)nb * L.in * sizeof(VT), off = (size_t)tid << 14;
+        if (off < bytes)
+            prefetch_l2(reinterpret_cast<const unsigned char*>(x + (size_t)b0 * L.in) + off, (uint32_t)min(bytes - off, (size_t)1 << 14));
+    }
 
     pdl_wait();
     // Stage the CTA's x rows, widened to fp32, transposed to [column][b].  Loads are issued kXStage at a time
