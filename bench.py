@@ -500,8 +500,8 @@ def main():
 VARIANT_NAMES = {1: "simple", 2: "splitk", 3: "batch", 4: "dense_tc", 5: "slab"}
 # DRAM bytes (read + written) of one launch from an ncu capture, keyed by (workload, kernel, launch shape); see profiles/.
 CAPTURED_TRAFFIC = {
-    # profiles/cfi_dense_split_kernel_c2_768x3072_k77_b256.md: 10.285 MB read (dense copy + x), 0 written (y still in L2)
-    ("c2", "cfi_dense_split_kernel<128>", json.dumps({"batch_tile": 128, "cluster_k_split": 2})): 10.285e6,
+    # profiles/cfi_dense_split_kernel_c2_768x3072_k77_b256.md: 10.307 MB read (dense copy + x), 0 written (y still in L2)
+    ("c2", "cfi_dense_split_kernel<96>", json.dumps({"batch_tile": 96, "cluster_k_split": 2})): 10.307e6,
 }
 
 
