@@ -728,7 +728,8 @@ SplitkShape splitk_shape(const cfi_layer* l, int batch) {
     if (fit <= 2 && lanes >= (int64_t)l->sm_count * 512) s.threads = 512;
     const int groups = s.threads / s.g;
     const int ctas_one_row_each = (l->d.out + groups - 1) / groups;
-    const int target = l->sm_count * fit;
+    s.grid_y = (batch + s.bt - 1) / s.bt;
+    const int target = std::max(1, l->sm_count * fit / s.grid_y);  // the batch tiles share the wave
     s.rows_per_group = std::max(1, (ctas_one_row_each + target - 1) / target);
     // x loads in flight per staging thread: 8 when 4 would need more than one round and the grid is small enough
     // that the extra registers do not cost a wave.

@@ -57,6 +57,13 @@ cfi_slab_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int ba
     // and where its quads start in each of this CTA's slabs (an ablated row has none).  Then every row's run of quads
     // is asked into L2 at once.  None of this belongs to an earlier kernel, so it all happens before the wait.
     const int nsl = slab_hi - slab_lo;
+    // Every row's quads (all slabs: the cluster's CTAs need them between them) are asked into L2 by the first CTA of the
+    // cluster, straight from the row table in global memory, while the metadata below is still on its way.
+    if (split == 0)
+        for (int i = tid; i < nrows; i += kSlabThreads) {
+            const int r = L.slot[o0 + i];
+            if (r >= 0) prefetch_l2(wq + (size_t)r * L.stride_q * 2, (uint32_t)L.stride_q * 32u);
+        }
     int32_t* slot_s = reinterpret_cast<int32_t*>(part + (size_t)rows_pc * kSlabBT);
     int32_t* seg_s = slot_s + rows_pc;  // [rows_pc][nsl + 1]
     {
@@ -80,10 +87,6 @@ cfi_slab_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int ba
         }
     }
     __syncthreads();
-    for (int i = tid; i < nrows; i += kSlabThreads) {
-        const int r = slot_s[i], q0 = seg_s[i * (nsl + 1)], q1 = seg_s[i * (nsl + 1) + nsl];
-        if (r >= 0 && q1 > q0) prefetch_l2(wq + ((size_t)r * L.stride_q + q0) * 2, (uint32_t)(q1 - q0) * 32u);
-    }
     // x may belong to the kernel ahead and must not be read before that kernel is done; asking for this CTA's part of
     // it to be brought into L2 reads nothing (L2 is where that kernel's writes land, so nothing stale can be kept), and
     // a cold x is then on chip when the wait returns.  One request per batch row; addresses and sizes rounded to 16 bytes.
