@@ -224,10 +224,46 @@ __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* gr
     }
 }
 
+// A thread's run of 16 consecutive positions from `base`: kind (0: in neither pool, 1: active weight, 2: inactive position
+// of a live neuron) and key of each.  When the run lies inside one row and the arrays allow 16-byte loads it takes one
+// load of the 16 mask bytes and 16-byte loads of only those groups of four weights / gradients that are needed.
+__device__ __forceinline__ void load_run16(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
+                                           long long n, long long base, bool vec_ok, unsigned int (&keys)[16], uint8_t (&kind)[16]) {
+    if (vec_ok && base + 16 <= n) {
+        const uint4 m16 = *reinterpret_cast<const uint4*>(mask + base);
+        const unsigned int mw[4] = {m16.x, m16.y, m16.z, m16.w};
+        const bool live = row_count[(unsigned int)((unsigned long long)base / (unsigned int)in_f)] != 0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const unsigned int nz = __vcmpne4(mw[g], 0u);  // 0xff per nonzero mask byte
+            float4 wv = make_float4(0.f, 0.f, 0.f, 0.f), gv = wv;
+            if (nz != 0u) wv = *reinterpret_cast<const float4*>(w + base + 4 * g);
+            if (nz != 0xFFFFFFFFu && live) gv = *reinterpret_cast<const float4*>(grad + base + 4 * g);
+            const float we[4] = {wv.x, wv.y, wv.z, wv.w}, ge[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool on = ((nz >> (8 * e)) & 1u) != 0u;
+                kind[4 * g + e] = on ? 1 : live ? 2 : 0;
+                keys[4 * g + e] = on ? mag_bits(we[e]) : live ? ~mag_bits(ge[e]) : 0u;
+            }
+        }
+        return;
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        kind[e] = 0, keys[e] = 0;
+        const long long p = base + e;
+        if (p < n) {
+            if (mask[p]) kind[e] = 1, keys[e] = mag_bits(w[p]);
+            else if (row_count[(unsigned int)((unsigned long long)p / (unsigned int)in_f)] != 0) kind[e] = 2, keys[e] = ~mag_bits(grad[p]);
+        }
+    }
+}
+
 // After the four passes prefix is the key of the cut and `want` of the elements equal to it are taken, the first ones
 // in position order.  Per chunk of kChunk positions and per selection: how many equal the cut key.
 __global__ void tie_count_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
-                                 long long n, const SelectState* st, unsigned int* chunk_ties, int n_chunks) {
+                                 long long n, const SelectState* st, unsigned int* chunk_ties, int n_chunks, bool vec_ok) {
     __shared__ unsigned int s[2];
     if (threadIdx.x < 2) s[threadIdx.x] = 0;
     __syncthreads();
@@ -235,13 +271,13 @@ __global__ void tie_count_kernel(const float* w, const uint8_t* mask, const floa
     const bool on0 = st[0].want != 0, on1 = st[1].want != 0;
     const unsigned int cut0 = st[0].prefix, cut1 = st[1].prefix;
     unsigned int c0 = 0, c1 = 0;
+    unsigned int keys[16];
+    uint8_t kind[16];
+    load_run16(w, mask, grad, row_count, in_f, n, base, vec_ok, keys, kind);
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
-        const long long p = base + e;
-        if (p < n) {
-            if (mask[p]) c0 += (on0 && mag_bits(w[p]) == cut0) ? 1u : 0u;
-            else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) c1 += (on1 && ~mag_bits(grad[p]) == cut1) ? 1u : 0u;
-        }
+        c0 += (kind[e] == 1 && on0 && keys[e] == cut0) ? 1u : 0u;
+        c1 += (kind[e] == 2 && on1 && keys[e] == cut1) ? 1u : 0u;
     }
     if (c0) atomicAdd(&s[0], c0);
     if (c1) atomicAdd(&s[1], c1);
@@ -279,7 +315,7 @@ __global__ void chunk_scan_kernel(unsigned int* chunk_ties_both, int n_chunks) {
 // the first `want` in position order.
 __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f, long long n,
                             const SelectState* st, const unsigned int* chunk_ties, int n_chunks, uint8_t* drop,
-                            uint8_t* grow_top) {
+                            uint8_t* grow_top, bool vec_ok) {
     __shared__ unsigned int part[2][kThreads];
     const long long base = (long long)blockIdx.x * kChunk + (long long)threadIdx.x * 16;
     const unsigned long long want0 = st[0].want, want1 = st[1].want;
@@ -287,14 +323,9 @@ __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* gr
     unsigned int keys[16];
     uint8_t kind[16];  // 0: in neither pool, 1: active weight, 2: inactive position of a live neuron
     unsigned int mine0 = 0, mine1 = 0;
+    load_run16(w, mask, grad, row_count, in_f, n, base, vec_ok, keys, kind);
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
-        kind[e] = 0, keys[e] = 0;
-        const long long p = base + e;
-        if (p < n) {
-            if (mask[p]) kind[e] = 1, keys[e] = mag_bits(w[p]);
-            else if (row_count[(unsigned int)p / (unsigned int)in_f] != 0) kind[e] = 2, keys[e] = ~mag_bits(grad[p]);
-        }
         if (kind[e] == 1 && want0 != 0 && keys[e] == cut0) ++mine0;
         if (kind[e] == 2 && want1 != 0 && keys[e] == cut1) ++mine1;
     }
@@ -312,10 +343,10 @@ __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* gr
     // ties of each selection before this thread's first element
     unsigned long long rank0 = (unsigned long long)chunk_ties[blockIdx.x] + part[0][threadIdx.x] - mine0;
     unsigned long long rank1 = (unsigned long long)chunk_ties[(size_t)n_chunks + blockIdx.x] + part[1][threadIdx.x] - mine1;
+    unsigned int d16[4] = {0u, 0u, 0u, 0u}, g16[4] = {0u, 0u, 0u, 0u};  // the 16 flags of each kind, one byte each
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
-        if (base + e >= n) continue;
-        uint8_t f0 = 0, f1 = 0;
+        unsigned int f0 = 0, f1 = 0;
         if (kind[e] == 1 && want0 != 0) {
             if (keys[e] < cut0) f0 = 1;
             else if (keys[e] == cut0) f0 = rank0++ < want0 ? 1 : 0;
@@ -323,8 +354,19 @@ __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* gr
             if (keys[e] < cut1) f1 = 1;
             else if (keys[e] == cut1) f1 = rank1++ < want1 ? 1 : 0;
         }
-        drop[base + e] = f0;
-        grow_top[base + e] = f1;
+        d16[e >> 2] |= f0 << (8 * (e & 3));
+        g16[e >> 2] |= f1 << (8 * (e & 3));
+    }
+    if (vec_ok && base + 16 <= n) {
+        *reinterpret_cast<uint4*>(drop + base) = make_uint4(d16[0], d16[1], d16[2], d16[3]);
+        *reinterpret_cast<uint4*>(grow_top + base) = make_uint4(g16[0], g16[1], g16[2], g16[3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            if (base + e >= n) continue;
+            drop[base + e] = (uint8_t)((d16[e >> 2] >> (8 * (e & 3))) & 1u);
+            grow_top[base + e] = (uint8_t)((g16[e >> 2] >> (8 * (e & 3))) & 1u);
+        }
     }
 }
 
@@ -581,10 +623,14 @@ bool layer_select_both(const float* w, const uint8_t* mask, const float* grad, c
     for (int pass = 0; pass < 4; ++pass) {
         hist_kernel<<<hist_blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, out_f, in_f, pass, ws.state);
     }
-    tie_count_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks);
+    // 16-byte loads and stores of a thread's run of 16 positions: the run must lie inside one row, and the arrays (the
+    // workspace's flag arrays are 256-byte aligned) must start on 16-byte boundaries.
+    const bool vec_ok = (in_f % 16) == 0 && ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(grad) |
+                                               reinterpret_cast<uintptr_t>(mask)) & 15u) == 0;
+    tie_count_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks, vec_ok);
     chunk_scan_kernel<<<2, kThreads, 0, st>>>(ws.chunk_ties, chunks);
     mark_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks, ws.drop,
-                                             ws.grow_top);
+                                             ws.grow_top, vec_ok);
     return cudaGetLastError() == cudaSuccess;
 }
 
