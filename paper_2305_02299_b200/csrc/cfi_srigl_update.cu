@@ -288,26 +288,39 @@ __global__ void tie_count_kernel(const float* w, const uint8_t* mask, const floa
 // One block per selection: exclusive prefix sum of its per-chunk tie counts, in place.
 __global__ void chunk_scan_kernel(unsigned int* chunk_ties_both, int n_chunks) {
     unsigned int* chunk_ties = chunk_ties_both + (size_t)blockIdx.x * n_chunks;
-    __shared__ unsigned long long carry;
-    __shared__ unsigned int part[kThreads];
-    if (threadIdx.x == 0) carry = 0;
-    __syncthreads();
-    for (int c0 = 0; c0 < n_chunks; c0 += kThreads) {
-        const int c = c0 + threadIdx.x;
-        const unsigned int v = c < n_chunks ? chunk_ties[c] : 0u;
-        part[threadIdx.x] = v;
-        __syncthreads();
-        for (int off = 1; off < kThreads; off <<= 1) {  // inclusive scan of the block's values
-            const unsigned int add = threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
-            __syncthreads();
-            part[threadIdx.x] += add;
-            __syncthreads();
+    __shared__ unsigned long long warp_tot[kThreads / 32];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    // A thread takes 16 consecutive chunks at a time (the block 4096): their sum is scanned over the block with shuffles
+    // and one count per warp, then the thread walks its chunks.
+    unsigned long long carry = 0;
+    for (int c0 = 0; c0 < n_chunks; c0 += 16 * kThreads) {
+        const int first = c0 + 16 * threadIdx.x;
+        unsigned int v[16];
+        unsigned long long mine = 0;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v[e] = first + e < n_chunks ? chunk_ties[first + e] : 0u, mine += v[e];
+        unsigned long long incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
         }
-        const unsigned long long before = carry + part[threadIdx.x] - v;
-        if (c < n_chunks) chunk_ties[c] = (unsigned int)(before > 0xFFFFFFFFull ? 0xFFFFFFFFull : before);
+        if (lane == 31) warp_tot[wid] = incl;
         __syncthreads();
-        if (threadIdx.x == kThreads - 1) carry += part[kThreads - 1];
-        __syncthreads();
+        unsigned long long before = carry + incl - mine, total = 0;
+#pragma unroll
+        for (int i = 0; i < kThreads / 32; ++i) {
+            const unsigned long long p = warp_tot[i];
+            before += i < wid ? p : 0ull;
+            total += p;
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            if (first + e < n_chunks) chunk_ties[first + e] = (unsigned int)(before > 0xFFFFFFFFull ? 0xFFFFFFFFull : before);
+            before += v[e];
+        }
+        carry += total;
+        __syncthreads();  // warp_tot[] is rewritten by the next round
     }
 }
 
@@ -401,11 +414,14 @@ __global__ void ablate_kernel(const int* row_count, const int* salient, int out_
     if (threadIdx.x == 0) after = 0;
     __syncthreads();
     const double threshold = fmax(1.0, (double)gamma_sal * (double)sc->k);
+    int mine = 0;
     for (int r = threadIdx.x; r < out_f; r += blockDim.x) {
         const bool live = row_count[r] > 0 && !((double)salient[r] < threshold);
         survives[r] = live ? 1 : 0;
-        if (live) atomicAdd(&after, 1);
+        mine += live ? 1 : 0;
     }
+    for (int off = 16; off > 0; off >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, off);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&after, mine);
     __syncthreads();
     if (threadIdx.x == 0) {
         sc->live_after = after;
@@ -424,58 +440,50 @@ struct RowCut {
     int any;             // 0: nothing to select
 };
 
-// One warp: the first of 256 shared-memory bins whose running count reaches `want` (the last bin if none before it
-// does) and the count in the bins before it; eight bins per lane, one scan over the lanes.
-__device__ __forceinline__ void row_pick(const unsigned int* hist, unsigned int want, int& bin, unsigned int& below) {
-    const int lane = threadIdx.x & 31;
-    unsigned int v[8], mine = 0;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) v[e] = hist[8 * lane + e], mine += v[e];
-    unsigned int incl = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned int up = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += up;
-    }
-    unsigned int seen = incl - mine;
-    int found = 256;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        if (found == 256) {
-            if (seen + v[e] >= want) found = 8 * lane + e;
-            else seen += v[e];
-        }
-    }
-    bin = found;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) bin = min(bin, __shfl_xor_sync(0xffffffffu, bin, off));
-    if (bin > 255) bin = 255;
-    if (found == 256 && lane == 31) seen -= v[7];  // no bin before the last reaches `want`: the count below the last bin
-    below = __shfl_sync(0xffffffffu, seen, bin >> 3);
-}
-
 template <typename KeyOf>
 __device__ void row_select(int in_f, int m, KeyOf key_of, unsigned int* hist /*256, shared*/, RowCut* out /*shared*/) {
-    __shared__ unsigned int prefix, pmask, want;
+    __shared__ unsigned int prefix, pmask, want, warp_tot[kThreads / 32];
     if (threadIdx.x == 0) prefix = 0, pmask = 0, want = (unsigned int)(m > 0 ? m : 0);
     __syncthreads();
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     for (int pass = 0; pass < 4 && m > 0; ++pass) {
         for (int b = threadIdx.x; b < 256; b += blockDim.x) hist[b] = 0;
         __syncthreads();
         const int shift = 24 - 8 * pass;
         const unsigned int pre = prefix, pm = pmask;
+#pragma unroll 4
         for (int c = threadIdx.x; c < in_f; c += blockDim.x) {
             unsigned int key;
             if (key_of(c, key) && (key & pm) == pre) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
         __syncthreads();
-        if (threadIdx.x < 32) {
-            int b;
-            unsigned int seen;
-            row_pick(hist, want, b, seen);
-            if (threadIdx.x == 0) {
-                want -= seen;
-                prefix |= (unsigned int)b << shift;
+        // The bin that holds the `want`-th element, by the whole block (one bin per thread): the first bin whose running
+        // count reaches `want`, the last bin if none does.  A prefix count over the block (shuffles, then one count per
+        // warp); exactly one thread finds that the running count first reaches `want` in its bin.
+        {
+            const unsigned int h = hist[threadIdx.x], w0 = want;
+            unsigned int incl = h;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned int up = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += up;
+            }
+            if (lane == 31) warp_tot[wid] = incl;
+            __syncthreads();
+            unsigned int before = 0, total = 0;
+#pragma unroll
+            for (int i = 0; i < kThreads / 32; ++i) {
+                const unsigned int p = warp_tot[i];
+                before += i < wid ? p : 0u;
+                total += p;
+            }
+            const unsigned int excl = before + incl - h;
+            const bool here = excl < w0 && w0 <= excl + h;
+            const bool last_none = w0 > total && threadIdx.x == kThreads - 1;
+            __syncthreads();  // every thread has read `want`
+            if (here || last_none) {
+                want = w0 - excl;
+                prefix |= (unsigned int)threadIdx.x << shift;
                 pmask |= 255u << shift;
             }
         }
@@ -577,6 +585,152 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
         }
         carry += in_chunk;
         __syncthreads();  // part[] is rewritten by the next chunk
+    }
+}
+
+// The same step for rows whose length is a multiple of 16, whose arrays start on 16-byte boundaries and whose keys fit
+// in shared memory: a thread owns runs of 16 consecutive columns, so the row costs four dependent trips to memory (the
+// neuron's flag; mask and pruning flags, 16 bytes each; the keys, 16-byte loads of only the groups that hold candidates;
+// the weights once more for the write-back) instead of one per 256 columns and array, ties are ranked with one block-wide
+// prefix count per 4096 columns, and mask and weights go back in whole 16-byte stores.
+__global__ void __launch_bounds__(kThreads, 6) finalize_runs_kernel(float* w, uint8_t* mask, const float* grad, const uint8_t* drop, const uint8_t* survives,
+                                     int in_f, const Scalars* sc) {
+    extern __shared__ __align__(16) unsigned char row_smem[];  // keys[in_f] (4 bytes each), then state[in_f] (1 byte each)
+    __shared__ unsigned int hist[256];
+    __shared__ RowCut cut;
+    __shared__ int kept_count;
+    __shared__ unsigned int warp_tot[kThreads / 32];
+    const int r = blockIdx.x, t = threadIdx.x, lane = t & 31, wid = t >> 5, n_runs = in_f >> 4;
+    float* wr = w + (size_t)r * in_f;
+    uint8_t* mr = mask + (size_t)r * in_f;
+    const float* gr = grad + (size_t)r * in_f;
+    const uint8_t* dr = drop + (size_t)r * in_f;
+    if (!survives[r]) {  // ablated now or before: nothing left
+        for (int j = t; j < n_runs; j += kThreads) {
+            *reinterpret_cast<uint4*>(mr + 16 * j) = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) *reinterpret_cast<float4*>(wr + 16 * j + 4 * g) = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        return;
+    }
+    unsigned int* keys = reinterpret_cast<unsigned int*>(row_smem);
+    uint8_t* state = row_smem + (size_t)in_f * 4;  // 1 = kept after step 6, 0 = free
+    const int k_new = sc->k_new;
+    if (t == 0) kept_count = 0;
+    __syncthreads();
+    int mine = 0;
+    for (int j = t; j < n_runs; j += kThreads) {
+        const uint4 m = *reinterpret_cast<const uint4*>(mr + 16 * j), d = *reinterpret_cast<const uint4*>(dr + 16 * j);
+        uint4 st;  // a byte per column: 1 where the mask is set and the weight was not pruned in step 6
+        st.x = __vcmpne4(m.x, 0u) & __vcmpeq4(d.x, 0u) & 0x01010101u;
+        st.y = __vcmpne4(m.y, 0u) & __vcmpeq4(d.y, 0u) & 0x01010101u;
+        st.z = __vcmpne4(m.z, 0u) & __vcmpeq4(d.z, 0u) & 0x01010101u;
+        st.w = __vcmpne4(m.w, 0u) & __vcmpeq4(d.w, 0u) & 0x01010101u;
+        mine += __popc(st.x) + __popc(st.y) + __popc(st.z) + __popc(st.w);
+        *reinterpret_cast<uint4*>(state + 16 * j) = st;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, off);
+    if (lane == 0 && mine) atomicAdd(&kept_count, mine);
+    __syncthreads();
+    const int kept = kept_count;
+    const bool trim = kept > k_new;
+    const int m = trim ? kept - k_new : k_new - kept;
+    if (m > 0) {
+        const float* src = trim ? wr : gr;
+        const unsigned int flip = trim ? 0u : 0xFFFFFFFFu;  // regrowing: the complement, so that a larger gradient is a smaller key
+        for (int j = t; j < n_runs; j += kThreads) {
+            const uint4 st = *reinterpret_cast<const uint4*>(state + 16 * j);
+            const unsigned int sw[4] = {st.x, st.y, st.z, st.w};
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const unsigned int cand = trim ? sw[g] : (sw[g] ^ 0x01010101u);
+                uint4 kq = make_uint4(0u, 0u, 0u, 0u);
+                if (cand != 0u) {
+                    const float4 v = *reinterpret_cast<const float4*>(src + 16 * j + 4 * g);
+                    kq.x = (cand & 0x00000001u) ? (mag_bits(v.x) ^ flip) : 0u;
+                    kq.y = (cand & 0x00000100u) ? (mag_bits(v.y) ^ flip) : 0u;
+                    kq.z = (cand & 0x00010000u) ? (mag_bits(v.z) ^ flip) : 0u;
+                    kq.w = (cand & 0x01000000u) ? (mag_bits(v.w) ^ flip) : 0u;
+                }
+                *reinterpret_cast<uint4*>(keys + 16 * j + 4 * g) = kq;
+            }
+        }
+        __syncthreads();
+    }
+    auto key_of = [&](int c, unsigned int& key) {
+        key = keys[c];
+        return trim ? state[c] != 0 : state[c] == 0;
+    };
+    row_select(in_f, m, key_of, hist, &cut);
+    // Apply in column order, so that ties on the cut key go to the smaller columns: a tie's rank is the ties of the
+    // 4096-column chunks before (carried by every thread), of the threads before in this chunk (a prefix count over the
+    // block) and of the columns before in the thread's own run.
+    const bool any = cut.any != 0;
+    const unsigned int cut_key = cut.cut, cut_ties = cut.ties;
+    unsigned int carry = 0;
+    for (int j0 = 0; j0 < n_runs; j0 += kThreads) {
+        const int j = j0 + t;
+        const bool have = j < n_runs;
+        uint4 st = make_uint4(0u, 0u, 0u, 0u);
+        float4 wv[4];
+        if (have) {
+            st = *reinterpret_cast<const uint4*>(state + 16 * j);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) wv[g] = *reinterpret_cast<const float4*>(wr + 16 * j + 4 * g);  // in flight during the count
+        }
+        const unsigned int sw[4] = {st.x, st.y, st.z, st.w};
+        unsigned int my_ties = 0;
+        if (have && any) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const uint4 kq = *reinterpret_cast<const uint4*>(keys + 16 * j + 4 * g);
+                const unsigned int cand = trim ? sw[g] : (sw[g] ^ 0x01010101u);
+                my_ties += ((cand & 0x00000001u) && kq.x == cut_key) + ((cand & 0x00000100u) && kq.y == cut_key) +
+                           ((cand & 0x00010000u) && kq.z == cut_key) + ((cand & 0x01000000u) && kq.w == cut_key);
+            }
+        }
+        unsigned int incl = my_ties;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned int up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        if (lane == 31) warp_tot[wid] = incl;
+        __syncthreads();
+        unsigned int rank = carry + incl - my_ties, in_chunk = 0;
+#pragma unroll
+        for (int i = 0; i < kThreads / 32; ++i) {
+            const unsigned int p = warp_tot[i];
+            rank += i < wid ? p : 0u;
+            in_chunk += p;
+        }
+        if (have) {
+            unsigned int mo[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint4 kq = make_uint4(0u, 0u, 0u, 0u);
+                if (any) kq = *reinterpret_cast<const uint4*>(keys + 16 * j + 4 * g);
+                const unsigned int kk[4] = {kq.x, kq.y, kq.z, kq.w};
+                float we[4] = {wv[g].x, wv[g].y, wv[g].z, wv[g].w};
+                mo[g] = 0u;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool is_kept = ((sw[g] >> (8 * e)) & 1u) != 0u;
+                    const bool candidate = trim ? is_kept : !is_kept;
+                    const bool tie = any && candidate && kk[e] == cut_key;
+                    bool selected = any && candidate && kk[e] < cut_key;
+                    if (tie) selected = rank++ < cut_ties;
+                    const bool on = trim ? (is_kept && !selected) : (is_kept || selected);
+                    if (!on || !is_kept) we[e] = 0.0f;  // pruned, trimmed, free, or grown (starts at 0); a survivor keeps its value
+                    mo[g] |= (on ? 1u : 0u) << (8 * e);
+                }
+                *reinterpret_cast<float4*>(wr + 16 * j + 4 * g) = make_float4(we[0], we[1], we[2], we[3]);
+            }
+            *reinterpret_cast<uint4*>(mr + 16 * j) = make_uint4(mo[0], mo[1], mo[2], mo[3]);
+        }
+        carry += in_chunk;
+        __syncthreads();  // warp_tot[] is rewritten by the next chunk
     }
 }
 
@@ -724,7 +878,11 @@ extern "C" cfi_status_t cfi_srigl_update(float* w, uint8_t* mask, const float* g
     salient_kernel<<<out_features, kThreads, 0, st>>>(mask, ws.drop, ws.grow_top, in_features, ws.salient);
     ablate_kernel<<<1, kThreads, 0, st>>>(ws.row_count, ws.salient, out_features, in_features, gamma_sal, ws.scalars, ws.survives);
     const size_t row_bytes = (size_t)in_features * 5;  // keys and one state byte per column
-    if (row_bytes <= 40 * 1024)
+    const bool runs_ok = (in_features % 16) == 0 && ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(grad) |
+                                                         reinterpret_cast<uintptr_t>(mask)) & 15u) == 0;
+    if (row_bytes <= 40 * 1024 && runs_ok && in_features >= 2048)  // shorter rows leave most of a block's threads without a run
+        finalize_runs_kernel<<<out_features, kThreads, row_bytes, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
+    else if (row_bytes <= 40 * 1024)
         finalize_kernel<true><<<out_features, kThreads, row_bytes, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
     else
         finalize_kernel<false><<<out_features, kThreads, 0, st>>>(w, mask, grad, ws.drop, ws.survives, in_features, ws.scalars);
