@@ -55,6 +55,44 @@ def test_dense_split_tf32_every_launch_shape(tile, cluster):
         assert np.array_equal(y, y2)                      # fixed order of additions: the same bits every time
 
 
+@pytest.mark.parametrize("tile,cluster", [(16, 4), (48, 4), (64, 8), (96, 2), (128, 2), (32, 1)])
+def test_dense_split_tf32_chain_of_launches(tile, cluster):
+    """Back-to-back launches (a CUDA graph of 48 calls over 6 rotating layers; each launch lets its successor start
+    early and waits for its predecessor before it reads x): a long K, so that the ring wraps several times per CTA.
+    No wait may give up (status word), and every call must give the bits of the same call made alone."""
+    import torch
+    from paper_2305_02299_b200 import binding as cfi
+    in_f, out_f, k, B, n = 2048, 640, 64, 24, 6
+    layers, xs, ys, alone = [], [], [], []
+    for i in range(n):
+        L = inputs.make_layer(in_f, out_f, k, n_ablated=5, seed=900 + i)
+        x = inputs.make_x(B, in_f, seed=950 + i)
+        dl = device_layer(L, "f32", "gelu" if i % 2 else "none")
+        if i == 0:
+            y_ref, S = oracle_layer(L, x, "f32", "none")
+            assert scaled_error(run_device(dl, x, "f32", dense_shape=(tile, cluster)), y_ref, S) <= TOL["f32"]
+        alone.append(run_device(dl, x, "f32", dense_shape=(tile, cluster)))
+        layers.append(dl)
+        xs.append(torch.from_numpy(x).cuda())
+        ys.append(torch.empty((B, out_f), device="cuda"))
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i in range(n):
+            cfi.cfi_forward_dense(layers[i], xs[i], ys[i], B, tile=tile, cluster=cluster)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for j in range(48):
+                cfi.cfi_forward_dense(layers[j % n], xs[j % n], ys[j % n], B, tile=tile, cluster=cluster)
+        for _ in range(5):
+            graph.replay()
+        stream.synchronize()
+    for i in range(n):
+        assert cfi.cfi_device_status(layers[i]) == 0, (i, tile, cluster)
+        assert np.array_equal(ys[i].double().cpu().numpy(), alone[i]), (i, tile, cluster)
+        layers[i].close()
+
+
 def test_dense_split_tf32_shape_choice_and_bad_shapes():
     """The shape the library picks is one of the allowed ones and runs; values outside the sets are refused."""
     from paper_2305_02299_b200 import binding as cfi
