@@ -79,8 +79,14 @@ __global__ void setup_kernel(const int* row_count, int out_f, int in_f, long lon
     __syncthreads();
     long long my_act = 0;
     int my_live = 0, my_k = 0;
-    for (int r = threadIdx.x; r < out_f; r += blockDim.x)
-        if (row_count[r] > 0) my_act += row_count[r], ++my_live, my_k = max(my_k, row_count[r]);
+    for (int r0 = threadIdx.x; r0 < out_f; r0 += 8 * blockDim.x) {  // eight rows' loads in flight
+        int rc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) rc[u] = r0 + u * blockDim.x < out_f ? row_count[r0 + u * blockDim.x] : 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (rc[u] > 0) my_act += rc[u], ++my_live, my_k = max(my_k, rc[u]);
+    }
     for (int off = 16; off > 0; off >>= 1) {  // one set of atomics per warp
         my_act += __shfl_down_sync(0xffffffffu, my_act, off);
         my_live += __shfl_down_sync(0xffffffffu, my_live, off);
@@ -188,10 +194,10 @@ __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* gr
                     const bool inside = v < n4;
                     uchar4 m = make_uchar4(0, 0, 0, 0);
                     float4 wv = make_float4(0.f, 0.f, 0.f, 0.f), gv = wv;
-                    if (inside) {
+                    if (inside) {  // all three at once: a load that waited for the mask would cost a second trip to memory
                         m = m4[v];
-                        if (m.x | m.y | m.z | m.w) wv = w4[v];
-                        if (!(m.x && m.y && m.z && m.w)) gv = g4[v];
+                        wv = w4[v];
+                        gv = g4[v];
                     }
                     one(inside, m.x, wv.x, gv.x);
                     one(inside, m.y, wv.y, gv.y);
@@ -226,19 +232,24 @@ __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* gr
 
 // A thread's run of 16 consecutive positions from `base`: kind (0: in neither pool, 1: active weight, 2: inactive position
 // of a live neuron) and key of each.  When the run lies inside one row and the arrays allow 16-byte loads it takes one
-// load of the 16 mask bytes and 16-byte loads of only those groups of four weights / gradients that are needed.
+// load of the 16 mask bytes and four 16-byte loads each of the weights and the gradients, all requested together.
 __device__ __forceinline__ void load_run16(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
                                            long long n, long long base, bool vec_ok, unsigned int (&keys)[16], uint8_t (&kind)[16]) {
     if (vec_ok && base + 16 <= n) {
+        // Everything is requested at once: a load that waited for the mask would cost a second trip to memory.
         const uint4 m16 = *reinterpret_cast<const uint4*>(mask + base);
+        float4 w16[4], g16[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            w16[g] = *reinterpret_cast<const float4*>(w + base + 4 * g);
+            g16[g] = *reinterpret_cast<const float4*>(grad + base + 4 * g);
+        }
         const unsigned int mw[4] = {m16.x, m16.y, m16.z, m16.w};
         const bool live = row_count[(unsigned int)((unsigned long long)base / (unsigned int)in_f)] != 0;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
             const unsigned int nz = __vcmpne4(mw[g], 0u);  // 0xff per nonzero mask byte
-            float4 wv = make_float4(0.f, 0.f, 0.f, 0.f), gv = wv;
-            if (nz != 0u) wv = *reinterpret_cast<const float4*>(w + base + 4 * g);
-            if (nz != 0xFFFFFFFFu && live) gv = *reinterpret_cast<const float4*>(grad + base + 4 * g);
+            const float4 wv = w16[g], gv = g16[g];
             const float we[4] = {wv.x, wv.y, wv.z, wv.w}, ge[4] = {gv.x, gv.y, gv.z, gv.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -391,7 +402,18 @@ __global__ void salient_kernel(const uint8_t* mask, const uint8_t* drop, const u
     __syncthreads();
     int c = 0;
     const size_t base = (size_t)r * in_f;
-    if ((in_f & 3) == 0) {
+    if ((in_f & 15) == 0 && (reinterpret_cast<uintptr_t>(mask) & 15u) == 0) {  // (the flag arrays are 256-byte aligned)
+        const uint4 *m16 = reinterpret_cast<const uint4*>(mask + base), *d16 = reinterpret_cast<const uint4*>(drop + base),
+                    *g16 = reinterpret_cast<const uint4*>(grow_top + base);
+        for (int v = threadIdx.x; v < (in_f >> 4); v += blockDim.x) {
+            const uint4 m = m16[v], d = d16[v], g = g16[v];
+            // a byte is salient if (mask set and not dropped) or among the top gradients
+            c += (__popc((__vcmpne4(m.x, 0u) & __vcmpeq4(d.x, 0u)) | __vcmpne4(g.x, 0u)) +
+                  __popc((__vcmpne4(m.y, 0u) & __vcmpeq4(d.y, 0u)) | __vcmpne4(g.y, 0u)) +
+                  __popc((__vcmpne4(m.z, 0u) & __vcmpeq4(d.z, 0u)) | __vcmpne4(g.z, 0u)) +
+                  __popc((__vcmpne4(m.w, 0u) & __vcmpeq4(d.w, 0u)) | __vcmpne4(g.w, 0u))) >> 3;
+        }
+    } else if ((in_f & 3) == 0) {
         const uchar4 *m4 = reinterpret_cast<const uchar4*>(mask + base), *d4 = reinterpret_cast<const uchar4*>(drop + base),
                      *g4 = reinterpret_cast<const uchar4*>(grow_top + base);
         for (int v = threadIdx.x; v < (in_f >> 2); v += blockDim.x) {
@@ -415,10 +437,22 @@ __global__ void ablate_kernel(const int* row_count, const int* salient, int out_
     __syncthreads();
     const double threshold = fmax(1.0, (double)gamma_sal * (double)sc->k);
     int mine = 0;
-    for (int r = threadIdx.x; r < out_f; r += blockDim.x) {
-        const bool live = row_count[r] > 0 && !((double)salient[r] < threshold);
-        survives[r] = live ? 1 : 0;
-        mine += live ? 1 : 0;
+    for (int r0 = threadIdx.x; r0 < out_f; r0 += 8 * blockDim.x) {  // eight rows' loads in flight: one block walks all rows
+        int rc[8], sa[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int r = r0 + u * blockDim.x;
+            rc[u] = r < out_f ? row_count[r] : 0, sa[u] = r < out_f ? salient[r] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int r = r0 + u * blockDim.x;
+            if (r < out_f) {
+                const bool live = rc[u] > 0 && !((double)sa[u] < threshold);
+                survives[r] = live ? 1 : 0;
+                mine += live ? 1 : 0;
+            }
+        }
     }
     for (int off = 16; off > 0; off >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, off);
     if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&after, mine);
