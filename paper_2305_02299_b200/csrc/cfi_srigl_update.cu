@@ -474,8 +474,10 @@ struct RowCut {
     int any;             // 0: nothing to select
 };
 
-template <typename KeyOf>
-__device__ void row_select(int in_f, int m, KeyOf key_of, unsigned int* hist /*256, shared*/, RowCut* out /*shared*/) {
+// `count(prefix, prefix_mask, shift)` adds to hist[(key >> shift) & 255], with shared-memory atomics, every candidate of
+// the row whose key matches the prefix found so far.
+template <typename Count>
+__device__ void row_select(int m, Count count, unsigned int* hist /*256, shared*/, RowCut* out /*shared*/) {
     __shared__ unsigned int prefix, pmask, want, warp_tot[kThreads / 32];
     if (threadIdx.x == 0) prefix = 0, pmask = 0, want = (unsigned int)(m > 0 ? m : 0);
     __syncthreads();
@@ -484,12 +486,7 @@ __device__ void row_select(int in_f, int m, KeyOf key_of, unsigned int* hist /*2
         for (int b = threadIdx.x; b < 256; b += blockDim.x) hist[b] = 0;
         __syncthreads();
         const int shift = 24 - 8 * pass;
-        const unsigned int pre = prefix, pm = pmask;
-#pragma unroll 4
-        for (int c = threadIdx.x; c < in_f; c += blockDim.x) {
-            unsigned int key;
-            if (key_of(c, key) && (key & pm) == pre) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-        }
+        count(prefix, pmask, shift);
         __syncthreads();
         // The bin that holds the `want`-th element, by the whole block (one bin per thread): the first bin whose running
         // count reaches `want`, the last bin if none does.  A prefix count over the block (shuffles, then one count per
@@ -583,7 +580,12 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
     };
     // trim: the kept weights with the smallest magnitudes go; otherwise the free positions with the largest gradient
     // magnitudes come
-    row_select(in_f, m, key_of, hist, &cut);
+    row_select(m, [&](unsigned int pre, unsigned int pm, int shift) {
+        for (int c = threadIdx.x; c < in_f; c += blockDim.x) {
+            unsigned int key;
+            if (key_of(c, key) && (key & pm) == pre) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+    }, hist, &cut);
     // Apply, walking the row in column order so that ties on the cut key go to the smaller columns: a tie's rank is
     // the ties of the chunks before (carried by every thread), of the warps before in this chunk (one count per warp
     // in shared memory) and of the lanes before in its warp (a ballot).
@@ -627,7 +629,7 @@ __global__ void finalize_kernel(float* w, uint8_t* mask, const float* grad, cons
 // neuron's flag; mask and pruning flags, 16 bytes each; the keys, 16-byte loads of only the groups that hold candidates;
 // the weights once more for the write-back) instead of one per 256 columns and array, ties are ranked with one block-wide
 // prefix count per 4096 columns, and mask and weights go back in whole 16-byte stores.
-__global__ void __launch_bounds__(kThreads, 6) finalize_runs_kernel(float* w, uint8_t* mask, const float* grad, const uint8_t* drop, const uint8_t* survives,
+__global__ void __launch_bounds__(kThreads, 8) finalize_runs_kernel(float* w, uint8_t* mask, const float* grad, const uint8_t* drop, const uint8_t* survives,
                                      int in_f, const Scalars* sc) {
     extern __shared__ __align__(16) unsigned char row_smem[];  // keys[in_f] (4 bytes each), then state[in_f] (1 byte each)
     __shared__ unsigned int hist[256];
@@ -692,11 +694,19 @@ __global__ void __launch_bounds__(kThreads, 6) finalize_runs_kernel(float* w, ui
         }
         __syncthreads();
     }
-    auto key_of = [&](int c, unsigned int& key) {
-        key = keys[c];
-        return trim ? state[c] != 0 : state[c] == 0;
-    };
-    row_select(in_f, m, key_of, hist, &cut);
+    // Four columns per thread and step: one 16-byte read of the keys, one 4-byte read of the state bytes.
+    row_select(m, [&](unsigned int pre, unsigned int pm, int shift) {
+        const unsigned int flip_state = trim ? 0u : 0x01010101u;
+        for (int q = t; q < (in_f >> 2); q += kThreads) {
+            const unsigned int cand = reinterpret_cast<const unsigned int*>(state)[q] ^ flip_state;
+            if (cand == 0u) continue;
+            const uint4 kq = reinterpret_cast<const uint4*>(keys)[q];
+            if ((cand & 0x00000001u) && (kq.x & pm) == pre) atomicAdd(&hist[(kq.x >> shift) & 255u], 1u);
+            if ((cand & 0x00000100u) && (kq.y & pm) == pre) atomicAdd(&hist[(kq.y >> shift) & 255u], 1u);
+            if ((cand & 0x00010000u) && (kq.z & pm) == pre) atomicAdd(&hist[(kq.z >> shift) & 255u], 1u);
+            if ((cand & 0x01000000u) && (kq.w & pm) == pre) atomicAdd(&hist[(kq.w >> shift) & 255u], 1u);
+        }
+    }, hist, &cut);
     // Apply in column order, so that ties on the cut key go to the smaller columns: a tie's rank is the ties of the
     // 4096-column chunks before (carried by every thread), of the threads before in this chunk (a prefix count over the
     // block) and of the columns before in the thread's own run.
