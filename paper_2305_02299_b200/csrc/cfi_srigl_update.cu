@@ -7,7 +7,10 @@
 // pairs, ties to the smaller position", with key = the bits of |w| (a non-negative float orders like its bits) or
 // the complement of the bits of |grad| (so that a larger gradient is a smaller key).  They are done by radix
 // selection: four passes of 256-bin histograms over the digits of the key from the top, each pass narrowing to the
-// bin that holds the m-th element, then the ties on the final key are cut in position order with a prefix count.
+// bin that holds the m-th element, then the ties on the final key are cut in position order.  For the two layer-wide
+// selections the last pass also lists the few elements that match the first three digits; when a list holds them all
+// (the rule), the position of the last tie taken is selected from it and the marking pass is elementwise; inputs with
+// very many equal keys overflow the list and are ranked with per-chunk tie counts and a prefix sum instead.
 //
 // Readings where Sec. 3.1 leaves a choice (the same as the CPU oracle used by the tests takes): already ablated
 // neurons stay out; a weight is salient if it is active and not among the K smallest, or inactive and among the K
@@ -31,7 +34,19 @@ struct SelectState {
     unsigned int prefix, prefix_mask;
     unsigned int hist[256];
     unsigned int blocks_done;    // blocks of the running histogram sweep that have added their counts (first state only)
+    // The last sweep also lists the elements that match the first three digits (key, position): a few hundred as a rule.
+    // If the list holds them all, the position of the last tie taken follows from it and the marking needs no ranking.
+    unsigned int listed;         // elements offered to the list (may exceed its capacity)
+    unsigned int last_tie;       // ties on the cut key are taken up to and including this position
+    unsigned int listed_all;     // 1: last_tie is valid
 };
+
+// Capacity of a selection's list: enough for ordinary key distributions, small against the layer; inputs with very many
+// equal keys overflow it and take the ranking path.
+__host__ __device__ inline unsigned int list_capacity(long long n) {
+    const long long c = n / 64;
+    return (unsigned int)(c < 64 ? 64 : c > 32768 ? 32768 : c);
+}
 
 struct Scalars {
     long long active_total, inactive_total;
@@ -106,7 +121,8 @@ __global__ void setup_kernel(const int* row_count, int out_f, int in_f, long lon
         if (kk > act) kk = act;
         if (kk > sc->inactive_total) kk = sc->inactive_total;
         for (int s = 0; s < 2; ++s)
-            st[s].want = (unsigned long long)kk, st[s].below = 0, st[s].prefix = 0, st[s].prefix_mask = 0, st[s].blocks_done = 0;
+            st[s].want = (unsigned long long)kk, st[s].below = 0, st[s].prefix = 0, st[s].prefix_mask = 0, st[s].blocks_done = 0,
+            st[s].listed = 0, st[s].last_tie = 0, st[s].listed_all = 0;
     }
     for (int s = 0; s < 2; ++s)
         for (int b = threadIdx.x; b < 256; b += blockDim.x) st[s].hist[b] = 0;
@@ -155,26 +171,96 @@ __device__ void pick_bin(int pass, SelectState* st) {
     }
 }
 
+// The whole block (kThreads threads), one selection, after its last digit has been picked: if the list holds every
+// element that matched the first three digits, the ties on the cut key are all in it, and the position of the last tie
+// taken (the `want`-th in position order) is found by radix selection over the listed positions.  Then "taken" is
+// key < cut, or key == cut and position <= last_tie: the marking needs neither tie counts nor ranks.
+__device__ void find_last_tie(SelectState* st, const uint2* list, unsigned int cap) {
+    __shared__ unsigned int hist[256], warp_tot[kThreads / 32], res[2], ties_total;
+    const int t = threadIdx.x, lane = t & 31, wid = t >> 5;
+    const unsigned int n = __ldcg(&st->listed);
+    if (n > cap) {  // the list overflowed (the same for the whole block): the ranking path decides
+        if (t == 0) st->listed_all = 0;
+        return;
+    }
+    const unsigned int cut = __ldcg(&st->prefix);
+    unsigned int want = (unsigned int)__ldcg(&st->want);  // ties to take
+    if (t == 0) ties_total = 0;
+    __syncthreads();
+    unsigned int mine = 0;
+    for (unsigned int i = t; i < n; i += kThreads) mine += __ldcg(&list[i]).x == cut ? 1u : 0u;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, off);
+    if (lane == 0 && mine) atomicAdd(&ties_total, mine);
+    __syncthreads();
+    if (want == 0 || ties_total <= want) {  // selection off, or every tie is taken
+        if (t == 0) st->last_tie = 0xFFFFFFFFu, st->listed_all = 1;
+        return;
+    }
+    unsigned int prefix = 0, pmask = 0;
+    for (int pass = 0; pass < 4; ++pass) {
+        hist[t] = 0;
+        __syncthreads();
+        const int shift = 24 - 8 * pass;
+        for (unsigned int i = t; i < n; i += kThreads) {
+            const uint2 e = __ldcg(&list[i]);
+            if (e.x == cut && (e.y & pmask) == prefix) atomicAdd(&hist[(e.y >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        const unsigned int h = hist[t];
+        unsigned int incl = h;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned int up = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        if (lane == 31) warp_tot[wid] = incl;
+        __syncthreads();
+        unsigned int before = 0;
+#pragma unroll
+        for (int i = 0; i < kThreads / 32; ++i) before += i < wid ? warp_tot[i] : 0u;
+        const unsigned int excl = before + incl - h;
+        if (excl < want && want <= excl + h) res[0] = (unsigned int)t, res[1] = excl;  // exactly one thread: want <= ties
+        __syncthreads();
+        prefix |= res[0] << shift;
+        pmask |= 255u << shift;
+        want -= res[1];
+        __syncthreads();  // res[] and hist[] are rewritten by the next pass
+    }
+    if (t == 0) st->last_tie = prefix, st->listed_all = 1;
+}
+
 // Histograms of digit `pass` (0 = top byte) for both layer-wide selections in one sweep over the layer: over the valid
 // elements of each whose key matches the prefix found so far.  Every position is valid for at most one of the two, so
 // one histogram of 512 bins (selection * 256 + digit) serves both.  A block takes whole rows, four columns per thread
 // and step when the row length is a multiple of four (16-byte loads of w and grad, 4-byte loads of the mask).
-__global__ void hist_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int out_f, int in_f,
-                            int pass, SelectState* st) {
+template <bool LAST>  // the last sweep (pass 3) also fills the lists; the others keep their smaller code
+__global__ void __launch_bounds__(kThreads, 8) hist_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int out_f, int in_f,
+                            int pass, SelectState* st, uint2* list, unsigned int cap) {
     __shared__ unsigned int h[512];
+    __shared__ int list_full[2];
+    if (threadIdx.x < 2) list_full[threadIdx.x] = 0;
     for (int b = threadIdx.x; b < 512; b += blockDim.x) h[b] = 0;
     __syncthreads();
     const bool on0 = st[0].want != 0, on1 = st[1].want != 0;
     if (on0 || on1) {
         const unsigned int prefix0 = st[0].prefix, pmask0 = st[0].prefix_mask, prefix1 = st[1].prefix, pmask1 = st[1].prefix_mask;
         const int shift = 24 - 8 * pass;
-        auto one = [&](bool inside, uint8_t m, float wv, float gv) {  // every lane of the warp calls it the same number of times
+        auto one = [&](bool inside, uint8_t m, float wv, float gv, size_t pos) {  // every lane of the warp calls it the same number of times
             bool take = false;
             unsigned int bin = 0;
             if (inside) {
                 const unsigned int key = m ? mag_bits(wv) : ~mag_bits(gv);
                 take = m ? (on0 && (key & pmask0) == prefix0) : (on1 && (key & pmask1) == prefix1);
                 bin = (m ? 0u : 256u) + ((key >> shift) & 255u);
+                if (LAST && take) {  // the last sweep lists what it counts, while the list has room
+                    const int sel = m ? 0 : 1;
+                    if (!list_full[sel]) {
+                        const unsigned int at = atomicAdd(&st[sel].listed, 1u);
+                        if (at < cap) list[(size_t)sel * cap + at] = make_uint2(key, (unsigned int)pos);
+                        else list_full[sel] = 1;
+                    }
+                }
             }
             // The top digit falls into a handful of bins (aggregate per warp); the later digits of the few elements that
             // still match the prefix spread out, and a plain atomic is cheaper there.
@@ -199,17 +285,17 @@ __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* gr
                         wv = w4[v];
                         gv = g4[v];
                     }
-                    one(inside, m.x, wv.x, gv.x);
-                    one(inside, m.y, wv.y, gv.y);
-                    one(inside, m.z, wv.z, gv.z);
-                    one(inside, m.w, wv.w, gv.w);
+                    one(inside, m.x, wv.x, gv.x, base + 4 * (size_t)v);
+                    one(inside, m.y, wv.y, gv.y, base + 4 * (size_t)v + 1);
+                    one(inside, m.z, wv.z, gv.z, base + 4 * (size_t)v + 2);
+                    one(inside, m.w, wv.w, gv.w, base + 4 * (size_t)v + 3);
                 }
             } else {
                 for (int c0 = 0; c0 < in_f; c0 += blockDim.x) {
                     const int c = c0 + threadIdx.x;
                     const bool inside = c < in_f;
                     const uint8_t m = inside ? mask[base + c] : 0;
-                    one(inside, m, inside && m ? w[base + c] : 0.f, inside && !m ? grad[base + c] : 0.f);
+                    one(inside, m, inside && m ? w[base + c] : 0.f, inside && !m ? grad[base + c] : 0.f, base + c);
                 }
             }
         }
@@ -226,6 +312,12 @@ __global__ void hist_kernel(const float* w, const uint8_t* mask, const float* gr
     if (last) {
         __threadfence();
         if (threadIdx.x < 64) pick_bin(pass, st + (threadIdx.x >> 5));
+        if (LAST) {  // both cuts are final
+            __syncthreads();
+            find_last_tie(st, list, cap);
+            __syncthreads();
+            find_last_tie(st + 1, list + cap, cap);
+        }
         if (threadIdx.x == 0) st[0].blocks_done = 0;
     }
 }
@@ -276,6 +368,7 @@ __device__ __forceinline__ void load_run16(const float* w, const uint8_t* mask, 
 __global__ void tie_count_kernel(const float* w, const uint8_t* mask, const float* grad, const int* row_count, int in_f,
                                  long long n, const SelectState* st, unsigned int* chunk_ties, int n_chunks, bool vec_ok) {
     __shared__ unsigned int s[2];
+    if (st[0].listed_all && st[1].listed_all) return;  // the marking will not ask for tie counts
     if (threadIdx.x < 2) s[threadIdx.x] = 0;
     __syncthreads();
     const long long base = (long long)blockIdx.x * kChunk + (long long)threadIdx.x * 16;
@@ -297,7 +390,8 @@ __global__ void tie_count_kernel(const float* w, const uint8_t* mask, const floa
 }
 
 // One block per selection: exclusive prefix sum of its per-chunk tie counts, in place.
-__global__ void chunk_scan_kernel(unsigned int* chunk_ties_both, int n_chunks) {
+__global__ void chunk_scan_kernel(unsigned int* chunk_ties_both, int n_chunks, const SelectState* st) {
+    if (st[0].listed_all && st[1].listed_all) return;
     unsigned int* chunk_ties = chunk_ties_both + (size_t)blockIdx.x * n_chunks;
     __shared__ unsigned long long warp_tot[kThreads / 32];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -348,38 +442,51 @@ __global__ void mark_kernel(const float* w, const uint8_t* mask, const float* gr
     uint8_t kind[16];  // 0: in neither pool, 1: active weight, 2: inactive position of a live neuron
     unsigned int mine0 = 0, mine1 = 0;
     load_run16(w, mask, grad, row_count, in_f, n, base, vec_ok, keys, kind);
-#pragma unroll
-    for (int e = 0; e < 16; ++e) {
-        if (kind[e] == 1 && want0 != 0 && keys[e] == cut0) ++mine0;
-        if (kind[e] == 2 && want1 != 0 && keys[e] == cut1) ++mine1;
-    }
-    part[0][threadIdx.x] = mine0;
-    part[1][threadIdx.x] = mine1;
-    __syncthreads();
-    for (int off = 1; off < kThreads; off <<= 1) {
-        const unsigned int add0 = threadIdx.x >= off ? part[0][threadIdx.x - off] : 0u;
-        const unsigned int add1 = threadIdx.x >= off ? part[1][threadIdx.x - off] : 0u;
-        __syncthreads();
-        part[0][threadIdx.x] += add0;
-        part[1][threadIdx.x] += add1;
-        __syncthreads();
-    }
-    // ties of each selection before this thread's first element
-    unsigned long long rank0 = (unsigned long long)chunk_ties[blockIdx.x] + part[0][threadIdx.x] - mine0;
-    unsigned long long rank1 = (unsigned long long)chunk_ties[(size_t)n_chunks + blockIdx.x] + part[1][threadIdx.x] - mine1;
     unsigned int d16[4] = {0u, 0u, 0u, 0u}, g16[4] = {0u, 0u, 0u, 0u};  // the 16 flags of each kind, one byte each
+    if (st[0].listed_all && st[1].listed_all) {
+        // Both lists held every candidate of the last digit: a tie is taken up to a known position, nothing to rank.
+        const unsigned int last0 = st[0].last_tie, last1 = st[1].last_tie;
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-        unsigned int f0 = 0, f1 = 0;
-        if (kind[e] == 1 && want0 != 0) {
-            if (keys[e] < cut0) f0 = 1;
-            else if (keys[e] == cut0) f0 = rank0++ < want0 ? 1 : 0;
-        } else if (kind[e] == 2 && want1 != 0) {
-            if (keys[e] < cut1) f1 = 1;
-            else if (keys[e] == cut1) f1 = rank1++ < want1 ? 1 : 0;
+        for (int e = 0; e < 16; ++e) {
+            const unsigned int pos = (unsigned int)(base + e);
+            const unsigned int f0 = (kind[e] == 1 && want0 != 0 && (keys[e] < cut0 || (keys[e] == cut0 && pos <= last0))) ? 1u : 0u;
+            const unsigned int f1 = (kind[e] == 2 && want1 != 0 && (keys[e] < cut1 || (keys[e] == cut1 && pos <= last1))) ? 1u : 0u;
+            d16[e >> 2] |= f0 << (8 * (e & 3));
+            g16[e >> 2] |= f1 << (8 * (e & 3));
         }
-        d16[e >> 2] |= f0 << (8 * (e & 3));
-        g16[e >> 2] |= f1 << (8 * (e & 3));
+    } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            if (kind[e] == 1 && want0 != 0 && keys[e] == cut0) ++mine0;
+            if (kind[e] == 2 && want1 != 0 && keys[e] == cut1) ++mine1;
+        }
+        part[0][threadIdx.x] = mine0;
+        part[1][threadIdx.x] = mine1;
+        __syncthreads();
+        for (int off = 1; off < kThreads; off <<= 1) {
+            const unsigned int add0 = threadIdx.x >= off ? part[0][threadIdx.x - off] : 0u;
+            const unsigned int add1 = threadIdx.x >= off ? part[1][threadIdx.x - off] : 0u;
+            __syncthreads();
+            part[0][threadIdx.x] += add0;
+            part[1][threadIdx.x] += add1;
+            __syncthreads();
+        }
+        // ties of each selection before this thread's first element
+        unsigned long long rank0 = (unsigned long long)chunk_ties[blockIdx.x] + part[0][threadIdx.x] - mine0;
+        unsigned long long rank1 = (unsigned long long)chunk_ties[(size_t)n_chunks + blockIdx.x] + part[1][threadIdx.x] - mine1;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            unsigned int f0 = 0, f1 = 0;
+            if (kind[e] == 1 && want0 != 0) {
+                if (keys[e] < cut0) f0 = 1;
+                else if (keys[e] == cut0) f0 = rank0++ < want0 ? 1 : 0;
+            } else if (kind[e] == 2 && want1 != 0) {
+                if (keys[e] < cut1) f1 = 1;
+                else if (keys[e] == cut1) f1 = rank1++ < want1 ? 1 : 0;
+            }
+            d16[e >> 2] |= f0 << (8 * (e & 3));
+            g16[e >> 2] |= f1 << (8 * (e & 3));
+        }
     }
     if (vec_ok && base + 16 <= n) {
         *reinterpret_cast<uint4*>(drop + base) = make_uint4(d16[0], d16[1], d16[2], d16[3]);
@@ -787,6 +894,7 @@ struct Workspace {
     uint8_t* drop;
     uint8_t* grow_top;
     unsigned int* chunk_ties;
+    uint2* list;            // 2 x list_capacity(n) (key, position) pairs
     SelectState* state;
     Scalars* scalars;
     size_t bytes;
@@ -807,6 +915,7 @@ Workspace carve(void* base, int out_f, int in_f) {
     w.drop = reinterpret_cast<uint8_t*>(take(n));
     w.grow_top = reinterpret_cast<uint8_t*>(take(n));
     w.chunk_ties = reinterpret_cast<unsigned int*>(take(2 * chunks * 4));
+    w.list = reinterpret_cast<uint2*>(take(2 * (size_t)list_capacity((long long)n) * sizeof(uint2)));
     w.state = reinterpret_cast<SelectState*>(take(2 * sizeof(SelectState)));
     w.scalars = reinterpret_cast<Scalars*>(take(sizeof(Scalars)));
     w.bytes = off;
@@ -819,14 +928,19 @@ bool layer_select_both(const float* w, const uint8_t* mask, const float* grad, c
     const int chunks = (int)((n + kChunk - 1) / kChunk);
     const int hist_blocks = out_f < 1184 ? out_f : 1184;  // whole rows per block, 8 CTAs per SM at most
     for (int pass = 0; pass < 4; ++pass) {
-        hist_kernel<<<hist_blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, out_f, in_f, pass, ws.state);
+        if (pass < 3)
+            hist_kernel<false><<<hist_blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, out_f, in_f, pass, ws.state, ws.list,
+                                                                 list_capacity(n));
+        else
+            hist_kernel<true><<<hist_blocks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, out_f, in_f, pass, ws.state, ws.list,
+                                                                list_capacity(n));
     }
     // 16-byte loads and stores of a thread's run of 16 positions: the run must lie inside one row, and the arrays (the
     // workspace's flag arrays are 256-byte aligned) must start on 16-byte boundaries.
     const bool vec_ok = (in_f % 16) == 0 && ((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(grad) |
                                                reinterpret_cast<uintptr_t>(mask)) & 15u) == 0;
     tie_count_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks, vec_ok);
-    chunk_scan_kernel<<<2, kThreads, 0, st>>>(ws.chunk_ties, chunks);
+    chunk_scan_kernel<<<2, kThreads, 0, st>>>(ws.chunk_ties, chunks, ws.state);
     mark_kernel<<<chunks, kThreads, 0, st>>>(w, mask, grad, ws.row_count, in_f, n, ws.state, ws.chunk_ties, chunks, ws.drop,
                                              ws.grow_top, vec_ok);
     return cudaGetLastError() == cudaSuccess;

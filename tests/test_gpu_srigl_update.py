@@ -78,6 +78,19 @@ def test_many_ties(seed):
     _compare(w, m, g, int(rng.integers(0, out_f * k + 1)), float(rng.choice([0.0, 0.25, 0.5, 1.0])))
 
 
+@pytest.mark.parametrize("levels", [3, 4096])
+def test_ties_with_and_without_room_in_the_candidate_list(levels):
+    """300 x 1024 with magnitudes and gradients quantised to `levels` values.  With 3 levels a third of the layer
+    equals the cut key: far more than the list of the last digit's candidates holds (4800 entries), so ties are ranked
+    by the counting path; with 4096 levels the ties at the cut fit the list and the marking takes them up to a position.
+    Both must equal the oracle bit for bit."""
+    w, m, g = _layer(300, 1024, 100, 7, seed=77)
+    q = float(levels)
+    w = (np.ceil(np.abs(w) * q / 4) * 4 / q * np.sign(w) * (m == 1)).astype(np.float32)
+    g = (np.round(g * q / 8) * 8 / q).astype(np.float32)
+    _compare(w, m, g, 9000, 0.3)
+
+
 def test_workspace_and_argument_checks():
     import ctypes
     import torch
