@@ -57,6 +57,17 @@ cfi_slab_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int ba
     // and where its quads start in each of this CTA's slabs (an ablated row has none).  Then every row's run of quads
     // is asked into L2 at once.  None of this belongs to an earlier kernel, so it all happens before the wait.
     const int nsl = slab_hi - slab_lo;
+    // x may belong to the kernel ahead and must not be read before that kernel is done; asking for this CTA's part of
+    // it to be brought into L2 reads nothing (L2 is where that kernel's writes land, so nothing stale can be kept), and
+    // a cold x is then on chip when the wait returns.  One request per batch row, addresses and sizes rounded to 16
+    // bytes, by the threads of the last warp: a request takes the issuing thread about a microsecond, which the first
+    // warps spend on the row table instead.
+    if (tid >= kSlabThreads - 32 && tid - (kSlabThreads - 32) < nb && ncols > 0) {
+        const int b = tid - (kSlabThreads - 32);
+        const uintptr_t p0 = reinterpret_cast<uintptr_t>(x + (size_t)(b0 + b) * L.in + col_lo), p1 = p0 + (size_t)ncols * sizeof(VT);
+        const uintptr_t lo = p0 & ~(uintptr_t)15, hi = min((p1 + 15) & ~(uintptr_t)15, reinterpret_cast<uintptr_t>(x + (size_t)batch * L.in) & ~(uintptr_t)15);
+        if (hi > lo) prefetch_l2(reinterpret_cast<const void*>(lo), (uint32_t)(hi - lo));
+    }
     // Every row's quads (all slabs: the cluster's CTAs need them between them) are asked into L2 by the first CTA of the
     // cluster, straight from the row table in global memory, while the metadata below is still on its way.
     if (split == 0)
@@ -87,14 +98,6 @@ cfi_slab_kernel(DevLayer L, const VT* __restrict__ x, VT* __restrict__ y, int ba
         }
     }
     __syncthreads();
-    // x may belong to the kernel ahead and must not be read before that kernel is done; asking for this CTA's part of
-    // it to be brought into L2 reads nothing (L2 is where that kernel's writes land, so nothing stale can be kept), and
-    // a cold x is then on chip when the wait returns.  One request per batch row; addresses and sizes rounded to 16 bytes.
-    if (tid < nb && ncols > 0) {
-        const uintptr_t p0 = reinterpret_cast<uintptr_t>(x + (size_t)(b0 + tid) * L.in + col_lo), p1 = p0 + (size_t)ncols * sizeof(VT);
-        const uintptr_t lo = p0 & ~(uintptr_t)15, hi = min((p1 + 15) & ~(uintptr_t)15, reinterpret_cast<uintptr_t>(x + (size_t)batch * L.in) & ~(uintptr_t)15);
-        if (hi > lo) prefetch_l2(reinterpret_cast<const void*>(lo), (uint32_t)(hi - lo));
-    }
     pdl_wait();  // x and y may belong to the kernel before this one
 
     // Stage x[b0 .. b0+15][col_lo .. col_lo+ncols) as xs[column][16]: a thread takes two columns at a time, 32 loads
